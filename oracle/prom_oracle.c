@@ -1,0 +1,270 @@
+/*
+ * CPU oracle for the ternary pointwise-convolution path of PROM.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain-loop statement of
+ * what the path computes.  It shares no code with the CUDA library and must
+ * never be called by it; only the tests, the smoke check and the benchmark's
+ * CPU-baseline leg may use it.  Nothing here is blocked, fused, vectorised by
+ * hand or reordered: every function is the definition written out so that it
+ * can be checked against the paper by eye.  Rows are split over OpenMP
+ * threads and that is the only parallelism.
+ *
+ * Notation (paper, Section 3.1): X is the int8 activation matrix [M, Cin]
+ * (NHWC pixels flattened to rows), W-hat is the ternary weight matrix
+ * [Cout, Cin] with entries in {-1, 0, +1}, and the layer output before
+ * scaling is  acc[m][o] = sum_k X[m][k] * W-hat[o][k]   (Section 3.1,
+ * inference form: the input is convolved directly with the ternary weights
+ * and scaled afterwards; Figure 12, inference branch).
+ *
+ * The paper scales the integer result by the per-output-channel factor alpha
+ * and the activation scale in floating point (Figure 12).  The build's
+ * contract replaces that by a static fixed-point requantisation per output
+ * channel; the reading taken is
+ *     t = acc + bias[o]
+ *     p = t * mult[o]                    (exact, 64-bit)
+ *     q = sign(p) * floor((|p| + 2^(s-1)) / 2^s),   s = 31 + shift[o]
+ *     y = min(act_max, max(act_min, q))
+ * i.e. one rounding of the exact product, ties away from zero.
+ *
+ * Pins (tests/test_oracle_*.py): brute force over all ternary matrices on
+ * tiny shapes against Python big integers, the add/sub identity of Section 2,
+ * all-zero and one-hot weights, an int64 library matmul, exact rational
+ * arithmetic for the requantiser, hand-built ties, and byte tables for the
+ * 2-bit codes.  No function in this file is "parity unpinned".
+ */
+#include <stdint.h>
+#include <stddef.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---- threads ----------------------------------------------------------- */
+
+int prom_ref_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void prom_ref_set_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* ---- 2-bit storage of ternary weights ---------------------------------- */
+/*
+ * The paper stores a ternary weight in 2 bits (Section 4, "Memory"; the
+ * storage column of Table 1 is consistent with it) but prints no format.
+ * Reading taken: the 2-bit two's-complement code of the value
+ *     0 -> 00,  +1 -> 01,  -1 -> 11,  (10 is never produced and is invalid)
+ * four codes per byte along Cin, weight k of output channel o in byte
+ * o*ceil(Cin/4) + k/4 at bits 2*(k%4) and 2*(k%4)+1; a row is padded to a
+ * whole byte with code 00.
+ */
+
+size_t prom_ref_packed_bytes(int cout, int cin)
+{
+    return (size_t)cout * (size_t)((cin + 3) / 4);
+}
+
+/* Returns the number of entries of w that are not in {-1,0,+1}; packed is
+ * written only when that number is 0. */
+long prom_ref_pack(const int8_t *w, int cout, int cin, uint8_t *packed)
+{
+    long bad = 0;
+    for (long i = 0; i < (long)cout * cin; ++i)
+        if (w[i] < -1 || w[i] > 1) ++bad;
+    if (bad) return bad;
+    int rowb = (cin + 3) / 4;
+    memset(packed, 0, (size_t)cout * rowb);
+    for (int o = 0; o < cout; ++o)
+        for (int k = 0; k < cin; ++k) {
+            int v = w[(long)o * cin + k];
+            unsigned code = (v == 0) ? 0u : (v == 1 ? 1u : 3u);
+            packed[(long)o * rowb + k / 4] |= (uint8_t)(code << (2 * (k % 4)));
+        }
+    return 0;
+}
+
+/* Returns the number of invalid codes (10) met, padding codes that are not 00
+ * included; w is written in any case (an invalid code decodes to 0). */
+long prom_ref_unpack(const uint8_t *packed, int cout, int cin, int8_t *w)
+{
+    long bad = 0;
+    int rowb = (cin + 3) / 4;
+    for (int o = 0; o < cout; ++o)
+        for (int k = 0; k < rowb * 4; ++k) {
+            unsigned code = (packed[(long)o * rowb + k / 4] >> (2 * (k % 4))) & 3u;
+            int v = 0;
+            if (code == 1u) v = 1;
+            else if (code == 3u) v = -1;
+            else if (code == 2u) ++bad;
+            if (k < cin) w[(long)o * cin + k] = (int8_t)v;
+            else if (code != 0u && code != 2u) ++bad;
+        }
+    return bad;
+}
+
+/* ---- requantisation ----------------------------------------------------- */
+
+int32_t prom_ref_requant_scalar(int32_t t, int32_t mult, int shift,
+                                int act_min, int act_max)
+{
+    int64_t p = (int64_t)t * (int64_t)mult;
+    int s = 31 + shift;
+    int64_t half = (int64_t)1 << (s - 1);
+    int64_t a = p < 0 ? -p : p;
+    int64_t q = (a + half) >> s;          /* a + half >= 0: the shift is a floor */
+    if (p < 0) q = -q;
+    if (q < act_min) q = act_min;
+    if (q > act_max) q = act_max;
+    return (int32_t)q;
+}
+
+void prom_ref_requant(const int32_t *t, long n, int32_t mult, int shift,
+                      int act_min, int act_max, int32_t *q)
+{
+    for (long i = 0; i < n; ++i)
+        q[i] = prom_ref_requant_scalar(t[i], mult, shift, act_min, act_max);
+}
+
+/* ---- the convolution, multiply form ------------------------------------- */
+/*
+ * x: [m, cin] int8, rows `x_row_stride` bytes apart (cin when dense);
+ * w: [cout, cin] int8 with ternary values; acc (optional): [m, cout] int32;
+ * y (optional): [m, cout] int8.  bias/mult/shift: [cout].
+ */
+void prom_ref_conv_mul(const int8_t *x, long m, int cin, long x_row_stride,
+                       const int8_t *w, int cout,
+                       const int32_t *bias, const int32_t *mult, const int8_t *shift,
+                       int act_min, int act_max,
+                       int32_t *acc_out, int8_t *y)
+{
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < m; ++r) {
+        const int8_t *xr = x + r * x_row_stride;
+        for (int o = 0; o < cout; ++o) {
+            const int8_t *wo = w + (long)o * cin;
+            int32_t acc = 0;
+            for (int k = 0; k < cin; ++k)
+                acc += (int32_t)xr[k] * (int32_t)wo[k];
+            if (acc_out) acc_out[r * cout + o] = acc;
+            if (y) {
+                int32_t t = acc + bias[o];
+                y[r * cout + o] = (int8_t)prom_ref_requant_scalar(
+                    t, mult[o], shift[o], act_min, act_max);
+            }
+        }
+    }
+}
+
+/* ---- the convolution, add/subtract form (Section 2: a product with a
+ * ternary weight reduces to a sum of input channels) ---------------------- */
+void prom_ref_conv_addsub(const int8_t *x, long m, int cin, long x_row_stride,
+                          const int8_t *w, int cout,
+                          const int32_t *bias, const int32_t *mult, const int8_t *shift,
+                          int act_min, int act_max,
+                          int32_t *acc_out, int8_t *y)
+{
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < m; ++r) {
+        const int8_t *xr = x + r * x_row_stride;
+        for (int o = 0; o < cout; ++o) {
+            const int8_t *wo = w + (long)o * cin;
+            int32_t plus = 0, minus = 0;
+            for (int k = 0; k < cin; ++k) {
+                if (wo[k] == 1) plus += xr[k];
+                else if (wo[k] == -1) minus += xr[k];
+                /* a zero weight needs no work */
+            }
+            int32_t acc = plus - minus;
+            if (acc_out) acc_out[r * cout + o] = acc;
+            if (y) {
+                int32_t t = acc + bias[o];
+                y[r * cout + o] = (int8_t)prom_ref_requant_scalar(
+                    t, mult[o], shift[o], act_min, act_max);
+            }
+        }
+    }
+}
+
+/* ---- spatial subsampling: the depthwise stand-in ------------------------ */
+/*
+ * The depthwise 3x3 convolution between expand and project (Section 2) is
+ * modelled as the identity on values plus its spatial stride: output pixel
+ * (i, j) of a stride-2 site is input pixel (2i, 2j).  in: [batch, h, w, c],
+ * out: [batch, h/stride, w/stride, c].
+ */
+void prom_ref_subsample(const int8_t *in, int batch, int h, int w, int c,
+                        int stride, int8_t *out)
+{
+    int ho = h / stride, wo = w / stride;
+    for (int b = 0; b < batch; ++b)
+        for (int i = 0; i < ho; ++i)
+            for (int j = 0; j < wo; ++j)
+                memcpy(out + (((long)b * ho + i) * wo + j) * c,
+                       in + (((long)b * h + i * stride) * w + j * stride) * c,
+                       (size_t)c);
+}
+
+/* ---- the layer sequence -------------------------------------------------- */
+/*
+ * Runs n pointwise layers back to back: the output of layer i is the input
+ * of layer i+1; a layer with in_stride 2 reads pixel (2i, 2j) of its input
+ * for its own pixel (i, j), in place of materialising the subsampled tensor.
+ * cin/cout/in_stride: [n]; w: n pointers to ternary [cout, cin];
+ * bias/mult/shift: n pointers to [cout] arrays.  Returns 0, or -1 when the
+ * shapes do not chain or a buffer cannot be had.
+ */
+int prom_ref_layer_seq(int n, const int *cin, const int *cout, const int *in_stride,
+                       const int8_t *const *w,
+                       const int32_t *const *bias, const int32_t *const *mult,
+                       const int8_t *const *shift,
+                       int act_min, int act_max,
+                       const int8_t *x0, int batch, int h0, int w0,
+                       int8_t *y_out)
+{
+    int h = h0, wd = w0;
+    const int8_t *cur = x0;
+    int8_t *own = NULL;
+    for (int l = 0; l < n; ++l) {
+        if (l > 0 && cin[l] != cout[l - 1]) { free(own); return -1; }
+        int st = in_stride[l];
+        if (st != 1 && st != 2) { free(own); return -1; }
+        if (h % st || wd % st) { free(own); return -1; }
+        int ho = h / st, wo = wd / st;
+        long m = (long)batch * ho * wo;
+        int8_t *dst = (l == n - 1) ? y_out : (int8_t *)malloc((size_t)m * cout[l]);
+        if (!dst) { free(own); return -1; }
+#pragma omp parallel for schedule(static)
+        for (long r = 0; r < m; ++r) {
+            long b = r / ((long)ho * wo);
+            long ij = r % ((long)ho * wo);
+            long i = ij / wo, j = ij % wo;
+            const int8_t *xr = cur + (((long)b * h + i * st) * wd + j * st) * cin[l];
+            for (int o = 0; o < cout[l]; ++o) {
+                const int8_t *wl = w[l] + (long)o * cin[l];
+                int32_t acc = 0;
+                for (int k = 0; k < cin[l]; ++k)
+                    acc += (int32_t)xr[k] * (int32_t)wl[k];
+                dst[r * cout[l] + o] = (int8_t)prom_ref_requant_scalar(
+                    acc + bias[l][o], mult[l][o], shift[l][o], act_min, act_max);
+            }
+        }
+        free(own);
+        own = (l == n - 1) ? NULL : dst;
+        cur = dst;
+        h = ho; wd = wo;
+    }
+    return 0;
+}

@@ -1,0 +1,188 @@
+"""ctypes front end of the CPU oracle (``prom_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's
+CPU-baseline leg import this; the CUDA library and its binding never do.
+Arrays are numpy; nothing here computes anything, it only marshals arguments.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "prom_oracle.c")
+_LIB = os.path.join(_HERE, "libprom_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (``-O2 -fopenmp``) unless it is up to date."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-shared", "-fPIC",
+                           "-Wall", "-o", tmp, _SRC])
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        i8p, u8p, i32p = C.POINTER(C.c_int8), C.POINTER(C.c_uint8), C.POINTER(C.c_int32)
+        L.prom_ref_threads.restype = C.c_int
+        L.prom_ref_set_threads.argtypes = [C.c_int]
+        L.prom_ref_packed_bytes.restype = C.c_size_t
+        L.prom_ref_packed_bytes.argtypes = [C.c_int, C.c_int]
+        L.prom_ref_pack.restype = C.c_long
+        L.prom_ref_pack.argtypes = [i8p, C.c_int, C.c_int, u8p]
+        L.prom_ref_unpack.restype = C.c_long
+        L.prom_ref_unpack.argtypes = [u8p, C.c_int, C.c_int, i8p]
+        L.prom_ref_requant_scalar.restype = C.c_int32
+        L.prom_ref_requant_scalar.argtypes = [C.c_int32, C.c_int32, C.c_int, C.c_int, C.c_int]
+        L.prom_ref_requant.argtypes = [i32p, C.c_long, C.c_int32, C.c_int, C.c_int, C.c_int, i32p]
+        conv = [i8p, C.c_long, C.c_int, C.c_long, i8p, C.c_int, i32p, i32p, i8p,
+                C.c_int, C.c_int, i32p, i8p]
+        L.prom_ref_conv_mul.argtypes = conv
+        L.prom_ref_conv_addsub.argtypes = conv
+        L.prom_ref_subsample.argtypes = [i8p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, i8p]
+        L.prom_ref_layer_seq.restype = C.c_int
+        L.prom_ref_layer_seq.argtypes = [
+            C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
+            C.POINTER(i8p), C.POINTER(i32p), C.POINTER(i32p), C.POINTER(i8p),
+            C.c_int, C.c_int, i8p, C.c_int, C.c_int, C.c_int, i8p]
+        _lib = L
+    return _lib
+
+
+def _p(a, ct):
+    return a.ctypes.data_as(C.POINTER(ct))
+
+
+def _c(a, dt):
+    a = np.ascontiguousarray(a, dtype=dt)
+    return a
+
+
+def threads() -> int:
+    return int(lib().prom_ref_threads())
+
+
+def set_threads(n: int) -> None:
+    lib().prom_ref_set_threads(int(n))
+
+
+def packed_bytes(cout: int, cin: int) -> int:
+    return int(lib().prom_ref_packed_bytes(cout, cin))
+
+
+def pack(w) -> np.ndarray:
+    """Ternary int8 [cout, cin] -> 2-bit codes [cout, ceil(cin/4)] (uint8).
+    Raises ValueError when an entry is outside {-1, 0, +1}."""
+    w = _c(w, np.int8)
+    cout, cin = w.shape
+    out = np.zeros((cout, (cin + 3) // 4), dtype=np.uint8)
+    bad = lib().prom_ref_pack(_p(w, C.c_int8), cout, cin, _p(out, C.c_uint8))
+    if bad:
+        raise ValueError(f"{bad} weight(s) outside {{-1,0,+1}}")
+    return out
+
+
+def unpack(packed, cout: int, cin: int):
+    """2-bit codes -> (ternary int8 [cout, cin], number of invalid codes)."""
+    packed = _c(packed, np.uint8).reshape(cout, (cin + 3) // 4)
+    w = np.zeros((cout, cin), dtype=np.int8)
+    bad = lib().prom_ref_unpack(_p(packed, C.c_uint8), cout, cin, _p(w, C.c_int8))
+    return w, int(bad)
+
+
+def requant_scalar(t: int, mult: int, shift: int, act_min: int = 0, act_max: int = 127) -> int:
+    return int(lib().prom_ref_requant_scalar(int(t), int(mult), int(shift), act_min, act_max))
+
+
+def requant(t, mult: int, shift: int, act_min: int = 0, act_max: int = 127) -> np.ndarray:
+    t = _c(t, np.int32).ravel()
+    q = np.empty_like(t)
+    lib().prom_ref_requant(_p(t, C.c_int32), t.size, int(mult), int(shift), act_min, act_max,
+                           _p(q, C.c_int32))
+    return q
+
+
+def _conv(fn, x, w, bias, mult, shift, act_min, act_max, want_acc, want_y):
+    x = _c(x, np.int8)
+    w = _c(w, np.int8)
+    m, cin = x.shape
+    cout, cin2 = w.shape
+    assert cin == cin2
+    bias = _c(bias, np.int32)
+    mult = _c(mult, np.int32)
+    shift = _c(shift, np.int8)
+    assert bias.size == cout and mult.size == cout and shift.size == cout
+    acc = np.empty((m, cout), dtype=np.int32) if want_acc else None
+    y = np.empty((m, cout), dtype=np.int8) if want_y else None
+    fn(_p(x, C.c_int8), m, cin, cin, _p(w, C.c_int8), cout,
+       _p(bias, C.c_int32), _p(mult, C.c_int32), _p(shift, C.c_int8),
+       act_min, act_max,
+       _p(acc, C.c_int32) if want_acc else None,
+       _p(y, C.c_int8) if want_y else None)
+    return acc, y
+
+
+def conv_mul(x, w, bias, mult, shift, act_min=0, act_max=127, want_acc=False):
+    """Multiply form. Returns y [m, cout] int8 (and acc int32 when want_acc)."""
+    acc, y = _conv(lib().prom_ref_conv_mul, x, w, bias, mult, shift, act_min, act_max,
+                   want_acc, True)
+    return (y, acc) if want_acc else y
+
+
+def conv_addsub(x, w, bias, mult, shift, act_min=0, act_max=127, want_acc=False):
+    """Add/subtract form of the same layer."""
+    acc, y = _conv(lib().prom_ref_conv_addsub, x, w, bias, mult, shift, act_min, act_max,
+                   want_acc, True)
+    return (y, acc) if want_acc else y
+
+
+def subsample(x, stride: int) -> np.ndarray:
+    x = _c(x, np.int8)
+    b, h, w, c = x.shape
+    out = np.empty((b, h // stride, w // stride, c), dtype=np.int8)
+    lib().prom_ref_subsample(_p(x, C.c_int8), b, h, w, c, stride, _p(out, C.c_int8))
+    return out
+
+
+def layer_seq(layers, x0, act_min=0, act_max=127) -> np.ndarray:
+    """layers: list of dicts with cin, cout, in_stride, w (ternary int8 [cout, cin]),
+    bias, mult, shift.  x0: [batch, h0, w0, cin0] int8.  Returns the last
+    layer's output [batch, h, w, cout]."""
+    x0 = _c(x0, np.int8)
+    batch, h0, w0, c0 = x0.shape
+    n = len(layers)
+    assert c0 == layers[0]["cin"]
+    ws = [_c(l["w"], np.int8) for l in layers]
+    bs = [_c(l["bias"], np.int32) for l in layers]
+    ms = [_c(l["mult"], np.int32) for l in layers]
+    ss = [_c(l["shift"], np.int8) for l in layers]
+    IA = C.c_int * n
+    cin = IA(*[int(l["cin"]) for l in layers])
+    cout = IA(*[int(l["cout"]) for l in layers])
+    st = IA(*[int(l["in_stride"]) for l in layers])
+    i8p, i32p = C.POINTER(C.c_int8), C.POINTER(C.c_int32)
+    wp = (i8p * n)(*[_p(a, C.c_int8) for a in ws])
+    bp = (i32p * n)(*[_p(a, C.c_int32) for a in bs])
+    mp = (i32p * n)(*[_p(a, C.c_int32) for a in ms])
+    sp = (i8p * n)(*[_p(a, C.c_int8) for a in ss])
+    h, w = h0, w0
+    for l in layers:
+        h //= l["in_stride"]
+        w //= l["in_stride"]
+    y = np.empty((batch, h, w, layers[-1]["cout"]), dtype=np.int8)
+    rc = lib().prom_ref_layer_seq(n, cin, cout, st, wp, bp, mp, sp, act_min, act_max,
+                                  _p(x0, C.c_int8), batch, h0, w0, _p(y, C.c_int8))
+    if rc != 0:
+        raise ValueError("layer sequence does not chain")
+    return y
