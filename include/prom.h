@@ -1,0 +1,190 @@
+/*
+ * prom.h -- C ABI of the B200 (sm_100a) ternary pointwise-convolution library.
+ *
+ * The library computes the inference form of PROM's quantised 1x1 convolution
+ * (paper, Section 3.1 and Figure 12, inference branch): int8 activations are
+ * convolved directly with ternary weights W-hat in {-1,0,+1}^{Cout x Cin}, so
+ * that every product is a signed copy of an input value (Section 2), and the
+ * integer result is scaled per output channel afterwards.
+ *
+ * Layout: activations are NHWC, i.e. a row-major matrix X[M][Cin] with
+ * M = batch*H*W; the output is Y[M][Cout]; weights are [Cout][Cin].
+ *
+ * For every row m and output channel o the library returns exactly
+ *
+ *     acc = sum_k X[m][k] * W[o][k]                       (int32, exact)
+ *     t   = acc + bias[o]
+ *     p   = t * mult[o]                                   (exact)
+ *     q   = sign(p) * floor((|p| + 2^(s-1)) / 2^s),  s = 31 + shift[o]
+ *     Y[m][o] = min(act_max, max(act_min, q))
+ *
+ * The paper applies the per-channel weight scale and the activation scale in
+ * floating point (Figure 12: "dequantize after convolution"); this library
+ * takes them, with BatchNorm and the next layer's activation scale folded in,
+ * as the fixed-point pair (mult, shift): one rounding of the exact product,
+ * ties away from zero.  Integer sums and this rounding are exact, so there is
+ * one correct byte per output.
+ *
+ * General conventions
+ *   - Every pointer named *_dev is device memory of the current CUDA device,
+ *     owned by the caller; *_host is host memory (pinned for overlap).
+ *   - The library allocates nothing the caller must free.  It keeps small
+ *     internal caches (tensor-map plans, index lists of the add/sub variant)
+ *     that prom_shutdown() releases.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Convolution calls are asynchronous on that stream.
+ *   - Errors are return codes; nothing aborts or traps.  Argument errors are
+ *     found on the host before any launch.  Conditions only the device can
+ *     see (constants out of range, a bounded wait that ran out) are recorded
+ *     in a device status word read by prom_last_device_status().
+ *   - Calls are re-entrant across streams; two calls that write the same
+ *     output race like any two kernels would.
+ */
+#ifndef PROM_H_
+#define PROM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PROM_OK = 0,
+    PROM_ERR_NULL,         /* a required pointer is NULL */
+    PROM_ERR_SHAPE,        /* a size is non-positive, too large, or shapes do not chain */
+    PROM_ERR_ALIGN,        /* a base pointer is not 16-byte aligned */
+    PROM_ERR_BAD_WEIGHT,   /* a weight outside {-1,0,+1} / an invalid 2-bit code */
+    PROM_ERR_BAD_REQUANT,  /* mult/shift/bias/clamp outside the documented range */
+    PROM_ERR_WORKSPACE,    /* workspace too small */
+    PROM_ERR_UNSUPPORTED,  /* the requested variant cannot run this shape */
+    PROM_ERR_CUDA,         /* a CUDA runtime/driver call failed */
+    PROM_ERR_TIMEOUT       /* a bounded device-side wait ran out */
+} prom_status;
+
+typedef enum {
+    PROM_VARIANT_AUTO = 0, /* the library picks TC where it applies, else SMALLK, else NAIVE */
+    PROM_VARIANT_TC,       /* TMA + tcgen05 int8 MMA into TMEM, fused epilogue */
+    PROM_VARIANT_SMALLK,   /* CUDA-core dot products for small Cin */
+    PROM_VARIANT_ADDSUB,   /* additions and subtractions only on activation values */
+    PROM_VARIANT_NAIVE     /* one thread per output, plain loops (tests) */
+} prom_variant;
+
+/* Per-output-channel requantisation (stands in for the paper's division by the
+ * weight and activation scales, Figure 12).  bias/mult/shift: device arrays of
+ * `cout` entries.  Ranges: 0 <= mult < 2^31, 0 <= shift <= 31,
+ * |bias| <= 2^28, -128 <= act_min <= act_max <= 127.  The clamp is checked on
+ * the host; the arrays are checked on the device by the kernels that read
+ * them (a violation sets PROM_ERR_BAD_REQUANT in the device status word and
+ * the affected output tile is left unwritten). */
+typedef struct {
+    const int32_t *bias;
+    const int32_t *mult;
+    const int8_t  *shift;
+    int act_min, act_max;
+} prom_requant;
+
+/* One layer of a sequence.  in_stride (1 or 2) is the spatial subsampling
+ * applied to this layer's input: the depthwise convolution that sits between
+ * an expand and a project convolution (Section 2) is modelled as the identity
+ * on values plus its stride, so output pixel (i, j) reads input pixel
+ * (in_stride*i, in_stride*j). */
+typedef struct {
+    int cin, cout;
+    int in_stride;
+    const uint8_t *w_packed;   /* device, prom_packed_bytes(cout, cin) bytes */
+    prom_requant rq;
+} prom_layer;
+
+/* Bytes of the 2-bit form of a [cout][cin] ternary matrix: cout*ceil(cin/4).
+ * The paper counts a ternary weight as 2 bits of storage (Section 4, Memory;
+ * Table 1) without fixing a format; this library's is: code 00 = 0, 01 = +1,
+ * 11 = -1 (10 invalid); weight k of channel o in byte o*ceil(cin/4) + k/4 at
+ * bits 2*(k%4), 2*(k%4)+1; rows padded to a whole byte with 00. */
+size_t prom_packed_bytes(int cout, int cin);
+
+/* Packs device int8 ternary weights w_dev[cout][cin] into packed_dev.
+ * "Weights can be quantized and fixed in advance" (Figure 12): this runs once
+ * per layer, off the hot path.  Synchronises `cuda_stream`.  Returns
+ * PROM_ERR_BAD_WEIGHT (packed_dev contents then unspecified) if any value is
+ * outside {-1,0,+1}; PROM_ERR_WORKSPACE if packed_bytes is too small. */
+prom_status prom_pack_ternary(const int8_t *w_dev, int cout, int cin,
+                              uint8_t *packed_dev, size_t packed_bytes,
+                              void *cuda_stream);
+
+/* One ternary pointwise convolution with fused requantisation (Section 3.1,
+ * inference form; formula at the top of this file).
+ *   x_dev        [m][cin]  int8, dense rows, 16-byte aligned base
+ *   w_packed_dev 2-bit weights of [cout][cin], 16-byte aligned base
+ *   y_dev        [m][cout] int8, 16-byte aligned base, must not overlap x_dev
+ * m >= 0 (m == 0 is a no-op), 1 <= cin <= 4096, 1 <= cout <= 4096.
+ * TC needs cin % 8 == 0 and cout % 8 == 0 (and even m when cin or cout is not
+ * a multiple of 16); SMALLK needs cin % 4 == 0 and cin <= 64; ADDSUB and NAIVE
+ * take any shape.  An explicit variant that cannot run the shape returns
+ * PROM_ERR_UNSUPPORTED; AUTO always finds one. */
+prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin,
+                            const uint8_t *w_packed_dev, int cout,
+                            const prom_requant *rq, int8_t *y_dev,
+                            prom_variant variant, void *cuda_stream);
+
+/* Test/debug: the raw accumulators acc[m][cout] (int32) of the same layer,
+ * computed by the plain one-thread-per-output kernel. */
+prom_status prom_pw_conv_i8_acc32(const int8_t *x_dev, int64_t m, int cin,
+                                  const uint8_t *w_packed_dev, int cout,
+                                  int32_t *acc_dev, void *cuda_stream);
+
+/* Same convolution with HOST activations and output: copies x_host to the
+ * device, runs, copies the result back, all asynchronous on `cuda_stream`
+ * (pinned host memory is needed for the copies to be asynchronous).
+ * workspace_dev must hold m*cin + m*cout bytes (each rounded up to 256). */
+prom_status prom_pw_conv_i8_host(const int8_t *x_host, int64_t m, int cin,
+                                 const uint8_t *w_packed_dev, int cout,
+                                 const prom_requant *rq, int8_t *y_host,
+                                 void *workspace_dev, size_t workspace_bytes,
+                                 prom_variant variant, void *cuda_stream);
+
+/* A sequence of pointwise layers, each reading the previous one's output
+ * (the expand -> depthwise -> project block structure of Section 2 with the
+ * depthwise stage reduced to its stride).  Input x0_dev is
+ * [batch][h0][w0][layers[0].cin]; the result y_out_dev is
+ * [batch][h][w][layers[n-1].cout] with h, w divided by every in_stride.
+ * Intermediate activations live in the caller's workspace (two ping-pong
+ * regions); prom_layer_seq_workspace_bytes gives the size needed (0 on a
+ * shape error).  `variant` applies to every layer (AUTO picks per layer). */
+size_t prom_layer_seq_workspace_bytes(const prom_layer *layers, int n,
+                                      int batch, int h0, int w0);
+prom_status prom_pw_layer_seq(const prom_layer *layers, int n,
+                              const int8_t *x0_dev, int batch, int h0, int w0,
+                              void *workspace_dev, size_t workspace_bytes,
+                              int8_t *y_out_dev,
+                              prom_variant variant, void *cuda_stream);
+
+/* Same sequence with HOST input and output; the workspace must additionally
+ * hold the input and the output (prom_layer_seq_host_workspace_bytes). */
+size_t prom_layer_seq_host_workspace_bytes(const prom_layer *layers, int n,
+                                           int batch, int h0, int w0);
+prom_status prom_pw_layer_seq_host(const prom_layer *layers, int n,
+                                   const int8_t *x0_host, int batch, int h0, int w0,
+                                   void *workspace_dev, size_t workspace_bytes,
+                                   int8_t *y_out_host,
+                                   prom_variant variant, void *cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns and clears the device status word:
+ * PROM_OK, PROM_ERR_BAD_REQUANT, PROM_ERR_BAD_WEIGHT (invalid 2-bit code met
+ * by a kernel) or PROM_ERR_TIMEOUT. */
+prom_status prom_last_device_status(void *cuda_stream);
+
+/* Number of kernels this library has launched since it was loaded (all
+ * streams, this process); used by the benchmark to count launches. */
+uint64_t prom_launch_count(void);
+
+/* Frees the library's internal caches (all devices).  Optional. */
+void prom_shutdown(void);
+
+const char *prom_status_string(prom_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PROM_H_ */

@@ -1,0 +1,233 @@
+"""Thin ctypes binding over the C-ABI library (``include/prom.h``).
+
+Argument marshalling only: every function hands device (or host) pointers of
+torch tensors to the entry point of the same name; all arithmetic runs in the
+library's CUDA kernels.  There is no fallback: if the library is missing, or a
+tensor lives on the wrong device, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libprom.so")
+
+PROM_OK = 0
+(PROM_ERR_NULL, PROM_ERR_SHAPE, PROM_ERR_ALIGN, PROM_ERR_BAD_WEIGHT, PROM_ERR_BAD_REQUANT,
+ PROM_ERR_WORKSPACE, PROM_ERR_UNSUPPORTED, PROM_ERR_CUDA, PROM_ERR_TIMEOUT) = range(1, 10)
+
+VARIANTS = {"auto": 0, "tc": 1, "smallk": 2, "addsub": 3, "naive": 4}
+
+EXPORTS = [
+    "prom_packed_bytes", "prom_pack_ternary", "prom_pw_conv_i8", "prom_pw_conv_i8_acc32",
+    "prom_pw_conv_i8_host", "prom_layer_seq_workspace_bytes", "prom_pw_layer_seq",
+    "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
+    "prom_launch_count", "prom_shutdown", "prom_status_string",
+]
+
+
+class PromRequant(C.Structure):
+    _fields_ = [("bias", C.c_void_p), ("mult", C.c_void_p), ("shift", C.c_void_p),
+                ("act_min", C.c_int), ("act_max", C.c_int)]
+
+
+class PromLayer(C.Structure):
+    _fields_ = [("cin", C.c_int), ("cout", C.c_int), ("in_stride", C.c_int),
+                ("w_packed", C.c_void_p), ("rq", PromRequant)]
+
+
+class PromError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {status_string(code)} (prom_status {code})")
+        self.code = code
+
+
+_lib = None
+
+
+def lib():
+    """Loads ``libprom.so`` (built in-tree by ``build.build()``); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run paper_2505_03254_b200.build.build()")
+        L = C.CDLL(LIB_PATH)
+        vp, i64, i32, sz = C.c_void_p, C.c_int64, C.c_int, C.c_size_t
+        L.prom_packed_bytes.restype = sz
+        L.prom_packed_bytes.argtypes = [i32, i32]
+        L.prom_pack_ternary.restype = i32
+        L.prom_pack_ternary.argtypes = [vp, i32, i32, vp, sz, vp]
+        L.prom_pw_conv_i8.restype = i32
+        L.prom_pw_conv_i8.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant), vp, i32, vp]
+        L.prom_pw_conv_i8_acc32.restype = i32
+        L.prom_pw_conv_i8_acc32.argtypes = [vp, i64, i32, vp, i32, vp, vp]
+        L.prom_pw_conv_i8_host.restype = i32
+        L.prom_pw_conv_i8_host.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant), vp,
+                                           vp, sz, i32, vp]
+        L.prom_layer_seq_workspace_bytes.restype = sz
+        L.prom_layer_seq_workspace_bytes.argtypes = [C.POINTER(PromLayer), i32, i32, i32, i32]
+        L.prom_pw_layer_seq.restype = i32
+        L.prom_pw_layer_seq.argtypes = [C.POINTER(PromLayer), i32, vp, i32, i32, i32, vp, sz, vp,
+                                        i32, vp]
+        L.prom_layer_seq_host_workspace_bytes.restype = sz
+        L.prom_layer_seq_host_workspace_bytes.argtypes = [C.POINTER(PromLayer), i32, i32, i32, i32]
+        L.prom_pw_layer_seq_host.restype = i32
+        L.prom_pw_layer_seq_host.argtypes = [C.POINTER(PromLayer), i32, vp, i32, i32, i32, vp, sz,
+                                             vp, i32, vp]
+        L.prom_last_device_status.restype = i32
+        L.prom_last_device_status.argtypes = [vp]
+        L.prom_launch_count.restype = C.c_uint64
+        L.prom_shutdown.restype = None
+        L.prom_status_string.restype = C.c_char_p
+        L.prom_status_string.argtypes = [i32]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().prom_status_string(int(code)).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != PROM_OK:
+        raise PromError(code, what)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous {dtype}")
+    return t.data_ptr()
+
+
+def _variant(v) -> int:
+    return VARIANTS[v] if isinstance(v, str) else int(v)
+
+
+def packed_bytes(cout: int, cin: int) -> int:
+    return int(lib().prom_packed_bytes(cout, cin))
+
+
+def launch_count() -> int:
+    return int(lib().prom_launch_count())
+
+
+def last_device_status(stream=None) -> int:
+    return int(lib().prom_last_device_status(_stream(stream)))
+
+
+def shutdown() -> None:
+    lib().prom_shutdown()
+
+
+def pack_ternary(w: torch.Tensor, stream=None) -> torch.Tensor:
+    """prom_pack_ternary: device int8 [cout, cin] -> device uint8 [cout, ceil(cin/4)]."""
+    cout, cin = w.shape
+    out = torch.empty((cout, (cin + 3) // 4), dtype=torch.uint8, device=w.device)
+    _check(lib().prom_pack_ternary(_dev(w, torch.int8, "w"), cout, cin, out.data_ptr(),
+                                   out.numel(), _stream(stream)), "prom_pack_ternary")
+    return out
+
+
+def make_requant(bias: torch.Tensor, mult: torch.Tensor, shift: torch.Tensor,
+                 act_min: int = 0, act_max: int = 127) -> PromRequant:
+    return PromRequant(_dev(bias, torch.int32, "bias"), _dev(mult, torch.int32, "mult"),
+                       _dev(shift, torch.int8, "shift"), int(act_min), int(act_max))
+
+
+def pw_conv_i8(x: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequant,
+               y: Optional[torch.Tensor] = None, variant="auto", stream=None) -> torch.Tensor:
+    """prom_pw_conv_i8 on device tensors; x is [m, cin] int8."""
+    m, cin = x.shape
+    if y is None:
+        y = torch.empty((m, cout), dtype=torch.int8, device=x.device)
+    _check(lib().prom_pw_conv_i8(_dev(x, torch.int8, "x"), m, cin,
+                                 _dev(w_packed, torch.uint8, "w_packed"), cout, C.byref(rq),
+                                 _dev(y, torch.int8, "y"), _variant(variant), _stream(stream)),
+           "prom_pw_conv_i8")
+    return y
+
+
+def pw_conv_i8_acc32(x: torch.Tensor, w_packed: torch.Tensor, cout: int, stream=None) -> torch.Tensor:
+    m, cin = x.shape
+    acc = torch.empty((m, cout), dtype=torch.int32, device=x.device)
+    _check(lib().prom_pw_conv_i8_acc32(_dev(x, torch.int8, "x"), m, cin,
+                                       _dev(w_packed, torch.uint8, "w_packed"), cout,
+                                       acc.data_ptr(), _stream(stream)), "prom_pw_conv_i8_acc32")
+    return acc
+
+
+def pw_conv_i8_host(x_host: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequant,
+                    y_host: torch.Tensor, workspace: torch.Tensor, variant="auto", stream=None):
+    """prom_pw_conv_i8_host: host (pinned) activations in, host output out."""
+    m, cin = x_host.shape
+    if x_host.is_cuda or y_host.is_cuda:
+        raise ValueError("x_host / y_host must be host tensors")
+    _check(lib().prom_pw_conv_i8_host(x_host.data_ptr(), m, cin,
+                                      _dev(w_packed, torch.uint8, "w_packed"), cout, C.byref(rq),
+                                      y_host.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                      _variant(variant), _stream(stream)), "prom_pw_conv_i8_host")
+    return y_host
+
+
+class LayerSeq:
+    """A prom_layer array plus the tensors it points to (kept alive here)."""
+
+    def __init__(self, layers: Sequence[dict], act_min: int = 0, act_max: int = 127):
+        self.n = len(layers)
+        self._keep: List[torch.Tensor] = []
+        self.array = (PromLayer * self.n)()
+        for i, l in enumerate(layers):
+            for k in ("w_packed", "bias", "mult", "shift"):
+                self._keep.append(l[k])
+            self.array[i] = PromLayer(int(l["cin"]), int(l["cout"]), int(l["in_stride"]),
+                                      _dev(l["w_packed"], torch.uint8, "w_packed"),
+                                      make_requant(l["bias"], l["mult"], l["shift"], act_min, act_max))
+        self.cout_last = int(layers[-1]["cout"])
+        self.cin0 = int(layers[0]["cin"])
+        self.total_stride = 1
+        for l in layers:
+            self.total_stride *= int(l["in_stride"])
+
+    def workspace_bytes(self, batch: int, h0: int, w0: int) -> int:
+        return int(lib().prom_layer_seq_workspace_bytes(self.array, self.n, batch, h0, w0))
+
+    def host_workspace_bytes(self, batch: int, h0: int, w0: int) -> int:
+        return int(lib().prom_layer_seq_host_workspace_bytes(self.array, self.n, batch, h0, w0))
+
+
+def pw_layer_seq(seq: LayerSeq, x0: torch.Tensor, workspace: torch.Tensor,
+                 y_out: Optional[torch.Tensor] = None, variant="auto", stream=None) -> torch.Tensor:
+    """prom_pw_layer_seq on device tensors; x0 is [batch, h0, w0, cin0] int8."""
+    batch, h0, w0, _ = x0.shape
+    if y_out is None:
+        y_out = torch.empty((batch, h0 // seq.total_stride, w0 // seq.total_stride, seq.cout_last),
+                            dtype=torch.int8, device=x0.device)
+    _check(lib().prom_pw_layer_seq(seq.array, seq.n, _dev(x0, torch.int8, "x0"), batch, h0, w0,
+                                   workspace.data_ptr(), workspace.numel(),
+                                   _dev(y_out, torch.int8, "y_out"), _variant(variant),
+                                   _stream(stream)), "prom_pw_layer_seq")
+    return y_out
+
+
+def pw_layer_seq_host(seq: LayerSeq, x0_host: torch.Tensor, workspace: torch.Tensor,
+                      y_out_host: torch.Tensor, variant="auto", stream=None) -> torch.Tensor:
+    batch, h0, w0, _ = x0_host.shape
+    if x0_host.is_cuda or y_out_host.is_cuda:
+        raise ValueError("x0_host / y_out_host must be host tensors")
+    _check(lib().prom_pw_layer_seq_host(seq.array, seq.n, x0_host.data_ptr(), batch, h0, w0,
+                                        workspace.data_ptr(), workspace.numel(),
+                                        y_out_host.data_ptr(), _variant(variant), _stream(stream)),
+           "prom_pw_layer_seq_host")
+    return y_out_host

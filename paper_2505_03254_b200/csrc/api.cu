@@ -1,0 +1,614 @@
+// Host side of the C ABI (include/prom.h): argument checks, variant choice,
+// launch planning, tensor-map creation, and the layer-sequence driver.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <unordered_map>
+#include <vector>
+
+#include "prom.h"
+
+#include "common.cuh"
+#include "simple.cuh"
+#include "tc.cuh"
+#include "smallk.cuh"
+#include "addsub.cuh"
+
+namespace prom {
+
+static std::atomic<uint64_t> g_launches{0};
+
+struct DeviceInfo {
+    int sms = 0;
+    int smem_optin = 0;
+    bool ok = false;
+};
+
+static DeviceInfo device_info()
+{
+    static std::mutex mu;
+    static std::unordered_map<int, DeviceInfo> cache;
+    int dev = 0;
+    DeviceInfo d;
+    if (cudaGetDevice(&dev) != cudaSuccess) return d;
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = cache.find(dev);
+    if (it != cache.end()) return it->second;
+    if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) ==
+            cudaSuccess)
+        d.ok = true;
+    cache[dev] = d;
+    return d;
+}
+
+// ---- the layer as the host sees it -----------------------------------------------
+struct Conv {
+    const int8_t *x;
+    long long m;        // output rows
+    int cin, cout;
+    RowMap map;         // how output rows find their input rows
+    long long in_rows;  // rows of the input matrix
+    const uint8_t *w;
+    prom_requant rq;
+    int8_t *y;
+    cudaStream_t st;
+    bool pdl;           // chain to the previous kernel with programmatic dependent launch
+};
+
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static prom_status check_requant(const prom_requant *rq)
+{
+    if (!rq || !rq->bias || !rq->mult || !rq->shift) return PROM_ERR_NULL;
+    if (rq->act_min < -128 || rq->act_max > 127 || rq->act_min > rq->act_max)
+        return PROM_ERR_BAD_REQUANT;
+    return PROM_OK;
+}
+
+static prom_status check_conv(const int8_t *x, long long m, int cin, const uint8_t *w, int cout,
+                              const prom_requant *rq, const int8_t *y)
+{
+    if (!x || !w || !y) return PROM_ERR_NULL;
+    prom_status s = check_requant(rq);
+    if (s != PROM_OK) return s;
+    if (m < 0 || cin < 1 || cin > 4096 || cout < 1 || cout > 4096) return PROM_ERR_SHAPE;
+    if (m > (1ll << 40)) return PROM_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y)) return PROM_ERR_ALIGN;
+    return PROM_OK;
+}
+
+static int grid_for(long long work_items, int threads, int sms)
+{
+    long long blocks = (work_items + threads - 1) / threads;
+    long long cap = (long long)sms * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+static prom_status cuda_status(cudaError_t e) { return e == cudaSuccess ? PROM_OK : PROM_ERR_CUDA; }
+
+// ---- naive -------------------------------------------------------------------------------
+static prom_status launch_naive(const Conv &c, int32_t *acc_out)
+{
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    const int threads = 256;
+    int grid = grid_for(c.m * c.cout, threads, d.sms);
+    naive_conv_kernel<<<grid, threads, 0, c.st>>>(c.x, c.m, c.cin, c.map, c.w, c.cout, c.rq.bias,
+                                                  c.rq.mult, c.rq.shift, c.rq.act_min,
+                                                  c.rq.act_max, acc_out ? nullptr : c.y, acc_out);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+// ---- tensor-core variant: planning --------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) ==
+                cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+struct TcPlan {
+    tc::Params p;
+    CUtensorMap xmap;
+    int grid = 0;
+    size_t smem = 0;
+};
+
+static int round_up(int v, int a) { return (v + a - 1) / a * a; }
+
+// Fills everything of the plan that does not depend on pointers.  Returns
+// false when the tensor-core variant cannot run this shape.
+static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
+                          TcPlan &pl)
+{
+    tc::Params &p = pl.p;
+    memset(&p, 0, sizeof(p));
+    if (m <= 0 || (cin & 7) || (cout & 7)) return false;
+    int fold = 1;
+    if ((cin & 15) != 0) fold = 2;
+    if (fold == 2 && (map.stride != 1 || (m & 1))) return false;
+    int kf = cin * fold, nf = cout * fold;
+    if (kf > 4096) return false;
+
+    // subtiles: equal widths that divide nf, multiples of 16 (or a single 8-multiple one)
+    const int smem_max = d.smem_optin;
+    int n_sub = 0, nt = 0, groups = 1, subs_per_cta = 1, kc = (kf + 127) / 128;
+    size_t w_bytes = 0;
+    for (int s = (nf + 255) / 256; s <= nf / 8; ++s) {
+        if (nf % s) continue;
+        int w = nf / s;
+        if (s > 1 && (w & 15)) continue;
+        if (s == 1 && (w & 7)) continue;
+        int wp = round_up(w, 16);
+        size_t per_sub = (size_t)kc * wp * 128;
+        // resident weights must leave room for two activation stages and the staging rows
+        size_t fixed = 2 * tc::kStageBytes + 4 * 32 * (size_t)(w + 16) + (size_t)wp * 16 + 2048;
+        if (per_sub + fixed > (size_t)smem_max) continue;
+        n_sub = s; nt = w;
+        if ((size_t)s * per_sub <= 98304 && (size_t)s * per_sub + fixed + (size_t)(s - 1) * wp * 16 <=
+                                                (size_t)smem_max) {
+            groups = 1; subs_per_cta = s; w_bytes = (size_t)s * per_sub;
+        } else {
+            groups = s; subs_per_cta = 1; w_bytes = per_sub;
+        }
+        break;
+    }
+    if (!n_sub) return false;
+    if (n_sub == 1 && (nt & 15) && (nf != nt)) return false;
+
+    // tile rows
+    int tm = 128, x3d = 0, box_r = 0;
+    if (map.stride != 1) {
+        if (map.wo > 128) return false;
+        box_r = 128 / map.wo;
+        long long lines = m / map.wo;          // batch * ho
+        if (box_r > lines) box_r = (int)lines;
+        if (box_r > 256) box_r = 256;
+        tm = box_r * map.wo;
+        x3d = 1;
+    }
+    const int mode_b = (nt & 15) ? 1 : 0;
+    if (mode_b && (tm & 1)) return false;
+    long long rows = m / fold;
+    long long n_mtiles = (rows + tm - 1) / tm;
+    if (n_mtiles > 0x7fffffff) return false;
+
+    p.m_rows = rows; p.k0 = cin; p.n0 = cout; p.fold = fold; p.kf = kf; p.nf = nf;
+    p.tm = tm; p.n_mtiles = (int)n_mtiles; p.nt = nt; p.nt_pad = round_up(nt, 16);
+    p.n_sub = n_sub; p.groups = groups; p.subs_per_cta = subs_per_cta;
+    p.kc = kc;
+    int ksteps = (kf + 31) / 32;
+    p.ksteps_last = ksteps - 4 * (kc - 1);
+    p.acc_bufs = 2;
+    int cols = 2 * p.nt_pad, tc_cols = 32;
+    while (tc_cols < cols) tc_cols *= 2;
+    p.tmem_cols = tc_cols;
+    p.mode_b = mode_b;
+    p.out_pitch = mode_b ? nt : ((((nt >> 4) & 1) == 0) ? nt + 16 : nt);
+    p.x3d = x3d; p.box_r = box_r;
+    p.tx_bytes = x3d ? (uint32_t)(128 * map.wo * box_r) : (uint32_t)tc::kStageBytes;
+    p.inv_cpr = mode_b ? 0 : (uint32_t)(((1u << 20) + (nt >> 4) - 1) / (nt >> 4));
+
+    // shared-memory layout (offsets from the 1024-aligned base)
+    const int ncols_res = subs_per_cta * p.nt_pad;
+    const size_t out_bytes = (size_t)tc::kEpiWarps * 32 * p.out_pitch;
+    const size_t tail = round_up((int)out_bytes, 16) + (size_t)ncols_res * 8 + (size_t)ncols_res * 4 +
+                        round_up(ncols_res, 16) + 256;
+    // stages: 2 CTAs per SM when everything fits in half the shared memory with >= 3
+    // stages and 256 TMEM columns; otherwise one CTA with as many stages as fit (<= 8)
+    const size_t half = (size_t)(smem_max / 2) - 1024 - 1024;   // per-CTA share minus slack
+    int stages;
+    int occ = 1;
+    size_t base_need = w_bytes + tail;
+    if (p.tmem_cols <= 256 && base_need + 3 * (size_t)tc::kStageBytes <= half) {
+        occ = 2;
+        stages = (int)((half - base_need) / tc::kStageBytes);
+    } else {
+        stages = (int)(((size_t)smem_max - 1024 - base_need) / tc::kStageBytes);
+    }
+    if (stages > tc::kMaxStages) stages = tc::kMaxStages;
+    int need_stages = kc < 2 ? 2 : 2;
+    if (stages < need_stages) return false;
+    p.stages = stages;
+    uint32_t off = (uint32_t)stages * tc::kStageBytes;
+    p.off_w = off; off += (uint32_t)w_bytes;
+    p.off_out = off; off += (uint32_t)round_up((int)out_bytes, 16);
+    p.off_consts = off; off += (uint32_t)ncols_res * 8;
+    p.off_shift = off; off += (uint32_t)ncols_res * 4;
+    p.off_wmag = off; off += (uint32_t)round_up(ncols_res, 16);
+    p.off_bars = off; off += 256;
+    pl.smem = (size_t)off + 1024;
+    if (occ == 1 && p.tmem_cols == 512 && pl.smem * 2 <= (size_t)smem_max)
+        pl.smem = (size_t)smem_max / 2 + 1024;     // keep a second CTA (and its TMEM request) off the SM
+    if (pl.smem > (size_t)smem_max) return false;
+
+    long long slots = (long long)d.sms * occ;
+    long long workers = slots / groups;
+    if (workers < 1) workers = 1;
+    if (workers > n_mtiles) workers = n_mtiles;
+    pl.grid = (int)(workers * groups);
+    return true;
+}
+
+static bool tc_make_map(const Conv &c, TcPlan &pl)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const tc::Params &p = pl.p;
+    CUresult r;
+    if (!p.x3d) {
+        cuuint64_t dims[2] = {(cuuint64_t)p.kf, (cuuint64_t)p.m_rows};
+        cuuint64_t strides[1] = {(cuuint64_t)p.kf};
+        cuuint32_t box[2] = {128, 128};
+        cuuint32_t es[2] = {1, 1};
+        r = enc(&pl.xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(c.x), dims, strides,
+                box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        // [channel][wo, step stride*cin][batch*ho, step stride*win*cin]
+        const RowMap &mp = c.map;
+        cuuint64_t dims[3] = {(cuuint64_t)c.cin, (cuuint64_t)mp.wo, (cuuint64_t)(c.m / mp.wo)};
+        cuuint64_t strides[2] = {(cuuint64_t)mp.stride * c.cin,
+                                 (cuuint64_t)mp.stride * mp.win * c.cin};
+        cuuint32_t box[3] = {128, (cuuint32_t)mp.wo, (cuuint32_t)p.box_r};
+        cuuint32_t es[3] = {1, 1, 1};
+        r = enc(&pl.xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t *>(c.x), dims, strides,
+                box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    return r == CUDA_SUCCESS;
+}
+
+static prom_status launch_tc(const Conv &c)
+{
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    TcPlan pl;
+    if (!tc_shape_plan(c.m, c.cin, c.cout, c.map, d, pl)) return PROM_ERR_UNSUPPORTED;
+    if (!tc_make_map(c, pl)) return PROM_ERR_CUDA;
+    tc::Params &p = pl.p;
+    p.w_packed = c.w; p.bias = c.rq.bias; p.mult = c.rq.mult; p.shift = c.rq.shift;
+    p.act_min = c.rq.act_min; p.act_max = c.rq.act_max; p.y = c.y; p.pdl = c.pdl ? 1 : 0;
+
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin);
+    });
+    if (attr_err != cudaSuccess) return PROM_ERR_CUDA;
+
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)pl.grid);
+    cfg.blockDim = dim3(tc::kThreads);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = c.st;
+    cudaLaunchAttribute attr[1];
+    if (c.pdl) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    cudaError_t e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel, pl.xmap, p);
+    ++g_launches;
+    return cuda_status(e);
+}
+
+static bool tc_supported(const Conv &c)
+{
+    DeviceInfo d = device_info();
+    if (!d.ok) return false;
+    TcPlan pl;
+    return tc_shape_plan(c.m, c.cin, c.cout, c.map, d, pl);
+}
+
+// ---- variant choice --------------------------------------------------------------------------
+static prom_status run_conv(const Conv &c, prom_variant v)
+{
+    if (c.m == 0) return PROM_OK;
+    switch (v) {
+    case PROM_VARIANT_NAIVE: return launch_naive(c, nullptr);
+    case PROM_VARIANT_TC: return launch_tc(c);
+    case PROM_VARIANT_SMALLK: return smallk::launch(c.x, c.m, c.cin, c.map, c.w, c.cout, c.rq, c.y,
+                                                    c.st, g_launches);
+    case PROM_VARIANT_ADDSUB: return addsub::launch(c.x, c.m, c.cin, c.map, c.w, c.cout, c.rq, c.y,
+                                                    c.st, g_launches);
+    case PROM_VARIANT_AUTO:
+        if (tc_supported(c)) return launch_tc(c);
+        if (smallk::supported(c.cin, c.cout))
+            return smallk::launch(c.x, c.m, c.cin, c.map, c.w, c.cout, c.rq, c.y, c.st, g_launches);
+        return launch_naive(c, nullptr);
+    default: return PROM_ERR_UNSUPPORTED;
+    }
+}
+
+static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// Shapes of a sequence; false when it does not chain.
+struct SeqShape {
+    std::vector<long long> m;      // output rows per layer
+    std::vector<RowMap> map;
+    std::vector<int> h, w;
+};
+
+static bool seq_shapes(const prom_layer *layers, int n, int batch, int h0, int w0, SeqShape &s)
+{
+    if (!layers || n < 1 || batch < 1 || h0 < 1 || w0 < 1) return false;
+    int h = h0, w = w0;
+    for (int i = 0; i < n; ++i) {
+        const prom_layer &l = layers[i];
+        if (l.cin < 1 || l.cin > 4096 || l.cout < 1 || l.cout > 4096) return false;
+        if (i > 0 && l.cin != layers[i - 1].cout) return false;
+        if (l.in_stride != 1 && l.in_stride != 2) return false;
+        if (h % l.in_stride || w % l.in_stride) return false;
+        RowMap mp;
+        mp.stride = l.in_stride; mp.hin = h; mp.win = w;
+        h /= l.in_stride; w /= l.in_stride;
+        mp.ho = h; mp.wo = w;
+        s.map.push_back(mp);
+        s.m.push_back((long long)batch * h * w);
+        s.h.push_back(h); s.w.push_back(w);
+    }
+    return true;
+}
+
+static void seq_regions(const prom_layer *layers, int n, const SeqShape &s, size_t &a, size_t &b)
+{
+    a = b = 0;
+    for (int i = 0; i + 1 < n; ++i) {
+        size_t bytes = round256((size_t)s.m[i] * layers[i].cout);
+        if (i & 1) { if (bytes > b) b = bytes; }
+        else { if (bytes > a) a = bytes; }
+    }
+}
+
+static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, int batch, int h0,
+                           int w0, void *ws, size_t ws_bytes, int8_t *y_out, prom_variant variant,
+                           cudaStream_t st)
+{
+    SeqShape s;
+    if (!seq_shapes(layers, n, batch, h0, w0, s)) return PROM_ERR_SHAPE;
+    size_t ra, rb;
+    seq_regions(layers, n, s, ra, rb);
+    if (ra + rb > 0) {
+        if (!ws) return PROM_ERR_NULL;
+        if (!aligned16(ws)) return PROM_ERR_ALIGN;
+        if (ws_bytes < ra + rb) return PROM_ERR_WORKSPACE;
+    }
+    int8_t *reg[2] = {static_cast<int8_t *>(ws), static_cast<int8_t *>(ws) + ra};
+    // validate everything before the first launch
+    for (int i = 0; i < n; ++i) {
+        if (!layers[i].w_packed) return PROM_ERR_NULL;
+        prom_status e = check_requant(&layers[i].rq);
+        if (e != PROM_OK) return e;
+        if (!aligned16(layers[i].w_packed)) return PROM_ERR_ALIGN;
+    }
+    const int8_t *cur = x0;
+    long long in_rows = (long long)batch * h0 * w0;
+    for (int i = 0; i < n; ++i) {
+        Conv c;
+        c.x = cur; c.m = s.m[i]; c.cin = layers[i].cin; c.cout = layers[i].cout;
+        c.map = s.map[i]; c.in_rows = in_rows;
+        c.w = layers[i].w_packed; c.rq = layers[i].rq;
+        c.y = (i == n - 1) ? y_out : reg[i & 1];
+        c.st = st;
+        c.pdl = i > 0;
+        prom_status e = run_conv(c, variant);
+        if (e != PROM_OK) return e;
+        cur = c.y;
+        in_rows = c.m;
+    }
+    return PROM_OK;
+}
+
+}  // namespace prom
+
+using namespace prom;
+
+extern "C" {
+
+size_t prom_packed_bytes(int cout, int cin)
+{
+    if (cout < 0 || cin < 0) return 0;
+    return (size_t)cout * (size_t)((cin + 3) / 4);
+}
+
+prom_status prom_pack_ternary(const int8_t *w_dev, int cout, int cin, uint8_t *packed_dev,
+                              size_t packed_bytes, void *cuda_stream)
+{
+    if (!w_dev || !packed_dev) return PROM_ERR_NULL;
+    if (cout < 1 || cin < 1 || cout > 4096 || cin > 4096) return PROM_ERR_SHAPE;
+    if (packed_bytes < prom_packed_bytes(cout, cin)) return PROM_ERR_WORKSPACE;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    unsigned int *bad = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void **>(&bad), g_pack_bad) != cudaSuccess)
+        return PROM_ERR_CUDA;
+    if (cudaMemsetAsync(bad, 0, sizeof(unsigned int), st) != cudaSuccess) return PROM_ERR_CUDA;
+    long long total = (long long)cout * ((cin + 3) / 4);
+    pack_ternary_kernel<<<grid_for(total, 256, d.sms), 256, 0, st>>>(w_dev, cout, cin, packed_dev,
+                                                                     bad);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return PROM_ERR_CUDA;
+    unsigned int host_bad = 0;
+    if (cudaMemcpyAsync(&host_bad, bad, sizeof(host_bad), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return PROM_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return PROM_ERR_CUDA;
+    return host_bad ? PROM_ERR_BAD_WEIGHT : PROM_OK;
+}
+
+prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin, const uint8_t *w_packed_dev,
+                            int cout, const prom_requant *rq, int8_t *y_dev, prom_variant variant,
+                            void *cuda_stream)
+{
+    prom_status s = check_conv(x_dev, m, cin, w_packed_dev, cout, rq, y_dev);
+    if (s != PROM_OK) return s;
+    Conv c;
+    c.x = x_dev; c.m = m; c.cin = cin; c.cout = cout;
+    c.map = RowMap{1, 1, 1, 1, 1};
+    c.in_rows = m;
+    c.w = w_packed_dev; c.rq = *rq; c.y = y_dev;
+    c.st = static_cast<cudaStream_t>(cuda_stream);
+    c.pdl = false;
+    return run_conv(c, variant);
+}
+
+prom_status prom_pw_conv_i8_acc32(const int8_t *x_dev, int64_t m, int cin,
+                                  const uint8_t *w_packed_dev, int cout, int32_t *acc_dev,
+                                  void *cuda_stream)
+{
+    if (!x_dev || !w_packed_dev || !acc_dev) return PROM_ERR_NULL;
+    if (m < 0 || cin < 1 || cin > 4096 || cout < 1 || cout > 4096) return PROM_ERR_SHAPE;
+    if (m == 0) return PROM_OK;
+    Conv c;
+    c.x = x_dev; c.m = m; c.cin = cin; c.cout = cout;
+    c.map = RowMap{1, 1, 1, 1, 1};
+    c.in_rows = m;
+    c.w = w_packed_dev;
+    c.rq = prom_requant{nullptr, nullptr, nullptr, 0, 127};
+    c.y = nullptr;
+    c.st = static_cast<cudaStream_t>(cuda_stream);
+    c.pdl = false;
+    return launch_naive(c, acc_dev);
+}
+
+prom_status prom_pw_conv_i8_host(const int8_t *x_host, int64_t m, int cin,
+                                 const uint8_t *w_packed_dev, int cout, const prom_requant *rq,
+                                 int8_t *y_host, void *workspace_dev, size_t workspace_bytes,
+                                 prom_variant variant, void *cuda_stream)
+{
+    if (!x_host || !y_host || !workspace_dev) return PROM_ERR_NULL;
+    if (m < 0 || cin < 1 || cout < 1) return PROM_ERR_SHAPE;
+    size_t xb = round256((size_t)m * cin), yb = round256((size_t)m * cout);
+    if (workspace_bytes < xb + yb) return PROM_ERR_WORKSPACE;
+    if (!aligned16(workspace_dev)) return PROM_ERR_ALIGN;
+    int8_t *xd = static_cast<int8_t *>(workspace_dev);
+    int8_t *yd = xd + xb;
+    prom_status s = check_conv(xd, m, cin, w_packed_dev, cout, rq, yd);
+    if (s != PROM_OK) return s;
+    if (m == 0) return PROM_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(xd, x_host, (size_t)m * cin, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PROM_ERR_CUDA;
+    s = prom_pw_conv_i8(xd, m, cin, w_packed_dev, cout, rq, yd, variant, cuda_stream);
+    if (s != PROM_OK) return s;
+    return cuda_status(cudaMemcpyAsync(y_host, yd, (size_t)m * cout, cudaMemcpyDeviceToHost, st));
+}
+
+size_t prom_layer_seq_workspace_bytes(const prom_layer *layers, int n, int batch, int h0, int w0)
+{
+    SeqShape s;
+    if (!seq_shapes(layers, n, batch, h0, w0, s)) return 0;
+    size_t a, b;
+    seq_regions(layers, n, s, a, b);
+    return a + b;
+}
+
+prom_status prom_pw_layer_seq(const prom_layer *layers, int n, const int8_t *x0_dev, int batch,
+                              int h0, int w0, void *workspace_dev, size_t workspace_bytes,
+                              int8_t *y_out_dev, prom_variant variant, void *cuda_stream)
+{
+    if (!layers || !x0_dev || !y_out_dev) return PROM_ERR_NULL;
+    if (!aligned16(x0_dev) || !aligned16(y_out_dev)) return PROM_ERR_ALIGN;
+    return run_seq(layers, n, x0_dev, batch, h0, w0, workspace_dev, workspace_bytes, y_out_dev,
+                   variant, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t prom_layer_seq_host_workspace_bytes(const prom_layer *layers, int n, int batch, int h0,
+                                           int w0)
+{
+    SeqShape s;
+    if (!seq_shapes(layers, n, batch, h0, w0, s)) return 0;
+    size_t a, b;
+    seq_regions(layers, n, s, a, b);
+    size_t xin = round256((size_t)batch * h0 * w0 * layers[0].cin);
+    size_t yout = round256((size_t)s.m[n - 1] * layers[n - 1].cout);
+    return a + b + xin + yout;
+}
+
+prom_status prom_pw_layer_seq_host(const prom_layer *layers, int n, const int8_t *x0_host,
+                                   int batch, int h0, int w0, void *workspace_dev,
+                                   size_t workspace_bytes, int8_t *y_out_host, prom_variant variant,
+                                   void *cuda_stream)
+{
+    if (!layers || !x0_host || !y_out_host || !workspace_dev) return PROM_ERR_NULL;
+    if (!aligned16(workspace_dev)) return PROM_ERR_ALIGN;
+    SeqShape s;
+    if (!seq_shapes(layers, n, batch, h0, w0, s)) return PROM_ERR_SHAPE;
+    size_t a, b;
+    seq_regions(layers, n, s, a, b);
+    size_t xin_raw = (size_t)batch * h0 * w0 * layers[0].cin;
+    size_t yout_raw = (size_t)s.m[n - 1] * layers[n - 1].cout;
+    size_t xin = round256(xin_raw), yout = round256(yout_raw);
+    if (workspace_bytes < a + b + xin + yout) return PROM_ERR_WORKSPACE;
+    int8_t *base = static_cast<int8_t *>(workspace_dev);
+    int8_t *xd = base + a + b, *yd = xd + xin;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(xd, x0_host, xin_raw, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return PROM_ERR_CUDA;
+    prom_status e = run_seq(layers, n, xd, batch, h0, w0, base, a + b, yd, variant, st);
+    if (e != PROM_OK) return e;
+    return cuda_status(cudaMemcpyAsync(y_out_host, yd, yout_raw, cudaMemcpyDeviceToHost, st));
+}
+
+prom_status prom_last_device_status(void *cuda_stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    unsigned int v = 0;
+    if (cudaMemcpyFromSymbolAsync(&v, g_status, sizeof(v), 0, cudaMemcpyDeviceToHost, st) !=
+        cudaSuccess)
+        return PROM_ERR_CUDA;
+    unsigned int zero = 0;
+    if (cudaMemcpyToSymbolAsync(g_status, &zero, sizeof(zero), 0, cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+        return PROM_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return PROM_ERR_CUDA;
+    return static_cast<prom_status>(v);
+}
+
+uint64_t prom_launch_count(void) { return g_launches.load(); }
+
+void prom_shutdown(void) { addsub::release_cache(); }
+
+const char *prom_status_string(prom_status s)
+{
+    switch (s) {
+    case PROM_OK: return "ok";
+    case PROM_ERR_NULL: return "null pointer";
+    case PROM_ERR_SHAPE: return "bad shape";
+    case PROM_ERR_ALIGN: return "misaligned pointer";
+    case PROM_ERR_BAD_WEIGHT: return "weight outside {-1,0,+1}";
+    case PROM_ERR_BAD_REQUANT: return "requantisation constants out of range";
+    case PROM_ERR_WORKSPACE: return "workspace too small";
+    case PROM_ERR_UNSUPPORTED: return "variant does not support this shape";
+    case PROM_ERR_CUDA: return "CUDA call failed";
+    case PROM_ERR_TIMEOUT: return "device-side wait ran out";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,86 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header
+declares, and rejects bad arguments on the host before touching CUDA."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2505_03254_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "prom.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(prom_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert "prom_pack_ternary" in names and "prom_pw_conv_i8" in names and "prom_pw_layer_seq" in names
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(binding.EXPORTS)
+
+
+def test_packed_bytes(lib):
+    assert binding.packed_bytes(384, 64) == 384 * 16
+    assert binding.packed_bytes(3, 6) == 6
+    assert binding.packed_bytes(1, 1) == 1
+    assert binding.packed_bytes(-1, 4) == 0
+
+
+def test_status_strings(lib):
+    seen = {binding.status_string(i) for i in range(10)}
+    assert len(seen) == 10 and "ok" in seen
+    assert binding.status_string(99) == "unknown status"
+
+
+def test_host_side_argument_checks(lib):
+    rq = binding.PromRequant(16, 16, 16, 0, 127)
+    A = 0x1000  # a 16-byte-aligned non-null address; never dereferenced by these calls
+    st = None
+    f = lib.prom_pw_conv_i8
+    assert f(None, 4, 8, A, 8, C.byref(rq), A, 0, st) == binding.PROM_ERR_NULL
+    assert f(A, 4, 8, A, 8, None, A, 0, st) == binding.PROM_ERR_NULL
+    assert f(A, -1, 8, A, 8, C.byref(rq), A, 0, st) == binding.PROM_ERR_SHAPE
+    assert f(A, 4, 0, A, 8, C.byref(rq), A, 0, st) == binding.PROM_ERR_SHAPE
+    assert f(A, 4, 8, A, 5000, C.byref(rq), A, 0, st) == binding.PROM_ERR_SHAPE
+    assert f(A + 4, 4, 8, A, 8, C.byref(rq), A, 0, st) == binding.PROM_ERR_ALIGN
+    bad = binding.PromRequant(16, 16, 16, 5, 4)
+    assert f(A, 4, 8, A, 8, C.byref(bad), A, 0, st) == binding.PROM_ERR_BAD_REQUANT
+    bad = binding.PromRequant(16, 16, 16, -129, 4)
+    assert f(A, 4, 8, A, 8, C.byref(bad), A, 0, st) == binding.PROM_ERR_BAD_REQUANT
+    bad = binding.PromRequant(0, 16, 16, 0, 127)
+    assert f(A, 4, 8, A, 8, C.byref(bad), A, 0, st) == binding.PROM_ERR_NULL
+    # m == 0 is a no-op
+    assert f(A, 0, 8, A, 8, C.byref(rq), A, 0, st) == binding.PROM_OK
+    assert lib.prom_pack_ternary(None, 4, 4, A, 4, st) == binding.PROM_ERR_NULL
+    assert lib.prom_pack_ternary(A, 4, 4, A, 3, st) == binding.PROM_ERR_WORKSPACE
+    assert lib.prom_pack_ternary(A, 0, 4, A, 3, st) == binding.PROM_ERR_SHAPE
+
+
+def test_layer_seq_shape_checks(lib):
+    L = binding.PromLayer
+    rq = binding.PromRequant(16, 16, 16, 0, 127)
+    arr = (L * 3)(L(8, 16, 1, 16, rq), L(16, 8, 2, 16, rq), L(8, 24, 1, 16, rq))
+    ws = lib.prom_layer_seq_workspace_bytes(arr, 3, 2, 8, 8)
+    # region A holds layer 0's output (2*8*8*16), region B layer 1's (2*4*4*8), each 256-rounded
+    assert ws == 2048 + 256
+    assert lib.prom_layer_seq_host_workspace_bytes(arr, 3, 2, 8, 8) == ws + 1024 + 768
+    arr[1].cin = 12          # does not chain
+    assert lib.prom_layer_seq_workspace_bytes(arr, 3, 2, 8, 8) == 0
+    arr[1].cin = 16
+    assert lib.prom_layer_seq_workspace_bytes(arr, 3, 2, 7, 8) == 0   # odd size under stride 2
+    A = 0x1000
+    assert lib.prom_pw_layer_seq(arr, 3, A, 2, 7, 8, A, 1 << 20, A, 0, None) == binding.PROM_ERR_SHAPE
+    assert lib.prom_pw_layer_seq(arr, 3, A, 2, 8, 8, A, 16, A, 0, None) == binding.PROM_ERR_WORKSPACE
+    assert lib.prom_pw_layer_seq(arr, 3, None, 2, 8, 8, A, 1 << 20, A, 0, None) == binding.PROM_ERR_NULL

@@ -1,0 +1,179 @@
+"""GPU parity: every variant of the library against the CPU oracle, byte for
+byte, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_03254_b200 import binding, build, synth
+from gpu_util import first_mismatch, make_case, oracle_y, run_variant, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    build.build()
+    binding.lib()
+    binding.last_device_status()
+    yield
+    assert binding.last_device_status() == binding.PROM_OK
+
+
+def test_pack_matches_oracle(oracle):
+    for seed, (cout, cin) in enumerate([(1, 1), (5, 3), (16, 24), (37, 145), (384, 64), (1280, 320)]):
+        w = synth.ternary_weights(seed, cout, cin, 0.5)
+        got = binding.pack_ternary(w.cuda()).cpu().numpy()
+        assert np.array_equal(got, oracle.pack(w.numpy()))
+
+
+def test_pack_rejects_invalid_weights():
+    w = torch.zeros((4, 8), dtype=torch.int8)
+    w[2, 5] = 2
+    with pytest.raises(binding.PromError) as e:
+        binding.pack_ternary(w.cuda())
+    assert e.value.code == binding.PROM_ERR_BAD_WEIGHT
+
+
+def test_acc32_matches_oracle(oracle):
+    x, lay = make_case(3, 77, 40, 24)
+    xd, wp, _ = to_device(x, lay)
+    acc = binding.pw_conv_i8_acc32(xd, wp, 24).cpu().numpy()
+    _, want = oracle.conv_mul(x.numpy(), lay["w"].numpy(), lay["bias"].numpy(), lay["mult"].numpy(),
+                              lay["shift"].numpy(), want_acc=True)
+    assert np.array_equal(acc, want)
+
+
+# (m, cin, cout): several tiles and a ragged tail, odd channel counts included
+NAIVE_SHAPES = [(1, 1, 1), (196, 64, 384), (300, 24, 144), (129, 7, 5), (1000, 145, 37)]
+TC_SHAPES = [(196, 64, 384), (1, 16, 16), (127, 16, 96), (128, 32, 16), (129, 96, 24),
+             (1000, 144, 32), (777, 192, 64), (515, 384, 96), (300, 576, 160), (260, 960, 320),
+             (333, 320, 1280), (2000, 16, 96), (386, 24, 144), (258, 144, 24), (130, 40, 8),
+             (4100, 64, 384), (200, 160, 960), (131, 960, 160), (64, 8, 8), (50000, 32, 192)]
+SMALLK_SHAPES = [(196, 64, 384), (1000, 16, 96), (129, 24, 144), (333, 4, 3), (500, 32, 16), (77, 60, 10)]
+ADDSUB_SHAPES = [(196, 64, 384), (1000, 16, 96), (129, 24, 144), (300, 145, 37), (260, 960, 320),
+                 (131, 600, 9)]
+
+
+@pytest.mark.parametrize("m,cin,cout", NAIVE_SHAPES)
+def test_naive(oracle, m, cin, cout):
+    x, lay = make_case(10, m, cin, cout)
+    got = run_variant(*to_device(x, lay), cout, "naive")
+    assert first_mismatch(got, oracle_y(oracle, x, lay)) is None
+
+
+@pytest.mark.parametrize("m,cin,cout", TC_SHAPES)
+def test_tc(oracle, m, cin, cout):
+    x, lay = make_case(11, m, cin, cout)
+    got = run_variant(*to_device(x, lay), cout, "tc")
+    assert first_mismatch(got, oracle_y(oracle, x, lay)) is None
+
+
+@pytest.mark.parametrize("m,cin,cout", SMALLK_SHAPES)
+def test_smallk(oracle, m, cin, cout):
+    x, lay = make_case(12, m, cin, cout)
+    got = run_variant(*to_device(x, lay), cout, "smallk")
+    assert first_mismatch(got, oracle_y(oracle, x, lay)) is None
+
+
+@pytest.mark.parametrize("m,cin,cout", ADDSUB_SHAPES)
+@pytest.mark.parametrize("zero_frac", [0.3, 0.9])
+def test_addsub(oracle, m, cin, cout, zero_frac):
+    x, lay = make_case(13, m, cin, cout, zero_frac)
+    got = run_variant(*to_device(x, lay), cout, "addsub")
+    assert first_mismatch(got, oracle_y(oracle, x, lay)) is None
+
+
+@pytest.mark.parametrize("variant", ["naive", "tc", "smallk", "addsub", "auto"])
+def test_signed_clamp_and_wide_shifts(oracle, variant):
+    """act_min < 0 pins the rounding of negative values; shifts 0..20 leave the
+    tensor-core variant's fast epilogue."""
+    x, lay = make_case(14, 517, 32, 48, shift_lo=0, shift_hi=20)
+    xd, wp, consts = to_device(x, lay)
+    for lo, hi in [(-128, 127), (-5, 90), (0, 127), (3, 100)]:
+        got = run_variant(xd, wp, consts, 48, variant, lo, hi)
+        assert first_mismatch(got, oracle_y(oracle, x, lay, lo, hi)) is None
+
+
+@pytest.mark.parametrize("variant", ["tc", "smallk", "addsub", "naive"])
+def test_ties_on_device(oracle, variant):
+    """mult = 2^30, shift = 0, bias = 0: every odd accumulator is a tie."""
+    m, cin, cout = 256, 16, 16
+    x = synth.act_uniform_i8(15, (m, cin))
+    lay = synth.make_layer(15, cin, cout, 0.5)
+    lay["bias"] = torch.zeros(cout, dtype=torch.int32)
+    lay["mult"] = torch.full((cout,), 1 << 30, dtype=torch.int32)
+    lay["shift"] = torch.zeros(cout, dtype=torch.int8)
+    xd, wp, consts = to_device(x, lay)
+    for lo, hi in [(-128, 127), (0, 127)]:
+        got = run_variant(xd, wp, consts, cout, variant, lo, hi)
+        assert first_mismatch(got, oracle_y(oracle, x, lay, lo, hi)) is None
+
+
+def test_extreme_values(oracle):
+    """All activations -128 against all +1 / all -1 weights at Cin = 960."""
+    m, cin, cout = 130, 960, 16
+    x = torch.full((m, cin), -128, dtype=torch.int8)
+    lay = synth.make_layer(16, cin, cout, 0.0)
+    lay["w"][:8] = 1
+    lay["w"][8:] = -1
+    xd, wp, consts = to_device(x, lay)
+    for variant in ["tc", "addsub", "naive"]:
+        for lo, hi in [(0, 127), (-128, 127)]:
+            got = run_variant(xd, wp, consts, cout, variant, lo, hi)
+            assert first_mismatch(got, oracle_y(oracle, x, lay, lo, hi)) is None
+
+
+def test_bad_constants_are_reported():
+    x, lay = make_case(17, 64, 16, 16)
+    lay["shift"][3] = 40
+    xd, wp, consts = to_device(x, lay)
+    for variant in ["naive", "tc", "smallk", "addsub"]:
+        run_variant(xd, wp, consts, 16, variant)
+        assert binding.last_device_status() == binding.PROM_ERR_BAD_REQUANT
+    assert binding.last_device_status() == binding.PROM_OK
+
+
+def test_invalid_code_is_reported():
+    x, lay = make_case(18, 64, 16, 16)
+    xd, wp, consts = to_device(x, lay)
+    wp[2, 1] = 0b00100000          # code 10 in the third slot
+    for variant in ["naive", "tc", "smallk", "addsub"]:
+        run_variant(xd, wp, consts, 16, variant)
+        assert binding.last_device_status() == binding.PROM_ERR_BAD_WEIGHT
+
+
+def test_unsupported_shapes_are_refused():
+    x, lay = make_case(19, 65, 20, 12)
+    xd, wp, consts = to_device(x, lay)
+    rq = binding.make_requant(*consts)
+    for variant in ["tc"]:
+        with pytest.raises(binding.PromError) as e:
+            binding.pw_conv_i8(xd, wp, 12, rq, variant=variant)
+        assert e.value.code == binding.PROM_ERR_UNSUPPORTED
+    x, lay = make_case(19, 64, 128, 12)
+    xd, wp, consts = to_device(x, lay)
+    with pytest.raises(binding.PromError) as e:
+        binding.pw_conv_i8(xd, wp, 12, binding.make_requant(*consts), variant="smallk")
+    assert e.value.code == binding.PROM_ERR_UNSUPPORTED
+
+
+def test_auto_handles_any_shape(oracle):
+    for m, cin, cout in [(65, 20, 12), (33, 7, 5), (131, 24, 144), (100, 2000, 8)]:
+        x, lay = make_case(20, m, cin, cout)
+        got = run_variant(*to_device(x, lay), cout, "auto")
+        assert first_mismatch(got, oracle_y(oracle, x, lay)) is None
+
+
+def test_host_buffer_entry_point(oracle):
+    m, cin, cout = 700, 64, 96
+    x, lay = make_case(21, m, cin, cout)
+    _, wp, consts = to_device(x, lay)
+    rq = binding.make_requant(*consts)
+    xh = x.pin_memory()
+    yh = torch.empty((m, cout), dtype=torch.int8).pin_memory()
+    ws = torch.empty(((m * cin + 255) // 256 * 256 + (m * cout + 255) // 256 * 256,),
+                     dtype=torch.uint8, device="cuda")
+    binding.pw_conv_i8_host(xh, wp, cout, rq, yh, ws)
+    torch.cuda.synchronize()
+    assert first_mismatch(yh.numpy(), oracle_y(oracle, x, lay)) is None

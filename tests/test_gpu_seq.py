@@ -1,0 +1,109 @@
+"""GPU parity of the layer sequence and of the benchmark configurations."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_03254_b200 import binding, build, synth
+from gpu_util import first_mismatch, make_case, oracle_y, run_variant, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    build.build()
+    binding.lib()
+    binding.last_device_status()
+    yield
+    assert binding.last_device_status() == binding.PROM_OK
+
+
+def build_sequence(seed, table, zero_frac=0.5):
+    host, dev = [], []
+    for i, l in enumerate(table):
+        d = synth.make_layer(seed, l.cin, l.cout, zero_frac, index=i + 1)
+        host.append(dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride, w=d["w"].numpy(),
+                         bias=d["bias"].numpy(), mult=d["mult"].numpy(), shift=d["shift"].numpy()))
+        dev.append(dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride,
+                        w_packed=binding.pack_ternary(d["w"].cuda()), bias=d["bias"].cuda(),
+                        mult=d["mult"].cuda(), shift=d["shift"].cuda()))
+    return host, binding.LayerSeq(dev)
+
+
+@pytest.mark.parametrize("variant", ["auto", "naive", "tc"])
+@pytest.mark.parametrize("batch,hw", [(2, 32), (3, 64)])
+def test_mobilenetv2_sequence_small(oracle, variant, batch, hw):
+    """All 34 layers, chained, at a reduced image size (several tiles per layer
+    early on, ragged tiles and single-tile layers late)."""
+    table = synth.mobilenetv2_pointwise_layers(h0=hw, w0=hw)
+    host, seq = build_sequence(31, table)
+    x0 = synth.act_post_relu6(31, (batch, hw, hw, 32))
+    ws = torch.empty((seq.workspace_bytes(batch, hw, hw),), dtype=torch.uint8, device="cuda")
+    y = binding.pw_layer_seq(seq, x0.cuda(), ws, variant=variant)
+    torch.cuda.synchronize()
+    want = oracle.layer_seq(host, x0.numpy())
+    assert y.shape == want.shape
+    assert first_mismatch(y.cpu().numpy().reshape(-1, 1280), want.reshape(-1, 1280)) is None
+
+
+def test_sequence_host_entry_point(oracle):
+    table = synth.mobilenetv2_pointwise_layers(h0=32, w0=32)[:9]
+    host, seq = build_sequence(32, table)
+    x0 = synth.act_post_relu6(32, (2, 32, 32, 32))
+    ws = torch.empty((seq.host_workspace_bytes(2, 32, 32),), dtype=torch.uint8, device="cuda")
+    want = oracle.layer_seq(host, x0.numpy())
+    yh = torch.empty(want.shape, dtype=torch.int8).pin_memory()
+    binding.pw_layer_seq_host(seq, x0.pin_memory(), ws, yh)
+    torch.cuda.synchronize()
+    assert np.array_equal(yh.numpy(), want)
+
+
+def test_every_layer_standalone_at_its_channel_counts(oracle):
+    """Each of the 34 layer shapes on a fresh seeded post-ReLU6 input (chained
+    activations shrink towards the bias, which makes them weak evidence)."""
+    table = synth.mobilenetv2_pointwise_layers()
+    seen = set()
+    for i, l in enumerate(table):
+        if (l.cin, l.cout) in seen:
+            continue
+        seen.add((l.cin, l.cout))
+        m = 1000 + 2 * i
+        x, lay = make_case(100 + i, m, l.cin, l.cout, act="relu6")
+        got = run_variant(*to_device(x, lay), l.cout, "auto")
+        assert first_mismatch(got, oracle_y(oracle, x, lay)) is None, l
+
+
+def test_config1_and_config4_shapes(oracle):
+    for seed, (m, cin, cout, act) in enumerate([(196, 64, 384, "i8"), (3000, 960, 160, "u7"),
+                                                (3000, 160, 960, "u7"), (3000, 320, 1280, "u7")]):
+        x, lay = make_case(synth.BASE_SEED + seed, m, cin, cout, act=act)
+        xd, wp, consts = to_device(x, lay)
+        want = oracle_y(oracle, x, lay)
+        for variant in ["tc", "addsub"]:
+            got = run_variant(xd, wp, consts, cout, variant)
+            assert first_mismatch(got, want) is None, (m, cin, cout, variant)
+
+
+def test_config2_full_size_sampled_rows(oracle):
+    """Config 2 at full size (M = 802816) in the launch shape the benchmark
+    times; the oracle evaluates sampled rows (rows are independent)."""
+    m, cin, cout = 64 * 112 * 112, 16, 96
+    x = synth.act_post_relu6(synth.BASE_SEED + 2, (m, cin), device="cuda")
+    lay = synth.make_layer(synth.BASE_SEED + 2, cin, cout, 0.5)
+    wp = binding.pack_ternary(lay["w"].cuda())
+    consts = (lay["bias"].cuda(), lay["mult"].cuda(), lay["shift"].cuda())
+    rows = np.unique(np.concatenate([np.arange(0, 512), np.arange(m - 512, m),
+                                     np.random.default_rng(0).integers(0, m, 20000)]))
+    xs = x[torch.from_numpy(rows).cuda()].cpu()
+    want = oracle_y(oracle, xs, lay)
+    for variant in ["tc", "smallk", "auto"]:
+        y = torch.empty((m, cout), dtype=torch.int8, device="cuda")
+        binding.pw_conv_i8(x, wp, cout, binding.make_requant(*consts), y=y, variant=variant)
+        got = y[torch.from_numpy(rows).cuda()].cpu().numpy()
+        assert first_mismatch(got, want) is None, variant
+        # all variants agree everywhere
+        if variant == "tc":
+            ref = y.clone()
+        else:
+            assert torch.equal(y, ref)
