@@ -1,0 +1,496 @@
+#!/usr/bin/env python
+"""Benchmark of the ternary pointwise-convolution path.
+
+One step = the 34 pointwise layers of MobileNetV2-1.0 at 224x224 for a batch of
+128 images, chained through `prom_pw_layer_seq` (int8 NHWC activations,
+2-bit ternary weights, fused requantisation).  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
+
+`--impl reference` times the plain CPU oracle instead (host cores, bounded
+sample per step).  `--sweep FILE` runs the shape/sparsity sweep of single
+layers (tensor-core and add/sub variants) and writes one JSON record per point.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+BATCH = 128
+METRIC = "MobileNetV2 all-1x1-layers images/s"
+UNIT = "images/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio on B200 (4.5 : 2.25)
+FLUSH_BYTES = 512 << 20       # > 2x the 126 MB L2
+
+
+# --------------------------------------------------------------------------- helpers
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    except Exception:
+        return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS,
+                    bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def layer_bytes(m, cin, cout):
+    """Algorithmic bytes of one layer: activations in, activations out, 2-bit
+    weights, 9 bytes of requantisation constants per output channel."""
+    return m * cin + m * cout + cout * ((cin + 3) // 4) + 9 * cout
+
+
+def layer_ops(m, cin, cout):
+    return 2 * m * cin * cout
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons of one GPU while a region runs."""
+
+    def __init__(self, device_index: int):
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = torch.cuda.get_device_properties(device_index).uuid
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            self._nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    _NAMES = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+              0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting",
+              0x10: "sync_boost", 0x100: "display_clock_setting"}
+
+    def _once(self):
+        nv = self._nv
+        mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+        try:
+            r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+        except Exception:
+            r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+        self.samples.append(mhz)
+        for bit, name in self._NAMES.items():
+            if r & bit:
+                self.reasons.add(name)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self._once()
+            except Exception:
+                return
+            time.sleep(0.02)
+
+    def start(self):
+        if self._h is None:
+            return
+        self._stop.clear()
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+
+    def stop(self):
+        if self._thr is not None:
+            self._stop.set()
+            self._thr.join()
+            self._thr = None
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def build_network(seed, synth, binding=None, device=None):
+    """Layer table plus per-layer weights/constants: host arrays for the oracle,
+    and (when a binding is given) packed device tensors for the library."""
+    table = synth.mobilenetv2_pointwise_layers()
+    host, dev = [], []
+    for i, l in enumerate(table):
+        d = synth.make_layer(seed, l.cin, l.cout, 0.5, index=i + 1)
+        host.append(dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride, w=d["w"].numpy(),
+                         bias=d["bias"].numpy(), mult=d["mult"].numpy(), shift=d["shift"].numpy()))
+        if binding is not None:
+            dev.append(dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride,
+                            w_packed=binding.pack_ternary(d["w"].to(device)),
+                            bias=d["bias"].to(device), mult=d["mult"].to(device),
+                            shift=d["shift"].to(device)))
+    return table, host, dev
+
+
+# --------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """The CPU oracle, as it stands, on the host cores: each step is the whole
+    34-layer sequence over a bounded number of images."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from oracle import prom_oracle
+    from paper_2505_03254_b200 import synth
+    prom_oracle.build()
+    seed = synth.BASE_SEED + 3
+    _, host, _ = build_network(seed, synth)
+    x1 = synth.act_post_relu6(seed, (1, 112, 112, 32)).numpy()
+    t0 = time.perf_counter()
+    prom_oracle.layer_seq(host, x1)
+    t1 = max(time.perf_counter() - t0, 1e-4)
+    total = args.steps + args.warmup
+    images = int(max(1, min(BATCH, 120.0 / (total * t1))))
+    x = synth.act_post_relu6(seed, (images, 112, 112, 32)).numpy()
+    for _ in range(args.warmup):
+        prom_oracle.layer_seq(host, x)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        prom_oracle.layer_seq(host, x)
+    dt = time.perf_counter() - t0
+    value = images * args.steps / dt
+    cores = prom_oracle.threads()
+    sample = f"{images} image(s) of the batch-{BATCH} workload per step, all 34 layers"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "configs[2]: MobileNetV2-1.0 @224, all 34 1x1 layers, chained, "
+                               f"batch {BATCH}; reference arm steps over {images} image(s)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+    return 0
+
+
+# --------------------------------------------------------------------------- GPU arm
+def time_region(torch, fn, steps, dist_on):
+    """Times `steps` calls of fn with CUDA events on the current stream, bracketed
+    by barrier + synchronize; returns milliseconds (max over ranks)."""
+    import torch.distributed as dist
+    stream = torch.cuda.current_stream()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    if dist_on:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(steps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if dist_on:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    if dist_on:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def cold_time_us(torch, fn, flush, iters=20, warm=3):
+    """Median/min device time of one launch with L2 flushed before each."""
+    stream = torch.cuda.current_stream()
+    ts = []
+    for i in range(warm + iters):
+        flush.fill_(i & 0x7F)
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        e1.synchronize()
+        if i >= warm:
+            ts.append(e0.elapsed_time(e1) * 1e3)
+    return statistics.median(ts), min(ts)
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2505_03254_b200 import binding, build, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist_on = world > 1
+    if dist_on:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if dist_on:
+        dist.barrier()
+    binding.lib()
+    pk = peaks()
+    p_i8 = INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12
+    bw = pk["hbm_gbs"] * 1e9
+
+    seed = synth.BASE_SEED + 3
+    table, host, dev = build_network(seed, synth, binding, "cuda")
+    seq = binding.LayerSeq(dev)
+    x0 = synth.act_post_relu6(seed, (BATCH, 112, 112, 32), device="cuda")
+    ws = torch.empty((seq.workspace_bytes(BATCH, 112, 112),), dtype=torch.uint8, device="cuda")
+    y = torch.empty((BATCH, 7, 7, 1280), dtype=torch.int8, device="cuda")
+    variant = args.variant
+
+    def step():
+        binding.pw_layer_seq(seq, x0, ws, y_out=y, variant=variant)
+
+    sampler = ClockSampler(local)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if binding.last_device_status() != binding.PROM_OK:
+        raise RuntimeError("device status not OK after warm-up")
+
+    # ---- device-resident timing ------------------------------------------------
+    sampler.start()
+    l0 = binding.launch_count()
+    ms = time_region(torch, step, args.steps, dist_on)
+    launches = binding.launch_count() - l0
+    ms_per_step = ms / args.steps
+    value = world * BATCH * args.steps / (ms * 1e-3)
+
+    # ---- end to end: pinned host input -> device -> sequence -> host output ------
+    x0_host = x0.cpu().pin_memory()
+    y_host = torch.empty((BATCH, 7, 7, 1280), dtype=torch.int8).pin_memory()
+    ws_host = torch.empty((seq.host_workspace_bytes(BATCH, 112, 112),), dtype=torch.uint8,
+                          device="cuda")
+
+    def step_e2e():
+        binding.pw_layer_seq_host(seq, x0_host, ws_host, y_host, variant=variant)
+
+    for _ in range(3):
+        step_e2e()
+    e2e_steps = args.steps
+    ms_e2e = time_region(torch, step_e2e, e2e_steps, dist_on)
+    sampler.stop()
+    e2e_value = world * BATCH * e2e_steps / (ms_e2e * 1e-3)
+    same = bool(torch.equal(y_host, y.cpu()))
+    del ws_host
+
+    status = binding.last_device_status()
+    if status != binding.PROM_OK:
+        raise RuntimeError(f"device status {status} after the timed region")
+
+    # ---- roofline of the step ----------------------------------------------------
+    ms_layers = [BATCH * l.h * l.w for l in table]
+    step_bytes = sum(layer_bytes(m, l.cin, l.cout) for m, l in zip(ms_layers, table))
+    step_ops = sum(layer_ops(m, l.cin, l.cout) for m, l in zip(ms_layers, table))
+    roof_us = [max(layer_bytes(m, l.cin, l.cout) / bw, layer_ops(m, l.cin, l.cout) / p_i8) * 1e6
+               for m, l in zip(ms_layers, table)]
+    achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "tc_conv_kernel", "achieved": achieved,
+                "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
+                "peak_source": pk["source"], "traffic": None,
+                "launches_per_step": launches / args.steps,
+                "bytes_per_launch": step_bytes / (launches / args.steps),
+                "us_per_launch": ms_per_step * 1e3 / (launches / args.steps),
+                "step_roofline_us": sum(roof_us),
+                "step_roofline_frac": sum(roof_us) / (ms_per_step * 1e3)}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": f"configs[2]: MobileNetV2-1.0 @224, all 34 ternary 1x1 layers, "
+                               f"chained, batch {BATCH} per GPU, post-ReLU6 int8 NHWC input "
+                               f"[{BATCH},112,112,32], P(0)=0.5 ternary weights",
+                   "variant": variant, "seed": seed,
+                   "l2": "no flush: a step moves 877 MB through buffers of up to 154 MB (> 126 MB L2)",
+                   "parallelism": f"batch sharded over {world} GPU(s), no collective"},
+        "gops": step_ops / (ms_per_step * 1e-3) / 1e9,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x0_host.numel()),
+                "d2h_bytes_per_step": int(y_host.numel()), "ms_per_step": ms_e2e / e2e_steps,
+                "matches_device_run": same},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "clocks": sampler.summary(),
+    }
+
+    if rank == 0 and world == 1 and not args.no_detail:
+        out["layers"] = per_layer_detail(torch, binding, synth, table, dev, seed, bw, p_i8, variant)
+        out["single_layer"] = single_layer_configs(torch, binding, synth, bw, p_i8)
+        cold_us = sum(r["us"] for r in out["layers"])
+        roofline["sum_layer_cold_us"] = cold_us
+        roofline["sum_layer_cold_frac"] = sum(roof_us) / cold_us
+
+    if rank == 0 and world == 1 and not args.no_cpu:
+        from oracle import prom_oracle
+        prom_oracle.build()
+        xh = x0_host.numpy()
+        t0 = time.perf_counter()
+        want = prom_oracle.layer_seq(host, xh)
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": BATCH / dt, "unit": UNIT, "cores": prom_oracle.threads(),
+                               "kind": "oracle",
+                               "sample": f"one full step (batch {BATCH}, 34 layers), {dt:.2f} s"}
+        out["parity"] = bool((want == y.cpu().numpy()).all())
+    elif rank == 0:
+        out["cpu_baseline"] = None
+
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if dist_on:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def per_layer_detail(torch, binding, synth, table, dev, seed, bw, p_i8, variant):
+    """Cold-L2 time of every layer on its own (a one-layer sequence so that the
+    stride-2 sampling stays folded into the loads)."""
+    flush = torch.empty((FLUSH_BYTES,), dtype=torch.uint8, device="cuda")
+    rows = []
+    for i, (l, d) in enumerate(zip(table, dev)):
+        hin, win = l.h * l.in_stride, l.w * l.in_stride
+        x = synth.act_post_relu6(seed + 100 + i, (BATCH, hin, win, l.cin), device="cuda")
+        yy = torch.empty((BATCH, l.h, l.w, l.cout), dtype=torch.int8, device="cuda")
+        one = binding.LayerSeq([d])
+        wsd = torch.empty((16,), dtype=torch.uint8, device="cuda")
+        fn = lambda: binding.pw_layer_seq(one, x, wsd, y_out=yy, variant=variant)
+        med, mn = cold_time_us(torch, fn, flush)
+        m = BATCH * l.h * l.w
+        b, o = layer_bytes(m, l.cin, l.cout), layer_ops(m, l.cin, l.cout)
+        roof = max(b / bw, o / p_i8) * 1e6
+        rows.append({"i": i + 1, "name": l.name, "k": l.cin, "n": l.cout, "m": m,
+                     "stride": l.in_stride, "us": round(med, 2), "us_min": round(mn, 2),
+                     "gbs": round(b / med / 1e3, 1), "tops": round(o / med / 1e6, 1),
+                     "roof_us": round(roof, 2), "frac": round(roof / med, 3)})
+        del x, yy
+    return rows
+
+
+def single_layer_configs(torch, binding, synth, bw, p_i8):
+    """Configs 1, 2 and 4 as single layers (cold L2), every variant that runs them."""
+    flush = torch.empty((FLUSH_BYTES,), dtype=torch.uint8, device="cuda")
+    cases = [("configs[0]", 196, 64, 384, "i8"), ("configs[1]", 64 * 112 * 112, 16, 96, "relu6"),
+             ("configs[3]a", 25088, 960, 160, "u7"), ("configs[3]b", 25088, 160, 960, "u7"),
+             ("configs[3]c", 25088, 320, 1280, "u7")]
+    out = []
+    for ci, (name, m, cin, cout, act) in enumerate(cases):
+        seed = synth.BASE_SEED + 10 + ci
+        gen = {"i8": synth.act_uniform_i8, "relu6": synth.act_post_relu6,
+               "u7": synth.act_uniform_0_127}[act]
+        x = gen(seed, (m, cin), device="cuda")
+        lay = synth.make_layer(seed, cin, cout, 0.5, device="cuda")
+        wp = binding.pack_ternary(lay["w"])
+        rq = binding.make_requant(lay["bias"], lay["mult"], lay["shift"])
+        y = torch.empty((m, cout), dtype=torch.int8, device="cuda")
+        b, o = layer_bytes(m, cin, cout), layer_ops(m, cin, cout)
+        roof = max(b / bw, o / p_i8) * 1e6
+        for variant in ("tc", "smallk", "addsub"):
+            try:
+                fn = lambda: binding.pw_conv_i8(x, wp, cout, rq, y=y, variant=variant)
+                fn()
+            except binding.PromError:
+                continue
+            med, mn = cold_time_us(torch, fn, flush, iters=10 if variant == "addsub" else 20)
+            out.append({"workload": name, "m": m, "k": cin, "n": cout, "variant": variant,
+                        "us": round(med, 2), "gops": round(o / med / 1e3, 1),
+                        "gbs": round(b / med / 1e3, 1), "roof_us": round(roof, 2),
+                        "frac": round(roof / med, 4)})
+    return out
+
+
+# --------------------------------------------------------------------------- sweep
+def run_sweep(args):
+    """Shape and sparsity sweep of single layers: the tensor-core (or, where it
+    does not apply, small-K) variant and the add/sub variant on every point."""
+    import torch
+    from paper_2505_03254_b200 import binding, build, synth
+    torch.cuda.set_device(0)
+    build.build()
+    binding.lib()
+    pk = peaks()
+    bw, p_i8 = pk["hbm_gbs"] * 1e9, INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12
+    flush = torch.empty((FLUSH_BYTES,), dtype=torch.uint8, device="cuda")
+    ms_list = synth.CONFIG5_M if not args.sweep_small else synth.CONFIG5_M[:2]
+    n = 0
+    with open(args.sweep, "w") as f:
+        for m in ms_list:
+            for cin in synth.CONFIG5_CIN:
+                x = synth.act_uniform_i8(synth.BASE_SEED + 5, (m, cin), device="cuda")
+                for cout in synth.CONFIG5_COUT:
+                    y = torch.empty((m, cout), dtype=torch.int8, device="cuda")
+                    for z in synth.CONFIG5_ZERO:
+                        lay = synth.make_layer(synth.BASE_SEED + 5, cin, cout, z, device="cuda")
+                        wp = binding.pack_ternary(lay["w"])
+                        rq = binding.make_requant(lay["bias"], lay["mult"], lay["shift"])
+                        b, o = layer_bytes(m, cin, cout), layer_ops(m, cin, cout)
+                        roof = max(b / bw, o / p_i8) * 1e6
+                        nnz = int((lay["w"] != 0).sum().item())
+                        for variant in ("tc", "addsub"):
+                            used = variant
+                            try:
+                                fn = lambda: binding.pw_conv_i8(x, wp, cout, rq, y=y, variant=used)
+                                fn()
+                            except binding.PromError:
+                                used = "auto"
+                                fn = lambda: binding.pw_conv_i8(x, wp, cout, rq, y=y, variant=used)
+                                fn()
+                            iters = 5 if variant == "addsub" else 10
+                            med, mn = cold_time_us(torch, fn, flush, iters=iters, warm=1)
+                            rec = {"m": m, "k": cin, "n": cout, "zero_frac": z, "variant": variant,
+                                   "ran_as": used, "us": round(med, 2),
+                                   "gops": round(o / med / 1e3, 1), "gbs": round(b / med / 1e3, 1),
+                                   "roof_us": round(roof, 2), "frac": round(roof / med, 4),
+                                   "adds": m * nnz}
+                            f.write(json.dumps(rec) + "\n")
+                            f.flush()
+                            n += 1
+                    del y
+                del x
+    st = binding.last_device_status()
+    print(json.dumps({"sweep_points": n, "device_status": st, "file": args.sweep}), flush=True)
+    return 0 if st == binding.PROM_OK else 1
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", default="auto", choices=["auto", "tc", "naive"])
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
+    ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
+    ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.sweep:
+        return run_sweep(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -30,7 +30,7 @@ smallk_kernel(const int8_t *__restrict__ x, long long m, RowMap map,
     constexpr int CIN = KW * 4;
     extern __shared__ uint8_t sm[];
     int *ws = reinterpret_cast<int *>(sm);                       // [cout][KW] int8x4 words
-    int4 *cs = reinterpret_cast<int4 *>(sm + (size_t)cout * CIN); // {bias, mult, shift, ok}
+    int4 *cs = reinterpret_cast<int4 *>(sm + (((size_t)cout * CIN + 15) & ~(size_t)15)); // {bias, mult, shift, ok}
     // expand the weights (one byte of codes -> one word of four int8)
     bool bad_w = false;
     for (int i = threadIdx.x; i < cout * KW; i += kThreads) {
@@ -108,7 +108,7 @@ static inline prom_status launch(const int8_t *x, long long m, int cin, const Ro
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return PROM_ERR_CUDA;
-    size_t smem = (size_t)cout * cin + (size_t)cout * 16;
+    size_t smem = (((size_t)cout * cin + 15) & ~(size_t)15) + (size_t)cout * 16;
     long long blocks = (m + kThreads - 1) / kThreads;
     long long cap = (long long)sms * 8;
     int grid = (int)(blocks < cap ? blocks : cap);
