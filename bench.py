@@ -9,7 +9,7 @@ One step = the 34 pointwise layers of MobileNetV2-1.0 at 224x224 for a batch of
     python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
 
 `--impl reference` times the plain CPU oracle instead (host cores, bounded
-sample per step).  `--sweep FILE` runs the shape/sparsity sweep of single
+sample per step).  `--single M,K,N[,variant]` times one layer.  `--sweep FILE` runs the shape/sparsity sweep of single
 layers (tensor-core and add/sub variants) and writes one JSON record per point.
 """
 from __future__ import annotations
@@ -473,6 +473,37 @@ def run_sweep(args):
     return 0 if st == binding.PROM_OK else 1
 
 
+def run_single(args):
+    """One single layer M,K,N[,variant[,zero_frac]] launched a few times (for profiler captures)."""
+    import torch
+    from paper_2505_03254_b200 import binding, build, synth
+    torch.cuda.set_device(0)
+    build.build()
+    binding.lib()
+    parts = args.single.split(",")
+    m, cin, cout = int(parts[0]), int(parts[1]), int(parts[2])
+    variant = parts[3] if len(parts) > 3 else "auto"
+    z = float(parts[4]) if len(parts) > 4 else 0.5
+    pk = peaks()
+    bw, p_i8 = pk["hbm_gbs"] * 1e9, INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12
+    seed = synth.BASE_SEED + 2
+    x = synth.act_post_relu6(seed, (m, cin), device="cuda")
+    lay = synth.make_layer(seed, cin, cout, z, device="cuda")
+    wp = binding.pack_ternary(lay["w"])
+    rq = binding.make_requant(lay["bias"], lay["mult"], lay["shift"])
+    y = torch.empty((m, cout), dtype=torch.int8, device="cuda")
+    flush = torch.empty((FLUSH_BYTES,), dtype=torch.uint8, device="cuda")
+    fn = lambda: binding.pw_conv_i8(x, wp, cout, rq, y=y, variant=variant)
+    med, mn = cold_time_us(torch, fn, flush, iters=max(1, args.steps), warm=max(1, args.warmup))
+    b, o = layer_bytes(m, cin, cout), layer_ops(m, cin, cout)
+    roof = max(b / bw, o / p_i8) * 1e6
+    st = binding.last_device_status()
+    print(json.dumps({"single": [m, cin, cout], "variant": variant, "zero_frac": z, "us": med,
+                      "us_min": mn, "gbs": b / med / 1e3, "gops": o / med / 1e3, "roof_us": roof,
+                      "frac": roof / med, "device_status": st}), flush=True)
+    return 0 if st == binding.PROM_OK else 1
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -483,10 +514,13 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
+    ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.single:
+        return run_single(args)
     if args.sweep:
         return run_sweep(args)
     return run_gpu(args)
