@@ -170,6 +170,39 @@ prom_status prom_pw_layer_seq_host(const prom_layer *layers, int n,
                                    int8_t *y_out_host,
                                    prom_variant variant, void *cuda_stream);
 
+/* The ADDSUB variant of prom_pw_conv_i8 for callers that must not allocate.
+ * (The paper has no counterpart; this exists for integration reasons only.)
+ *
+ * Who needs it: the ordinary ADDSUB variant keeps its per-layer index lists in
+ * a buffer the library obtains with cudaMalloc on first use and replaces with a
+ * larger one (cudaFree + cudaMalloc) when a bigger layer comes along.  Those
+ * calls synchronise the whole device and can fail outright in a process whose
+ * memory pool or inference engine has already claimed all free device memory;
+ * a serving loop with a fixed memory budget, or a plug-in that runs inside
+ * someone else's arena, cannot afford either.  This entry point calls no
+ * cudaMalloc, cudaFree or other allocating routine, ever.
+ *
+ * How: the index lists go into a fixed array of PROM_STATIC_SCRATCH_BYTES that
+ * is part of the library's device image, so every GPU that loads the library
+ * holds that much memory until the process ends.  A layer fits when
+ *     256*ceil(cout*16/256) + 4*cout*(8*ceil(cin/8) + 8)  <=  PROM_STATIC_SCRATCH_BYTES
+ * (and cin <= 1536, the variant's own limit); cout = 1280, cin = 960 needs
+ * about 4.8 MiB.  A larger layer is refused with PROM_ERR_WORKSPACE before
+ * anything is launched.
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.  All calls
+ * on a device share the one array and each call rewrites the part it uses, so
+ * nothing needs clearing between calls, but two calls that may overlap on the
+ * GPU (different streams, no ordering between them) race on it: order them.
+ * Arguments, result and error codes are otherwise those of prom_pw_conv_i8
+ * with PROM_VARIANT_ADDSUB. */
+#define PROM_STATIC_SCRATCH_BYTES (6u << 20)
+prom_status prom_pw_conv_i8_addsub_static(const int8_t *x_dev, int64_t m, int cin,
+                                          const uint8_t *w_packed_dev, int cout,
+                                          const prom_requant *rq, int8_t *y_dev,
+                                          void *cuda_stream);
+
 /* Synchronises `cuda_stream`, then returns and clears the device status word:
  * PROM_OK, PROM_ERR_BAD_REQUANT, PROM_ERR_BAD_WEIGHT (invalid 2-bit code met
  * by a kernel) or PROM_ERR_TIMEOUT. */

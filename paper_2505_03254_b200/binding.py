@@ -27,7 +27,9 @@ EXPORTS = [
     "prom_pw_conv_i8_host", "prom_layer_seq_workspace_bytes", "prom_pw_layer_seq",
     "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
     "prom_launch_count", "prom_shutdown", "prom_status_string",
+    "prom_pw_conv_i8_addsub_static",
 ]
+STATIC_SCRATCH_BYTES = 6 << 20
 
 
 class PromRequant(C.Structure):
@@ -78,6 +80,9 @@ def lib():
         L.prom_pw_layer_seq_host.restype = i32
         L.prom_pw_layer_seq_host.argtypes = [C.POINTER(PromLayer), i32, vp, i32, i32, i32, vp, sz,
                                              vp, i32, vp]
+        L.prom_pw_conv_i8_addsub_static.restype = i32
+        L.prom_pw_conv_i8_addsub_static.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant),
+                                                    vp, vp]
         L.prom_last_device_status.restype = i32
         L.prom_last_device_status.argtypes = [vp]
         L.prom_launch_count.restype = C.c_uint64
@@ -156,6 +161,22 @@ def pw_conv_i8(x: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequa
                                  _dev(w_packed, torch.uint8, "w_packed"), cout, C.byref(rq),
                                  _dev(y, torch.int8, "y"), _variant(variant), _stream(stream)),
            "prom_pw_conv_i8")
+    return y
+
+
+def pw_conv_i8_addsub_static(x: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequant,
+                             y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """prom_pw_conv_i8_addsub_static: the add/sub variant on the library's built-in
+    scratch array, for callers that must not trigger a device allocation.  The
+    output tensor is the caller's; pass `y` to keep this wrapper from allocating too."""
+    m, cin = x.shape
+    if y is None:
+        y = torch.empty((m, cout), dtype=torch.int8, device=x.device)
+    _check(lib().prom_pw_conv_i8_addsub_static(_dev(x, torch.int8, "x"), m, cin,
+                                               _dev(w_packed, torch.uint8, "w_packed"), cout,
+                                               C.byref(rq), _dev(y, torch.int8, "y"),
+                                               _stream(stream)),
+           "prom_pw_conv_i8_addsub_static")
     return y
 
 

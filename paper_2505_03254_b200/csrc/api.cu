@@ -424,6 +424,31 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
     return PROM_OK;
 }
 
+
+// ---- the add/sub variant on built-in scratch (no allocation anywhere) --------------------
+// The index lists of the add/sub variant normally live in a buffer the library
+// grows with cudaMalloc.  This copy of the scratch is part of the loaded module
+// instead: PROM_STATIC_SCRATCH_BYTES of device memory on every GPU that loads
+// the library, held until the process exits.  In host code the array's name is
+// only a handle for the runtime, not a device address; the address a kernel can
+// use comes from cudaGetSymbolAddress, asked once per device.
+static __device__ __align__(256) uint8_t g_static_scratch[PROM_STATIC_SCRATCH_BYTES];
+
+static uint8_t *static_scratch_address()
+{
+    static std::mutex mu;
+    static std::unordered_map<int, uint8_t *> by_device;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = by_device.find(dev);
+    if (it != by_device.end()) return it->second;
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return nullptr;
+    by_device[dev] = static_cast<uint8_t *>(p);
+    return static_cast<uint8_t *>(p);
+}
+
 }  // namespace prom
 
 using namespace prom;
@@ -573,6 +598,23 @@ prom_status prom_pw_layer_seq_host(const prom_layer *layers, int n, const int8_t
     prom_status e = run_seq(layers, n, xd, batch, h0, w0, base, a + b, yd, variant, st);
     if (e != PROM_OK) return e;
     return cuda_status(cudaMemcpyAsync(y_out_host, yd, yout_raw, cudaMemcpyDeviceToHost, st));
+}
+
+prom_status prom_pw_conv_i8_addsub_static(const int8_t *x_dev, int64_t m, int cin,
+                                          const uint8_t *w_packed_dev, int cout,
+                                          const prom_requant *rq, int8_t *y_dev,
+                                          void *cuda_stream)
+{
+    prom_status s = check_conv(x_dev, m, cin, w_packed_dev, cout, rq, y_dev);
+    if (s != PROM_OK) return s;
+    if (cin > addsub::kMaxCin) return PROM_ERR_UNSUPPORTED;
+    if (addsub::scratch_bytes(cout, cin) > (size_t)PROM_STATIC_SCRATCH_BYTES)
+        return PROM_ERR_WORKSPACE;
+    if (m == 0) return PROM_OK;
+    uint8_t *scratch = static_scratch_address();
+    if (!scratch) return PROM_ERR_CUDA;
+    return addsub::launch_on(x_dev, m, cin, RowMap{1, 1, 1, 1, 1}, w_packed_dev, cout, *rq, y_dev,
+                             scratch, static_cast<cudaStream_t>(cuda_stream), g_launches);
 }
 
 prom_status prom_last_device_status(void *cuda_stream)
