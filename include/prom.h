@@ -212,6 +212,17 @@ prom_status prom_last_device_status(void *cuda_stream);
  * streams, this process); used by the benchmark to count launches. */
 uint64_t prom_launch_count(void);
 
+/* Tuning aid for the TC variant: forces the row fold, the subtile width, the
+ * number of output-channel groups, CTAs per SM (1 or 2) and the depth of the
+ * activation ring of later calls; 0 leaves a choice to the library.  A forced
+ * combination that does not fit makes TC report PROM_ERR_UNSUPPORTED.  Results
+ * never depend on the plan.  Not thread-safe.  prom_debug_tc_plan_query
+ * writes the plan the library would use for a plain [m][cin] x [cout] layer
+ * ({fold, nt, groups, grid, stages, accumulators, shared bytes, chunk bytes,
+ * estimate in 1/100 us}) and returns 1, or returns 0 if TC cannot run it. */
+void prom_debug_tc_plan(int fold, int nt, int groups, int occ, int stages);
+int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
+
 /* Frees the library's internal caches (all devices).  Optional. */
 void prom_shutdown(void);
 

@@ -27,7 +27,7 @@ EXPORTS = [
     "prom_pw_conv_i8_host", "prom_layer_seq_workspace_bytes", "prom_pw_layer_seq",
     "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
     "prom_launch_count", "prom_shutdown", "prom_status_string",
-    "prom_pw_conv_i8_addsub_static",
+    "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -83,6 +83,10 @@ def lib():
         L.prom_pw_conv_i8_addsub_static.restype = i32
         L.prom_pw_conv_i8_addsub_static.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant),
                                                     vp, vp]
+        L.prom_debug_tc_plan.restype = None
+        L.prom_debug_tc_plan.argtypes = [i32, i32, i32, i32, i32]
+        L.prom_debug_tc_plan_query.restype = i32
+        L.prom_debug_tc_plan_query.argtypes = [i64, i32, i32, C.POINTER(C.c_int)]
         L.prom_last_device_status.restype = i32
         L.prom_last_device_status.argtypes = [vp]
         L.prom_launch_count.restype = C.c_uint64
@@ -130,6 +134,20 @@ def launch_count() -> int:
 
 def last_device_status(stream=None) -> int:
     return int(lib().prom_last_device_status(_stream(stream)))
+
+
+def debug_tc_plan(fold: int = 0, nt: int = 0, groups: int = 0, occ: int = 0, stages: int = 0) -> None:
+    """prom_debug_tc_plan: force parts of the tensor-core launch plan (0 = automatic)."""
+    lib().prom_debug_tc_plan(fold, nt, groups, occ, stages)
+
+
+def debug_tc_plan_query(m: int, cin: int, cout: int):
+    """prom_debug_tc_plan_query: the plan for a plain layer as a dict, or None."""
+    out = (C.c_int * 9)()
+    if not lib().prom_debug_tc_plan_query(m, cin, cout, out):
+        return None
+    keys = ("fold", "nt", "groups", "grid", "stages", "nbuf", "smem", "cw", "est_us_x100")
+    return dict(zip(keys, list(out)))
 
 
 def shutdown() -> None:

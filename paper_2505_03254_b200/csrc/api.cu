@@ -25,6 +25,7 @@ static std::atomic<uint64_t> g_launches{0};
 struct DeviceInfo {
     int sms = 0;
     int smem_optin = 0;
+    int smem_total = 0;   // shared memory per SM
     bool ok = false;
 };
 
@@ -40,6 +41,8 @@ static DeviceInfo device_info()
     if (it != cache.end()) return it->second;
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
         cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) ==
+            cudaSuccess &&
+        cudaDeviceGetAttribute(&d.smem_total, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) ==
             cudaSuccess)
         d.ok = true;
     cache[dev] = d;
@@ -130,57 +133,40 @@ static EncodeTiledFn encode_tiled_fn()
 
 struct TcPlan {
     tc::Params p;
-    CUtensorMap xmap;
+    CUtensorMap xmap, ymap;
     int grid = 0;
     size_t smem = 0;
+    double est_us = 0;
 };
+
+// Tuning override (0 = automatic), set by prom_debug_tc_plan.
+struct TcTune { int fold, nt, groups, occ, stages; };
+static TcTune g_tune = {0, 0, 0, 0, 0};
 
 static int round_up(int v, int a) { return (v + a - 1) / a * a; }
 
-// Fills everything of the plan that does not depend on pointers.  Returns
-// false when the tensor-core variant cannot run this shape.
-static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
-                          TcPlan &pl)
+// Everything of a plan that follows from (fold, nt, groups, occ); false when it does not fit.
+static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
+                         int fold, int nt, int groups, int occ, int want_stages, TcPlan &pl)
 {
     tc::Params &p = pl.p;
     memset(&p, 0, sizeof(p));
-    if (m <= 0 || (cin & 7) || (cout & 7)) return false;
-    int fold = 1;
-    if ((cin & 15) != 0) fold = 2;
-    if (fold == 2 && (map.stride != 1 || (m & 1))) return false;
-    int kf = cin * fold, nf = cout * fold;
-    if (kf > 4096) return false;
-
-    // subtiles: equal widths that divide nf, multiples of 16 (or a single 8-multiple one)
-    const int smem_max = d.smem_optin;
-    int n_sub = 0, nt = 0, groups = 1, subs_per_cta = 1, kc = (kf + 127) / 128;
-    size_t w_bytes = 0;
-    for (int s = (nf + 255) / 256; s <= nf / 8; ++s) {
-        if (nf % s) continue;
-        int w = nf / s;
-        if (s > 1 && (w & 15)) continue;
-        if (s == 1 && (w & 7)) continue;
-        int wp = round_up(w, 16);
-        size_t per_sub = (size_t)kc * wp * 128;
-        // resident weights must leave room for two activation stages and the staging rows
-        size_t fixed = 2 * tc::kStageBytes + 4 * 32 * (size_t)(w + 16) + (size_t)wp * 16 + 2048;
-        if (per_sub + fixed > (size_t)smem_max) continue;
-        n_sub = s; nt = w;
-        if ((size_t)s * per_sub <= 98304 && (size_t)s * per_sub + fixed + (size_t)(s - 1) * wp * 16 <=
-                                                (size_t)smem_max) {
-            groups = 1; subs_per_cta = s; w_bytes = (size_t)s * per_sub;
-        } else {
-            groups = s; subs_per_cta = 1; w_bytes = per_sub;
-        }
-        break;
-    }
-    if (!n_sub) return false;
-    if (n_sub == 1 && (nt & 15) && (nf != nt)) return false;
+    const int kf = cin * fold, nf = cout * fold;
+    if (kf > 4096 || nf % nt) return false;
+    const int n_sub = nf / nt;
+    if (n_sub % groups) return false;
+    if (n_sub > 1 && ((nt & 15) || (nf & 15))) return false;     // tensor-map stores
+    if (n_sub == 1 && (nt & 7)) return false;
+    const int subs = n_sub / groups;
+    const int nt_pad = round_up(nt, 16);
+    if (nt_pad > 256) return false;
+    const int cw = kf <= 32 ? 32 : (kf <= 64 ? 64 : 128);
+    const int kc = (kf + cw - 1) / cw;
 
     // tile rows
     int tm = 128, x3d = 0, box_r = 0;
     if (map.stride != 1) {
-        if (map.wo > 128) return false;
+        if (fold != 1 || map.wo > 128) return false;
         box_r = 128 / map.wo;
         long long lines = m / map.wo;          // batch * ho
         if (box_r > lines) box_r = (int)lines;
@@ -188,96 +174,169 @@ static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, con
         tm = box_r * map.wo;
         x3d = 1;
     }
-    const int mode_b = (nt & 15) ? 1 : 0;
-    if (mode_b && (tm & 1)) return false;
-    long long rows = m / fold;
-    long long n_mtiles = (rows + tm - 1) / tm;
+    const long long rows = m / fold;
+    if ((nf & 15) && (tm & 1)) return false;     // slabs of the 1-D store start on 16-byte granules
+    const long long n_mtiles = (rows + tm - 1) / tm;
     if (n_mtiles > 0x7fffffff) return false;
 
-    p.m_rows = rows; p.k0 = cin; p.n0 = cout; p.fold = fold; p.kf = kf; p.nf = nf;
-    p.tm = tm; p.n_mtiles = (int)n_mtiles; p.nt = nt; p.nt_pad = round_up(nt, 16);
-    p.n_sub = n_sub; p.groups = groups; p.subs_per_cta = subs_per_cta;
-    p.kc = kc;
-    int ksteps = (kf + 31) / 32;
-    p.ksteps_last = ksteps - 4 * (kc - 1);
-    p.acc_bufs = 2;
-    int cols = 2 * p.nt_pad, tc_cols = 32;
-    while (tc_cols < cols) tc_cols *= 2;
-    p.tmem_cols = tc_cols;
-    p.mode_b = mode_b;
-    p.out_pitch = mode_b ? nt : ((((nt >> 4) & 1) == 0) ? nt + 16 : nt);
-    p.x3d = x3d; p.box_r = box_r;
-    p.tx_bytes = x3d ? (uint32_t)(128 * map.wo * box_r) : (uint32_t)tc::kStageBytes;
-    p.inv_cpr = mode_b ? 0 : (uint32_t)(((1u << 20) + (nt >> 4) - 1) / (nt >> 4));
-
-    // shared-memory layout (offsets from the 1024-aligned base)
-    const int ncols_res = subs_per_cta * p.nt_pad;
-    const size_t out_bytes = (size_t)tc::kEpiWarps * 32 * p.out_pitch;
-    const size_t tail = round_up((int)out_bytes, 16) + (size_t)ncols_res * 8 + (size_t)ncols_res * 4 +
-                        round_up(ncols_res, 16) + 256;
-    // stages: 2 CTAs per SM when everything fits in half the shared memory with >= 3
-    // stages and 256 TMEM columns; otherwise one CTA with as many stages as fit (<= 8)
-    const size_t half = (size_t)(smem_max / 2) - 1024 - 1024;   // per-CTA share minus slack
-    int stages;
-    int occ = 1;
-    size_t base_need = w_bytes + tail;
-    if (p.tmem_cols <= 256 && base_need + 3 * (size_t)tc::kStageBytes <= half) {
-        occ = 2;
-        stages = (int)((half - base_need) / tc::kStageBytes);
+    // tensor memory: two CTAs share the 512 columns, or one takes them all
+    int tmem_cols;
+    if (occ == 2) {
+        if (2 * nt_pad > 256) return false;
+        tmem_cols = 256;
     } else {
-        stages = (int)(((size_t)smem_max - 1024 - base_need) / tc::kStageBytes);
+        tmem_cols = 512;
     }
+    int nbuf = tmem_cols / nt_pad;
+    if (nbuf > tc::kMaxBufs) nbuf = tc::kMaxBufs;
+    if (nbuf < 2) return false;
+
+    const int ncols = subs * nt_pad;
+    const size_t stage_bytes = (size_t)128 * cw;
+    const size_t w_bytes = (size_t)subs * kc * nt_pad * cw;
+    const size_t wbias_bytes = (size_t)subs * nt_pad * 32;
+    const size_t out_bytes = (size_t)tc::kEpiWarps * 32 * nt;
+    const size_t fixed = w_bytes + wbias_bytes + tc::kAConstBytes + round_up((int)out_bytes, 128) +
+                         (size_t)ncols * 12 + tc::kLuts * 1024 + 256 + 1024 /* alignment slack */;
+    const size_t budget = occ == 2 ? (size_t)((d.smem_total - 2 * 1024) / 2) : (size_t)d.smem_optin;
+    if (budget > (size_t)d.smem_optin || fixed + 2 * stage_bytes > budget) return false;
+    int stages = (int)((budget - fixed) / stage_bytes);
+    const int share_x = (kc == 1 && subs > 1) ? 1 : 0;
+    int cap = share_x ? 4 : (kc >= 4 ? tc::kMaxStages : 6);
+    if (want_stages > 0) cap = want_stages;
+    if (stages > cap) stages = cap;
     if (stages > tc::kMaxStages) stages = tc::kMaxStages;
-    int need_stages = kc < 2 ? 2 : 2;
-    if (stages < need_stages) return false;
-    p.stages = stages;
-    uint32_t off = (uint32_t)stages * tc::kStageBytes;
+    if (stages < 2) return false;
+
+    p.m_rows = rows; p.k0 = cin; p.n0 = cout; p.fold = fold; p.kf = kf; p.nf = nf;
+    p.tm = tm; p.n_mtiles = (int)n_mtiles; p.nt = nt; p.nt_pad = nt_pad;
+    p.n_sub = n_sub; p.groups = groups; p.subs_per_cta = subs;
+    p.cw = cw; p.kc = kc;
+    p.ksteps_last = (kf - (kc - 1) * cw + 31) / 32;
+    p.stages = stages; p.nbuf = nbuf; p.tmem_cols = tmem_cols;
+    p.share_x = share_x;
+    p.store_2d = n_sub > 1 ? 1 : 0;
+    p.x3d = x3d; p.box_r = box_r;
+    p.tx_bytes = x3d ? (uint32_t)(cw * map.wo * box_r) : (uint32_t)stage_bytes;
+
+    uint32_t off = (uint32_t)(stages * stage_bytes);
     p.off_w = off; off += (uint32_t)w_bytes;
-    p.off_out = off; off += (uint32_t)round_up((int)out_bytes, 16);
-    p.off_consts = off; off += (uint32_t)ncols_res * 8;
-    p.off_shift = off; off += (uint32_t)ncols_res * 4;
-    p.off_wmag = off; off += (uint32_t)round_up(ncols_res, 16);
+    p.off_wbias = off; off += (uint32_t)wbias_bytes;
+    p.off_aconst = off; off += tc::kAConstBytes;
+    p.off_out = off; off += (uint32_t)round_up((int)out_bytes, 128);
+    p.off_mult = off; off += (uint32_t)ncols * 4;
+    p.off_bs = off; off += (uint32_t)ncols * 8;
+    p.off_lut = off; off += tc::kLuts * 1024;
     p.off_bars = off; off += 256;
     pl.smem = (size_t)off + 1024;
-    if (occ == 1 && p.tmem_cols == 512 && pl.smem * 2 <= (size_t)smem_max)
-        pl.smem = (size_t)smem_max / 2 + 1024;     // keep a second CTA (and its TMEM request) off the SM
-    if (pl.smem > (size_t)smem_max) return false;
+    if (occ == 1 && pl.smem * 2 + 2048 <= (size_t)d.smem_total)
+        pl.smem = (size_t)d.smem_total / 2;       // keep a second CTA (and its TMEM request) off the SM
+    if (pl.smem > (size_t)d.smem_optin) return false;
 
-    long long slots = (long long)d.sms * occ;
+    const long long slots = (long long)d.sms * occ;
     long long workers = slots / groups;
     if (workers < 1) workers = 1;
     if (workers > n_mtiles) workers = n_mtiles;
     pl.grid = (int)(workers * groups);
+
+    // rough time model (microseconds) used only to rank candidate plans
+    const double rounds = (double)((n_mtiles + workers - 1) / workers);
+    const double ctas_per_sm = (double)pl.grid / d.sms < 1.0 ? 1.0
+                               : ((double)pl.grid / d.sms > occ ? occ : (double)pl.grid / d.sms);
+    const double epi_rate = 30e3 / ctas_per_sm;              // outputs per microsecond per CTA
+    const double load_rate = 70e3 / ctas_per_sm;             // bytes per microsecond per CTA
+    const double t_epi = (double)tm * nt / epi_rate;
+    const double t_load = (double)kc * tm * (kf < cw ? kf : cw) / load_rate;
+    const double t_unit_first = (t_epi > t_load ? t_epi : t_load) + 0.15;
+    const double t_unit_next = share_x ? t_epi + 0.15 : t_unit_first;
+    const double pieces = (double)ncols * kc * (cw / 16);
+    const double prologue = 1.5 + pieces * 20.0 / 32.0 / (1.2 / ctas_per_sm) / 1900.0;
+    const double t_cta = prologue + rounds * (t_unit_first + (subs - 1) * t_unit_next) + 1.5;
+    const double bytes = (double)m * cin * (share_x || groups == 1 ? 1.0 : 1.0) + (double)m * cout;
+    const double t_mem = bytes / 6.0e6;
+    pl.est_us = t_cta > t_mem ? t_cta : t_mem;
     return true;
 }
 
-static bool tc_make_map(const Conv &c, TcPlan &pl)
+// Picks fold, subtile width, channel groups and occupancy.  Returns false when
+// the tensor-core variant cannot run this shape.
+static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
+                          TcPlan &best)
+{
+    if (m <= 0 || (cin & 7) || (cout & 7)) return false;
+    int fold = 1;
+    if (map.stride == 1) {
+        if ((cin & 15) || ((cout & 15) && m % 2 == 0)) fold = 2;
+        if (m % fold) return false;
+        while (fold * 2 <= 8 && fold * 2 * cin <= 128 && fold * 2 * cout <= 128 &&
+               m % (fold * 2) == 0)
+            fold *= 2;
+    }
+    if (g_tune.fold > 0) fold = g_tune.fold;
+    if (fold < 1 || fold > 8 || m % fold) return false;
+    const int nf = cout * fold;
+    bool found = false;
+    for (int nt = 8; nt <= 256 && nt <= nf; nt += 8) {
+        if (nf % nt) continue;
+        if (g_tune.nt > 0 && nt != g_tune.nt) continue;
+        const int n_sub = nf / nt;
+        for (int groups = 1; groups <= n_sub; ++groups) {
+            if (n_sub % groups) continue;
+            if (g_tune.groups > 0 && groups != g_tune.groups) continue;
+            for (int occ = 2; occ >= 1; --occ) {
+                if (g_tune.occ > 0 && occ != g_tune.occ) continue;
+                TcPlan pl;
+                if (!tc_fill_plan(m, cin, cout, map, d, fold, nt, groups, occ, g_tune.stages, pl))
+                    continue;
+                if (!found || pl.est_us < best.est_us) { best = pl; found = true; }
+            }
+        }
+    }
+    return found;
+}
+
+static bool tc_make_maps(const Conv &c, TcPlan &pl)
 {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
     const tc::Params &p = pl.p;
+    const CUtensorMapSwizzle sw = p.cw == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : (p.cw == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
     CUresult r;
     if (!p.x3d) {
         cuuint64_t dims[2] = {(cuuint64_t)p.kf, (cuuint64_t)p.m_rows};
         cuuint64_t strides[1] = {(cuuint64_t)p.kf};
-        cuuint32_t box[2] = {128, 128};
+        cuuint32_t box[2] = {(cuuint32_t)p.cw, 128};
         cuuint32_t es[2] = {1, 1};
         r = enc(&pl.xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(c.x), dims, strides,
-                box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     } else {
         // [channel][wo, step stride*cin][batch*ho, step stride*win*cin]
         const RowMap &mp = c.map;
         cuuint64_t dims[3] = {(cuuint64_t)c.cin, (cuuint64_t)mp.wo, (cuuint64_t)(c.m / mp.wo)};
         cuuint64_t strides[2] = {(cuuint64_t)mp.stride * c.cin,
                                  (cuuint64_t)mp.stride * mp.win * c.cin};
-        cuuint32_t box[3] = {128, (cuuint32_t)mp.wo, (cuuint32_t)p.box_r};
+        cuuint32_t box[3] = {(cuuint32_t)p.cw, (cuuint32_t)mp.wo, (cuuint32_t)p.box_r};
         cuuint32_t es[3] = {1, 1, 1};
         r = enc(&pl.xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t *>(c.x), dims, strides,
-                box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     }
-    return r == CUDA_SUCCESS;
+    if (r != CUDA_SUCCESS) return false;
+    if (p.store_2d) {
+        cuuint64_t dims[2] = {(cuuint64_t)p.nf, (cuuint64_t)p.m_rows};
+        cuuint64_t strides[1] = {(cuuint64_t)p.nf};
+        cuuint32_t box[2] = {(cuuint32_t)p.nt, 32};
+        cuuint32_t es[2] = {1, 1};
+        r = enc(&pl.ymap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, c.y, dims, strides, box, es,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return false;
+    } else {
+        pl.ymap = pl.xmap;      // unused by the kernel
+    }
+    return true;
 }
 
 static prom_status launch_tc(const Conv &c)
@@ -286,7 +345,7 @@ static prom_status launch_tc(const Conv &c)
     if (!d.ok) return PROM_ERR_CUDA;
     TcPlan pl;
     if (!tc_shape_plan(c.m, c.cin, c.cout, c.map, d, pl)) return PROM_ERR_UNSUPPORTED;
-    if (!tc_make_map(c, pl)) return PROM_ERR_CUDA;
+    if (!tc_make_maps(c, pl)) return PROM_ERR_CUDA;
     tc::Params &p = pl.p;
     p.w_packed = c.w; p.bias = c.rq.bias; p.mult = c.rq.mult; p.shift = c.rq.shift;
     p.act_min = c.rq.act_min; p.act_max = c.rq.act_max; p.y = c.y; p.pdl = c.pdl ? 1 : 0;
@@ -312,7 +371,7 @@ static prom_status launch_tc(const Conv &c)
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
-    cudaError_t e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel, pl.xmap, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel, pl.xmap, pl.ymap, p);
     ++g_launches;
     return cuda_status(e);
 }
@@ -633,6 +692,23 @@ prom_status prom_last_device_status(void *cuda_stream)
 }
 
 uint64_t prom_launch_count(void) { return g_launches.load(); }
+
+void prom_debug_tc_plan(int fold, int nt, int groups, int occ, int stages)
+{
+    g_tune = TcTune{fold, nt, groups, occ, stages};
+}
+
+int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9)
+{
+    DeviceInfo d = device_info();
+    if (!d.ok || !out9) return 0;
+    TcPlan pl;
+    if (!tc_shape_plan(m, cin, cout, RowMap{1, 1, 1, 1, 1}, d, pl)) return 0;
+    const tc::Params &p = pl.p;
+    out9[0] = p.fold; out9[1] = p.nt; out9[2] = p.groups; out9[3] = pl.grid; out9[4] = p.stages;
+    out9[5] = p.nbuf; out9[6] = (int)pl.smem; out9[7] = p.cw; out9[8] = (int)(pl.est_us * 100);
+    return 1;
+}
 
 void prom_shutdown(void) { addsub::release_cache(); }
 

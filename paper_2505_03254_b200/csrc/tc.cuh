@@ -1,23 +1,30 @@
 // The tensor-core variant: TMA-staged int8 activation tiles, ternary weights
 // expanded from their 2-bit form into shared memory once per CTA, tcgen05
-// int8 MMAs accumulating in tensor memory, and a fused requantising epilogue.
+// int8 MMAs accumulating in tensor memory, and a fused requantising epilogue
+// whose int8 rows leave through bulk (TMA) stores.
 //
 // Work decomposition
 //   tile      = `tm` consecutive output rows (<= 128; one MMA M block)
-//   subtile   = `nt` consecutive output channels (<= 256; one accumulator)
-//   K chunk   = 128 bytes of a row (one TMA box, one swizzle-128B atom wide)
+//   subtile   = `nt` consecutive output channels (one accumulator, <= 256)
+//   K chunk   = `cw` bytes of a row (32, 64 or 128: one TMA box, one swizzle span)
+//   unit      = (tile, subtile)
 // A CTA keeps the expanded weights of its subtiles resident for its whole
-// life and walks over tiles; warp 0 issues TMA loads, warp 1 issues MMAs,
-// warps 2..5 drain the accumulators (one TMEM lane quarter each).
+// life and walks over tiles.  Warp 0 issues TMA loads, warp 1 issues MMAs,
+// warps 2..9 are two epilogue groups of four warps (one TMEM lane quarter
+// each) that take units alternately.
 //
-// Row folding: when cin or cout is not a multiple of 16 the matrices are
-// viewed as X'[M/2][2*cin], Y'[M/2][2*cout] and the weights as the block
-// diagonal [[W,0],[0,W]]; Y' is then byte-for-byte the same memory as Y.
+// Row folding: with fold f the matrices are viewed as X'[M/f][f*cin],
+// Y'[M/f][f*cout] and the weights as the block diagonal diag(W, .., W); X' and
+// Y' are byte for byte the same memory as X and Y.  It makes channel counts
+// that are not multiples of 16 legal for TMA and gives tiny layers wider tiles.
 //
 // Fast epilogue (clamp [0,127], shifts of the CTA's channels within 4 of one
 // another, no overflow): channel c's weights are expanded as
-// +-2^(2+shmax-shift[c]), so that TMEM holds acc*2^(2+shmax-shift[c]) and
-//     v1 = (hi32((tmem + bias') * mult) + 2^shmax) >> shmax
+// +-2^(2+shmax-shift[c]) and its bias, scaled the same way, enters the
+// accumulator through one extra MMA k-step (a constant A block of 1s and 127s
+// against a block of base-127 bias digits), so that TMEM holds
+// t' = (acc + bias) * 2^(2+shmax-shift[c]) and
+//     v1 = (hi32(t' * mult) + 2^shmax) >> shmax
 // equals floor(t*mult / 2^(30+shift)) + 1 exactly; the result is
 // sat_u8(v1) >> 1.  Everything else takes the 64-bit definition.
 #pragma once
@@ -27,40 +34,41 @@
 
 namespace prom { namespace tc {
 
-constexpr int kThreads = 192;
-constexpr int kEpiWarps = 4;
-constexpr int kStageBytes = 128 * 128;
+constexpr int kThreads = 320;
+constexpr int kEpiWarps = 8;
+constexpr int kEpiGroups = 2;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 constexpr int kMaxStages = 8;
+constexpr int kMaxBufs = 4;
+constexpr int kLuts = 6;                 // magnitude 1, then 4, 8, 16, 32, 64
+constexpr int kAConstBytes = 128 * 32;
+constexpr int kBiasHiDigits = 30;        // A-const row: 1, 1, then 30 x 127
+constexpr int kBiasMax = 127 * 127 * kBiasHiDigits;
 
 struct Params {
     long long m_rows;   // rows of the folded problem
     int k0, n0;         // layer cin, cout
-    int fold;           // 1 or 2
+    int fold;
     int kf, nf;         // folded cin, cout
     int tm;             // rows per tile
     int n_mtiles;
     int nt, nt_pad;     // subtile width, MMA N
     int n_sub, groups, subs_per_cta;
+    int cw;             // chunk row bytes (32, 64, 128) = swizzle span
     int kc;             // K chunks per tile
-    int ksteps_last;    // 32-wide MMA steps in the last chunk (1..4)
-    int stages, acc_bufs, tmem_cols;
-    int out_pitch;      // staging row pitch in bytes
-    int mode_b;         // 1: nt % 16 == 8, linear staging
+    int ksteps_last;    // 32-wide MMA steps in the last chunk
+    int stages, nbuf, tmem_cols;
+    int share_x;        // kc == 1: one activation load serves all subtiles of the tile
+    int store_2d;       // 0: rows of a slab are contiguous in Y (one subtile), 1: tensor-map store
     int x3d, box_r;     // 3-D activation map (strided input); rows of dim 2 per tile
     uint32_t tx_bytes;
-    uint32_t inv_cpr;   // ceil(2^20 / (nt/16))
-    uint32_t off_w, off_out, off_consts, off_shift, off_wmag, off_bars;
+    uint32_t off_w, off_wbias, off_aconst, off_out, off_mult, off_bs, off_lut, off_bars;
     const uint8_t *w_packed;
     const int32_t *bias, *mult;
     const int8_t *shift;
     int act_min, act_max;
     int8_t *y;
     int pdl;            // launched with programmatic dependent launch
-};
-
-struct Ctx {
-    volatile int *abort_flag;
 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag)
@@ -80,21 +88,20 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 
-// K-major, 128-byte swizzle: 8-row atoms of 1024 bytes, stride 1024 between atoms.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
+// K-major operand with rows of `cw` bytes swizzled over a span of `cw` bytes:
+// 8-row atoms of 8*cw bytes, one after the other.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t cw)
 {
-    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) |
-           (2ull << 61);
+    const uint64_t mode = cw == 128 ? 2ull : (cw == 64 ? 4ull : 6ull);
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)((8u * cw) >> 4) << 32) |
+           (1ull << 46) | (mode << 61);
 }
 
-// 4 two-bit codes (one byte) -> 4 int8 lanes of magnitude `mag` / (256 - mag).
-__device__ __forceinline__ uint32_t expand4(uint32_t byte, uint32_t mag, uint32_t negmag,
-                                            uint32_t &invalid)
+// 16-byte piece j of row n inside a swizzled block with rows of cw bytes.
+__device__ __forceinline__ uint32_t swz_offset(uint32_t n, uint32_t j, uint32_t cw)
 {
-    uint32_t x = (byte | (byte << 6) | (byte << 12) | (byte << 18)) & 0x03030303u;
-    uint32_t b0 = x & 0x01010101u, b1 = (x >> 1) & 0x01010101u;
-    invalid |= b1 & ~b0;
-    return (b0 & ~b1) * mag + (b0 & b1) * negmag;
+    const uint32_t x = cw == 128 ? (n & 7u) : (cw == 64 ? ((n >> 1) & 3u) : ((n >> 2) & 1u));
+    return n * cw + ((j ^ x) << 4);
 }
 
 template <int NC>
@@ -105,12 +112,28 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&v)[NC])
     else ptx::tmem_ld_x8(taddr, v);
 }
 
-// Drain NC accumulator columns of this thread's row, requantise, and write the
-// packed bytes to the staging row.
-template <int NC, bool FAST>
-__device__ __forceinline__ void epi_cols(uint32_t taddr, const int2 *__restrict__ cb,
-                                         const int *__restrict__ csh, int shmax, int lo, int hi,
-                                         uint8_t *dst, bool mode_b)
+// Rows of the staging slab are nt bytes apart: 16-byte aligned only when nt is a
+// multiple of 16 (`wide`), 8-byte aligned otherwise.
+template <int NC>
+__device__ __forceinline__ void put_row(uint8_t *dst, const uint32_t (&out)[NC / 4], bool wide)
+{
+    if (NC >= 16 && wide) {
+#pragma unroll
+        for (int i = 0; i < NC / 16; ++i)
+            *reinterpret_cast<uint4 *>(dst + 16 * i) =
+                make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < NC / 8; ++i)
+            *reinterpret_cast<uint2 *>(dst + 8 * i) = make_uint2(out[2 * i], out[2 * i + 1]);
+    }
+}
+
+// NC accumulator columns of this thread's row: one mad.hi and one shift per
+// value, saturating pack, halve.
+template <int NC>
+__device__ __forceinline__ void epi_fast(uint32_t taddr, const int *__restrict__ cm, int shmax,
+                                         uint8_t *dst, bool wide)
 {
     uint32_t v[NC];
     tmem_ld<NC>(taddr, v);
@@ -119,61 +142,66 @@ __device__ __forceinline__ void epi_cols(uint32_t taddr, const int2 *__restrict_
     const int r = 1 << shmax;
 #pragma unroll
     for (int c = 0; c < NC; c += 4) {
-        int q[4];
-#pragma unroll
-        for (int e = 0; e < 4; e += 2) {
-            int4 bm = *reinterpret_cast<const int4 *>(cb + c + e);   // two channels
-            if constexpr (FAST) {
-                q[e] = ptx::mad_hi((int)v[c + e] + bm.x, bm.y, r) >> shmax;
-                q[e + 1] = ptx::mad_hi((int)v[c + e + 1] + bm.z, bm.w, r) >> shmax;
-            } else {
-                q[e] = requant_exact((int)v[c + e] + bm.x, bm.y, csh[c + e], lo, hi);
-                q[e + 1] = requant_exact((int)v[c + e + 1] + bm.z, bm.w, csh[c + e + 1], lo, hi);
-            }
-        }
-        if constexpr (FAST) {
-            uint32_t w = ptx::pack_sat_u8(q[3], q[2], 0u);
-            w = ptx::pack_sat_u8(q[1], q[0], w);
-            out[c / 4] = (w >> 1) & 0x7F7F7F7Fu;
-        } else {
-            out[c / 4] = ((uint32_t)q[0] & 0xFFu) | (((uint32_t)q[1] & 0xFFu) << 8) |
-                         (((uint32_t)q[2] & 0xFFu) << 16) | (((uint32_t)q[3] & 0xFFu) << 24);
-        }
+        const int4 mu = *reinterpret_cast<const int4 *>(cm + c);
+        const int q0 = ptx::mad_hi((int)v[c], mu.x, r) >> shmax;
+        const int q1 = ptx::mad_hi((int)v[c + 1], mu.y, r) >> shmax;
+        const int q2 = ptx::mad_hi((int)v[c + 2], mu.z, r) >> shmax;
+        const int q3 = ptx::mad_hi((int)v[c + 3], mu.w, r) >> shmax;
+        uint32_t w = ptx::pack_sat_u8(q3, q2, 0u);
+        w = ptx::pack_sat_u8(q1, q0, w);
+        out[c / 4] = (w >> 1) & 0x7F7F7F7Fu;
     }
-    if (!mode_b) {
-        if constexpr (NC >= 16) {
+    put_row<NC>(dst, out, wide);
+}
+
+// The 64-bit definition (any clamp, any shifts).
+template <int NC>
+__device__ __forceinline__ void epi_exact(uint32_t taddr, const int *__restrict__ cm,
+                                          const int2 *__restrict__ cbs, int lo, int hi, uint8_t *dst,
+                                          bool wide)
+{
+    uint32_t v[NC];
+    tmem_ld<NC>(taddr, v);
+    ptx::tmem_wait_ld();
+    uint32_t out[NC / 4];
 #pragma unroll
-            for (int i = 0; i < NC / 16; ++i)
-                *reinterpret_cast<uint4 *>(dst + 16 * i) =
-                    make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
+    for (int c = 0; c < NC; c += 4) {
+        uint32_t w = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int2 bs = cbs[c + e];
+            const int q = requant_exact((int)v[c + e] + bs.x, cm[c + e], bs.y, lo, hi);
+            w |= ((uint32_t)q & 0xFFu) << (8 * e);
         }
-    } else {
-#pragma unroll
-        for (int i = 0; i < NC / 8; ++i)
-            *reinterpret_cast<uint2 *>(dst + 8 * i) = make_uint2(out[2 * i], out[2 * i + 1]);
+        out[c / 4] = w;
     }
+    put_row<NC>(dst, out, wide);
 }
 
 template <bool FAST>
-__device__ __forceinline__ void epi_subtile(const Params &p, uint32_t taddr, const int2 *cb,
-                                            const int *csh, int shmax, uint8_t *dst_row)
+__device__ __forceinline__ void epi_subtile(const Params &p, uint32_t taddr, const int *cm,
+                                            const int2 *cbs, int shmax, uint8_t *dst_row)
 {
+    const bool wide = (p.nt & 15) == 0;
     int c = 0;
-    for (; c + 32 <= p.nt; c += 32)
-        epi_cols<32, FAST>(taddr + c, cb + c, csh + c, shmax, p.act_min, p.act_max, dst_row + c,
-                           p.mode_b);
+    for (; c + 32 <= p.nt; c += 32) {
+        if constexpr (FAST) epi_fast<32>(taddr + c, cm + c, shmax, dst_row + c, wide);
+        else epi_exact<32>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide);
+    }
     if (c + 16 <= p.nt) {
-        epi_cols<16, FAST>(taddr + c, cb + c, csh + c, shmax, p.act_min, p.act_max, dst_row + c,
-                           p.mode_b);
+        if constexpr (FAST) epi_fast<16>(taddr + c, cm + c, shmax, dst_row + c, wide);
+        else epi_exact<16>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide);
         c += 16;
     }
-    if (c + 8 <= p.nt)
-        epi_cols<8, FAST>(taddr + c, cb + c, csh + c, shmax, p.act_min, p.act_max, dst_row + c,
-                          true);
+    if (c + 8 <= p.nt) {
+        if constexpr (FAST) epi_fast<8>(taddr + c, cm + c, shmax, dst_row + c, wide);
+        else epi_exact<8>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide);
+    }
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
-tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const Params p)
+__global__ void __launch_bounds__(kThreads, 2)
+tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
+               const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>(
@@ -182,39 +210,45 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const Params p)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     uint8_t *w_smem = smem + p.off_w;
-    int2 *cb = reinterpret_cast<int2 *>(smem + p.off_consts);       // {bias', mult} per column
-    int *csh = reinterpret_cast<int *>(smem + p.off_shift);         // shift per column
-    uint8_t *cwmag = smem + p.off_wmag;                             // log2 weight magnitude
+    uint8_t *wbias_smem = smem + p.off_wbias;
+    uint8_t *aconst_smem = smem + p.off_aconst;
+    int *cmult = reinterpret_cast<int *>(smem + p.off_mult);        // mult per resident column
+    int2 *cbs = reinterpret_cast<int2 *>(smem + p.off_bs);          // {bias, shift} per column
+    uint32_t *lut = reinterpret_cast<uint32_t *>(smem + p.off_lut); // [kLuts][256]
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + p.off_bars);
-    // barrier slots: full[stages], empty[stages], tfull[2], tempty[2], drain
+    // barrier slots: full[kMaxStages], empty[kMaxStages], tfull[kMaxBufs], tempty[kMaxBufs], drain
     const uint32_t bar_full = ptx::smem_u32(bars);
     const uint32_t bar_empty = bar_full + 8 * kMaxStages;
     const uint32_t bar_tfull = bar_empty + 8 * kMaxStages;
-    const uint32_t bar_tempty = bar_tfull + 16;
-    const uint32_t bar_drain = bar_tempty + 16;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + 2 * kMaxStages + 5);
-    volatile int *flags = reinterpret_cast<volatile int *>(bars + 2 * kMaxStages + 6);
+    const uint32_t bar_tempty = bar_tfull + 8 * kMaxBufs;
+    const uint32_t bar_drain = bar_tempty + 8 * kMaxBufs;
+    constexpr int kBarSlots = 2 * kMaxStages + 2 * kMaxBufs + 1;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + kBarSlots);
+    volatile int *flags = reinterpret_cast<volatile int *>(bars + kBarSlots + 1);
     // flags[0] abort, flags[1] shmin, flags[2] shmax, flags[3] bad constants, flags[4] slow path
 
     const int g = blockIdx.x % p.groups;
     const int worker = blockIdx.x / p.groups;
     const int nworkers = gridDim.x / p.groups;
     const int ncols_res = p.subs_per_cta * p.nt_pad;
+    const uint32_t cw = (uint32_t)p.cw;
+    const uint32_t stage_bytes = 128u * cw;
 
-    // ---- prologue: independent of the previous kernel's output ----------------
+    // ---- prologue: nothing here depends on the previous kernel's output -------------
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             ptx::mbar_init(bar_full + 8 * s, 1);
             ptx::mbar_init(bar_empty + 8 * s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < p.nbuf; ++b) {
             ptx::mbar_init(bar_tfull + 8 * b, 1);
-            ptx::mbar_init(bar_tempty + 8 * b, kEpiWarps);
+            ptx::mbar_init(bar_tempty + 8 * b, kEpiWarps / kEpiGroups);
         }
         ptx::mbar_init(bar_drain, 1);
         ptx::mbar_init_fence();
         flags[0] = 0; flags[1] = 31; flags[2] = 0; flags[3] = 0; flags[4] = 0;
         ptx::tma_prefetch_desc(&xmap);
+        if (p.store_2d) ptx::tma_prefetch_desc(&ymap);
     }
     __syncthreads();
     if (warp == 1) ptx::tmem_alloc(ptx::smem_u32((const void *)tmem_slot), (uint32_t)p.tmem_cols);
@@ -223,97 +257,169 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const Params p)
     {
         int mn = 31, mx = 0, bad = 0;
         for (int i = threadIdx.x; i < ncols_res; i += kThreads) {
-            int ls = i / p.nt_pad, c = i - ls * p.nt_pad;
-            int sub = g + ls * p.groups;
-            int nfold = sub * p.nt + c;
+            const int ls = i / p.nt_pad, c = i - ls * p.nt_pad;
+            const int nfold = (g + ls * p.groups) * p.nt + c;
+            int b = 0, mu = 0, sh = 0;
             if (c < p.nt && nfold < p.nf) {
-                int n = nfold % p.n0;
-                int b = p.bias[n], mu = p.mult[n], sh = p.shift[n];
-                if (!requant_ok(b, mu, sh)) bad = 1;
+                const int n = nfold % p.n0;
+                b = __ldg(p.bias + n); mu = __ldg(p.mult + n); sh = __ldg(p.shift + n);
+                if (!requant_ok(b, mu, sh)) { bad = 1; b = 0; mu = 0; sh = 0; }
                 mn = min(mn, sh); mx = max(mx, sh);
             }
+            cmult[i] = mu;
+            cbs[i] = make_int2(b, sh);
         }
         if (bad) flags[3] = 1;
-        atomicMin((int *)&flags[1], mn);
-        atomicMax((int *)&flags[2], mx);
+        if (mn <= mx) {
+            atomicMin((int *)&flags[1], mn);
+            atomicMax((int *)&flags[2], mx);
+        }
+        // code tables: byte of four 2-bit codes -> four int8 of magnitude 1, 4, 8, .., 64
+        for (int i = threadIdx.x; i < kLuts * 256; i += kThreads) {
+            const uint32_t t = (uint32_t)i >> 8, byte = (uint32_t)i & 255u;
+            const uint32_t mag = t == 0 ? 1u : (2u << t), neg = 256u - mag;
+            uint32_t word = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t code = (byte >> (2 * e)) & 3u;
+                const uint32_t val = code == 1u ? mag : (code == 3u ? neg : 0u);
+                word |= val << (8 * e);
+            }
+            lut[i] = word;
+        }
+        // the constant A block of the bias step: bytes 0,1 = 1, bytes 2..31 = 127
+        for (int i = threadIdx.x; i < 128 * 2; i += kThreads) {
+            const uint32_t r = (uint32_t)i >> 1, j = (uint32_t)i & 1u;
+            const uint4 val = j == 0 ? make_uint4(0x7F7F0101u, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu)
+                                     : make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+            *reinterpret_cast<uint4 *>(aconst_smem + swz_offset(r, j, 32u)) = val;
+        }
     }
     __syncthreads();
     const int shmax = flags[2];
     const bool bad_consts = flags[3] != 0;
     {
-        const bool span_ok = (p.act_min == 0 && p.act_max == 127) && (shmax - flags[1] <= 4);
+        const bool span_ok = (p.act_min == 0 && p.act_max == 127) && (shmax - flags[1] <= 4) &&
+                             shmax <= 24;
         int slow = span_ok ? 0 : 1;
-        for (int i = threadIdx.x; i < ncols_res; i += kThreads) {
-            int ls = i / p.nt_pad, c = i - ls * p.nt_pad;
-            int sub = g + ls * p.groups;
-            int nfold = sub * p.nt + c;
-            int b = 0, mu = 0, sh = 0;
-            if (c < p.nt && nfold < p.nf && !bad_consts) {
-                int n = nfold % p.n0;
-                b = p.bias[n]; mu = p.mult[n]; sh = p.shift[n];
+        if (span_ok)
+            for (int i = threadIdx.x; i < ncols_res; i += kThreads) {
+                const int ls = i / p.nt_pad, c = i - ls * p.nt_pad;
+                if (c >= p.nt || (g + ls * p.groups) * p.nt + c >= p.nf) continue;   // padding
+                const int2 bs = cbs[i];
+                const int lg = 2 + shmax - bs.y;
+                const long long ab = bs.x < 0 ? -(long long)bs.x : bs.x;
+                // |acc + bias| * 2^lg must stay below 2^31, the scaled bias within the digit range
+                if ((((long long)128 * p.k0 + ab) << lg) >= (1ll << 31) || (ab << lg) > kBiasMax)
+                    slow = 1;
             }
-            int lg = span_ok ? 2 + shmax - sh : 0;
-            // |acc + bias| * 2^lg must stay below 2^31
-            long long worst = ((long long)128 * p.k0 + (b < 0 ? -(long long)b : b)) << lg;
-            if (worst >= (1ll << 31)) slow = 1;
-            cwmag[i] = (uint8_t)lg;
-            csh[i] = sh;
-            cb[i] = make_int2(b, mu);      // bias is rescaled below once the path is known
-        }
         if (slow) flags[4] = 1;
     }
     __syncthreads();
     const bool fast = flags[4] == 0;
-    for (int i = threadIdx.x; i < ncols_res; i += kThreads) {
-        if (fast) cb[i].x = cb[i].x << cwmag[i];
-        else cwmag[i] = 0;
-    }
-    __syncthreads();
 
-    // expand the resident weights into the K-major swizzle-128B operand layout
+    // bias digits of the resident channels (fast path): row n of a 32-byte-swizzled block
+    if (fast)
+        for (int i = threadIdx.x; i < ncols_res; i += kThreads) {
+            const int ls = i / p.nt_pad, c = i - ls * p.nt_pad;
+            const int2 bs = cbs[i];
+            const int v = bs.x << (2 + shmax - bs.y);
+            int h = (v >= 0 ? v + 63 : v - 63) / 127;        // nearest multiple of 127
+            const int lo = v - 127 * h;                       // within [-63, 63]
+            uint32_t wd[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) wd[e] = 0;
+            wd[0] = (uint32_t)lo & 0xFFu;
+#pragma unroll
+            for (int d = 0; d < kBiasHiDigits; ++d) {
+                const int dig = h > 127 ? 127 : (h < -127 ? -127 : h);
+                h -= dig;
+                const int k = d + 2;
+                wd[k >> 2] |= ((uint32_t)dig & 0xFFu) << (8 * (k & 3));
+            }
+            uint8_t *blk = wbias_smem + (size_t)ls * p.nt_pad * 32;
+            *reinterpret_cast<uint4 *>(blk + swz_offset((uint32_t)c, 0u, 32u)) =
+                make_uint4(wd[0], wd[1], wd[2], wd[3]);
+            *reinterpret_cast<uint4 *>(blk + swz_offset((uint32_t)c, 1u, 32u)) =
+                make_uint4(wd[4], wd[5], wd[6], wd[7]);
+        }
+
+    // expand the resident weights into the K-major swizzled operand layout
     {
         const int rowb = (p.k0 + 3) >> 2;
-        const int pieces = p.subs_per_cta * p.kc * p.nt_pad * 8;
-        const bool quick = (p.fold == 1) && ((p.k0 & 15) == 0);
+        const bool quick = (p.k0 & 15) == 0;
+        const int cpr = p.cw >> 4;                        // 16-byte pieces per row
+        const int cpr_log2 = cpr == 8 ? 3 : (cpr == 4 ? 2 : 1);
+        const int per_blk = p.nt_pad * cpr;
+        const int nblk = p.subs_per_cta * p.kc;
         uint32_t invalid = 0;
-        for (int i = threadIdx.x; i < pieces; i += kThreads) {
-            int j = i & 7;
-            int n = (i >> 3) % p.nt_pad;
-            int blk = (i >> 3) / p.nt_pad;          // ls * kc + chunk
-            int ls = blk / p.kc, chunk = blk - ls * p.kc;
-            int kbase = chunk * 128 + j * 16;
-            if (chunk == p.kc - 1 && j * 16 >= p.ksteps_last * 32) continue;   // never read
-            int sub = g + ls * p.groups;
-            int nfold = sub * p.nt + n;
-            uint4 val = make_uint4(0, 0, 0, 0);
-            if (n < p.nt && nfold < p.nf && kbase < p.kf) {
-                uint32_t mag = 1u << cwmag[ls * p.nt_pad + n];
-                uint32_t negmag = 256u - mag;
-                if (quick) {
-                    uint32_t word = *reinterpret_cast<const uint32_t *>(
-                        p.w_packed + (size_t)nfold * rowb + (kbase >> 2));
-                    val.x = expand4(word & 0xFFu, mag, negmag, invalid);
-                    val.y = expand4((word >> 8) & 0xFFu, mag, negmag, invalid);
-                    val.z = expand4((word >> 16) & 0xFFu, mag, negmag, invalid);
-                    val.w = expand4(word >> 24, mag, negmag, invalid);
-                } else {
-                    int pn = nfold / p.n0, n_ch = nfold - pn * p.n0;
-                    uint32_t wd[4] = {0, 0, 0, 0};
-                    for (int e = 0; e < 16; ++e) {
-                        int kk = kbase + e;
-                        if (kk >= p.kf) break;
-                        int pk = kk / p.k0, k = kk - pk * p.k0;
-                        if (pk != pn) continue;
-                        int wv = weight_at(p.w_packed, rowb, n_ch, k);
-                        if (wv == -2) { invalid = 1; wv = 0; }
-                        uint32_t byte = wv == 0 ? 0u : (wv > 0 ? mag : negmag);
-                        wd[e >> 2] |= byte << (8 * (e & 3));
+        for (int blk = 0; blk < nblk; ++blk) {
+            const int ls = blk / p.kc, chunk = blk - ls * p.kc;
+            const int sub = g + ls * p.groups;
+            uint8_t *dst_blk = w_smem + (size_t)blk * p.nt_pad * cw;
+            const int jmax = (chunk == p.kc - 1) ? p.ksteps_last * 2 : cpr;   // pieces ever read
+            for (int base = 0; base < per_blk; base += 4 * kThreads) {
+                uint32_t word[4];
+                int tsel[4];
+                // loads first, so that they are in flight together
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int idx = base + u * kThreads + (int)threadIdx.x;
+                    word[u] = 0; tsel[u] = -1;
+                    if (idx >= per_blk) continue;
+                    const int n = idx >> cpr_log2, j = idx & (cpr - 1);
+                    if (j >= jmax) continue;
+                    tsel[u] = -2;                                  // write zeros
+                    const int nfold = sub * p.nt + n, kbase = chunk * p.cw + j * 16;
+                    if (n >= p.nt || nfold >= p.nf || kbase >= p.kf) continue;
+                    const int2 bs = cbs[ls * p.nt_pad + n];
+                    const int t = fast ? 1 + shmax - bs.y : 0;
+                    if (quick) {
+                        const int pn = nfold / p.n0, pk = kbase / p.k0;
+                        if (pn != pk) continue;                    // off the block diagonal
+                        const int n_ch = nfold - pn * p.n0, k = kbase - pk * p.k0;
+                        word[u] = __ldg(reinterpret_cast<const uint32_t *>(
+                            p.w_packed + (size_t)n_ch * rowb + (k >> 2)));
+                        tsel[u] = t;
+                    } else {
+                        tsel[u] = 16 + t;                          // element by element below
                     }
-                    val = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (tsel[u] == -1) continue;
+                    const int idx = base + u * kThreads + (int)threadIdx.x;
+                    const int n = idx >> cpr_log2, j = idx & (cpr - 1);
+                    uint4 val = make_uint4(0, 0, 0, 0);
+                    if (tsel[u] >= 16) {
+                        const int t = tsel[u] - 16;
+                        const uint32_t mag = t == 0 ? 1u : (2u << t), neg = 256u - mag;
+                        const int nfold = sub * p.nt + n, kbase = chunk * p.cw + j * 16;
+                        const int pn = nfold / p.n0, n_ch = nfold - pn * p.n0;
+                        uint32_t wd[4] = {0, 0, 0, 0};
+                        for (int e = 0; e < 16; ++e) {
+                            const int kk = kbase + e;
+                            if (kk >= p.kf) break;
+                            const int pk = kk / p.k0, k = kk - pk * p.k0;
+                            if (pk != pn) continue;
+                            int wv = weight_at(p.w_packed, rowb, n_ch, k);
+                            if (wv == -2) { invalid = 1; wv = 0; }
+                            const uint32_t byte = wv == 0 ? 0u : (wv > 0 ? mag : neg);
+                            wd[e >> 2] |= byte << (8 * (e & 3));
+                        }
+                        val = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                    } else if (tsel[u] >= 0) {
+                        const uint32_t w = word[u];
+                        invalid |= (w >> 1) & ~w & 0x55555555u;
+                        const uint32_t *tb = lut + tsel[u] * 256;
+                        val.x = tb[w & 0xFFu];
+                        val.y = tb[(w >> 8) & 0xFFu];
+                        val.z = tb[(w >> 16) & 0xFFu];
+                        val.w = tb[w >> 24];
+                    }
+                    *reinterpret_cast<uint4 *>(dst_blk + swz_offset((uint32_t)n, (uint32_t)j, cw)) = val;
                 }
             }
-            *reinterpret_cast<uint4 *>(w_smem + ((size_t)blk * p.nt_pad + n) * 128 +
-                                       ((j ^ (n & 7)) << 4)) = val;
         }
         if (invalid) raise_status(PROM_ERR_BAD_WEIGHT);
         if (bad_consts && threadIdx.x == 0) raise_status(PROM_ERR_BAD_REQUANT);
@@ -332,6 +438,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const Params p)
     // instruction descriptor: s8 x s8 -> s32, both K-major, M = 128, N = nt_pad
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.nt_pad >> 3) << 17) |
                            ((128u >> 4) << 24);
+    const int loads_per_tile = p.share_x ? 1 : p.subs_per_cta * p.kc;
 
     if (!bad_consts) {
         if (warp == 0) {
@@ -340,24 +447,23 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const Params p)
                 uint32_t it = 0;
                 bool ok = true;
                 for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers)
-                    for (int ls = 0; ls < p.subs_per_cta && ok; ++ls)
-                        for (int chunk = 0; chunk < p.kc; ++chunk, ++it) {
-                            uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                            if (!wait_bar(bar_empty + 8 * s, ph ^ 1u, flags)) { ok = false; break; }
-                            ptx::mbar_expect_tx(bar_full + 8 * s, p.tx_bytes);
-                            uint32_t dst = smem_base + s * kStageBytes;
-                            if (p.x3d)
-                                ptx::tma_load_3d(dst, &xmap, chunk * 128, 0, mt * p.box_r,
-                                                 bar_full + 8 * s);
-                            else
-                                ptx::tma_load_2d(dst, &xmap, chunk * 128, mt * p.tm,
-                                                 bar_full + 8 * s);
-                        }
+                    for (int l = 0; l < loads_per_tile; ++l, ++it) {
+                        const int chunk = p.share_x ? 0 : l % p.kc;
+                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                        if (!wait_bar(bar_empty + 8 * s, ph ^ 1u, flags)) { ok = false; break; }
+                        ptx::mbar_expect_tx(bar_full + 8 * s, p.tx_bytes);
+                        const uint32_t dst = smem_base + s * stage_bytes;
+                        if (p.x3d)
+                            ptx::tma_load_3d(dst, &xmap, chunk * p.cw, 0, mt * p.box_r,
+                                             bar_full + 8 * s);
+                        else
+                            ptx::tma_load_2d(dst, &xmap, chunk * p.cw, mt * p.tm, bar_full + 8 * s);
+                    }
                 if (!ok) {
                     // let the copies already issued land before the CTA goes away
-                    uint32_t first = it > (uint32_t)p.stages ? it - p.stages : 0;
+                    const uint32_t first = it > (uint32_t)p.stages ? it - p.stages : 0;
                     for (uint32_t j = first; j < it; ++j) {
-                        unsigned long long t0 = ptx::globaltimer();
+                        const unsigned long long t0 = ptx::globaltimer();
                         while (!ptx::mbar_try_wait(bar_full + 8 * (j % p.stages),
                                                    (j / p.stages) & 1u) &&
                                ptx::globaltimer() - t0 < kWaitLimitNs) {}
@@ -367,92 +473,107 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const Params p)
         } else if (warp == 1) {
             // ---- MMA issuer ---------------------------------------------------------
             if (lane == 0) {
-                uint32_t it = 0, tile_it = 0;
+                uint32_t it = 0, unit = 0;
                 bool ok = true;
                 const uint32_t w_addr = ptx::smem_u32(w_smem);
+                const uint32_t wb_addr = ptx::smem_u32(wbias_smem);
+                const uint64_t ac_desc = smem_desc(ptx::smem_u32(aconst_smem), 32u);
                 for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers)
-                    for (int ls = 0; ls < p.subs_per_cta && ok; ++ls, ++tile_it) {
-                        uint32_t b = tile_it % p.acc_bufs, tph = (tile_it / p.acc_bufs) & 1u;
+                    for (int ls = 0; ls < p.subs_per_cta && ok; ++ls, ++unit) {
+                        const uint32_t b = unit % p.nbuf, tph = (unit / p.nbuf) & 1u;
                         if (!wait_bar(bar_tempty + 8 * b, tph ^ 1u, flags)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
                         const uint32_t d_tmem = tmem_base + b * p.nt_pad;
-                        for (int chunk = 0; chunk < p.kc; ++chunk, ++it) {
-                            uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                            if (!wait_bar(bar_full + 8 * s, ph, flags)) { ok = false; break; }
-                            ptx::tc_fence_after_sync();
-                            const uint32_t a_addr = smem_base + s * kStageBytes;
+                        uint32_t acc = 0;
+                        for (int chunk = 0; chunk < p.kc; ++chunk) {
+                            const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
+                            if (!p.share_x || ls == 0) {
+                                if (!wait_bar(bar_full + 8 * s, ph, flags)) { ok = false; break; }
+                                ptx::tc_fence_after_sync();
+                            }
+                            const uint32_t a_addr = smem_base + s * stage_bytes;
                             const uint32_t b_addr =
-                                w_addr + (uint32_t)((ls * p.kc + chunk) * p.nt_pad) * 128u;
-                            const int nks = (chunk == p.kc - 1) ? p.ksteps_last : 4;
-                            for (int ks = 0; ks < nks; ++ks)
-                                ptx::mma_i8(d_tmem, smem_desc(a_addr + 32 * ks),
-                                            smem_desc(b_addr + 32 * ks), idesc,
-                                            (chunk | ks) != 0 ? 1u : 0u);
-                            ptx::mma_commit(bar_empty + 8 * s);
+                                w_addr + (uint32_t)((ls * p.kc + chunk) * p.nt_pad) * cw;
+                            const int nks = (chunk == p.kc - 1) ? p.ksteps_last : (p.cw >> 5);
+                            for (int ks = 0; ks < nks; ++ks) {
+                                ptx::mma_i8(d_tmem, smem_desc(a_addr + 32 * ks, cw),
+                                            smem_desc(b_addr + 32 * ks, cw), idesc, acc);
+                                acc = 1;
+                            }
+                            if (!p.share_x || ls == p.subs_per_cta - 1) {
+                                ptx::mma_commit(bar_empty + 8 * s);
+                                ++it;
+                            }
                         }
-                        if (ok) ptx::mma_commit(bar_tfull + 8 * b);
+                        if (!ok) break;
+                        if (fast)
+                            ptx::mma_i8(d_tmem, ac_desc,
+                                        smem_desc(wb_addr + (uint32_t)(ls * p.nt_pad) * 32u, 32u),
+                                        idesc, 1u);
+                        ptx::mma_commit(bar_tfull + 8 * b);
                     }
                 // every MMA has finished before tensor memory is released
                 ptx::mma_commit(bar_drain);
-                unsigned long long t0 = ptx::globaltimer();
-                while (!ptx::mbar_try_wait(bar_drain, 0) &&
-                       ptx::globaltimer() - t0 < kWaitLimitNs) {}
+                const unsigned long long t0 = ptx::globaltimer();
+                while (!ptx::mbar_try_wait(bar_drain, 0) && ptx::globaltimer() - t0 < kWaitLimitNs) {}
             }
         } else {
             // ---- epilogue ---------------------------------------------------------------
             const int q = warp & 3;                     // TMEM lane quarter of this warp
-            uint8_t *stage = smem + p.off_out + (size_t)(warp - 2) * 32 * p.out_pitch;
-            uint8_t *my_row = stage + lane * p.out_pitch;
-            uint32_t tile_it = 0;
+            const int grp = (warp - 2) >> 2;            // epilogue group: units grp, grp+2, ..
+            uint8_t *slab = smem + p.off_out + (size_t)(warp - 2) * 32 * p.nt;
+            uint8_t *my_row = slab + lane * p.nt;
+            const uint32_t slab_addr = ptx::smem_u32(slab);
+            uint32_t unit = 0;
             bool ok = true;
             for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers)
-                for (int ls = 0; ls < p.subs_per_cta && ok; ++ls, ++tile_it) {
-                    uint32_t b = tile_it % p.acc_bufs, tph = (tile_it / p.acc_bufs) & 1u;
+                for (int ls = 0; ls < p.subs_per_cta && ok; ++ls, ++unit) {
+                    if ((int)(unit & 1u) != grp) continue;
+                    const uint32_t b = unit % p.nbuf, tph = (unit / p.nbuf) & 1u;
                     if (!wait_bar(bar_tfull + 8 * b, tph, flags)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
+                    // the previous bulk store must have read the slab before it is rewritten
+                    ptx::bulk_wait_read0();
+                    __syncwarp();
                     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * p.nt_pad;
-                    const int2 *cbs = cb + ls * p.nt_pad;
-                    const int *cshs = csh + ls * p.nt_pad;
-                    if (fast) epi_subtile<true>(p, taddr, cbs, cshs, shmax, my_row);
-                    else epi_subtile<false>(p, taddr, cbs, cshs, shmax, my_row);
+                    const int *cms = cmult + ls * p.nt_pad;
+                    if (fast) epi_subtile<true>(p, taddr, cms, nullptr, shmax, my_row);
+                    else epi_subtile<false>(p, taddr, cms, cbs + ls * p.nt_pad, shmax, my_row);
                     ptx::tc_fence_before_sync();
+                    ptx::fence_proxy_async_smem();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
-
-                    // copy this warp's 32 staged rows out, coalesced
                     const long long row0 = (long long)mt * p.tm + q * 32;
-                    long long lim = p.m_rows - row0;
+                    const long long lim = p.m_rows - row0;
                     int rows_valid = p.tm - q * 32;
                     if (lim < rows_valid) rows_valid = (int)lim;
                     if (rows_valid > 32) rows_valid = 32;
-                    const int sub = g + ls * p.groups;
-                    if (rows_valid > 0) {
-                        if (!p.mode_b) {
-                            const int cpr = p.nt >> 4;
-                            const int total = rows_valid * cpr;
-                            int8_t *ybase = p.y + row0 * p.nf + (long long)sub * p.nt;
-                            for (int idx = lane; idx < total; idx += 32) {
-                                int r = (int)(((uint32_t)idx * p.inv_cpr) >> 20);
-                                int ch = idx - r * cpr;
-                                uint4 vv = *reinterpret_cast<const uint4 *>(stage + r * p.out_pitch +
-                                                                            ch * 16);
-                                *reinterpret_cast<uint4 *>(ybase + (long long)r * p.nf + ch * 16) = vv;
+                    if (!p.store_2d) {
+                        // one subtile spans the row: the slab is one contiguous range of Y
+                        if (lane == 0 && rows_valid > 0) {
+                            const uint32_t bytes = (uint32_t)(rows_valid * p.nf);
+                            const uint32_t whole = bytes & ~15u;      // bulk copies move 16-byte granules
+                            if (whole) {
+                                ptx::bulk_store(p.y + row0 * p.nf, slab_addr, whole);
+                                ptx::bulk_commit();
                             }
-                        } else {
-                            const int valid = rows_valid * p.nt;
-                            int8_t *ybase = p.y + row0 * p.nt;
-                            for (int off = lane * 16; off < valid; off += 512) {
-                                if (off + 16 <= valid)
-                                    *reinterpret_cast<uint4 *>(ybase + off) =
-                                        *reinterpret_cast<const uint4 *>(stage + off);
-                                else
-                                    *reinterpret_cast<uint2 *>(ybase + off) =
-                                        *reinterpret_cast<const uint2 *>(stage + off);
-                            }
+                            if (bytes & 15u)                          // odd last row of an 8-multiple width
+                                *reinterpret_cast<uint2 *>(p.y + row0 * p.nf + whole) =
+                                    *reinterpret_cast<const uint2 *>(slab + whole);
                         }
+                    } else if (rows_valid == 32) {
+                        if (lane == 0) {
+                            ptx::tma_store_2d(&ymap, (g + ls * p.groups) * p.nt, (int)row0, slab_addr);
+                            ptx::bulk_commit();
+                        }
+                    } else if (lane < rows_valid) {
+                        // a partial slab (short tile or end of the matrix) leaves row by row
+                        ptx::bulk_store(p.y + (row0 + lane) * p.nf + (g + ls * p.groups) * p.nt,
+                                        slab_addr + (uint32_t)(lane * p.nt), (uint32_t)p.nt);
+                        ptx::bulk_commit();
                     }
-                    __syncwarp();
                 }
+            ptx::bulk_wait_all();
         }
     }
 
