@@ -187,9 +187,10 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     } else {
         tmem_cols = 512;
     }
-    int nbuf = tmem_cols / nt_pad;
-    if (nbuf > tc::kMaxBufs) nbuf = tc::kMaxBufs;
-    if (nbuf < 2) return false;
+    // accumulator ring: an even length, so that each of the two epilogue groups keeps to its own
+    // accumulators
+    if (tmem_cols / nt_pad < 2) return false;
+    const int nbuf = tmem_cols / nt_pad >= 4 ? 4 : 2;
 
     const int ncols = subs * nt_pad;
     const size_t stage_bytes = (size_t)128 * cw;

@@ -37,7 +37,7 @@ namespace prom { namespace tc {
 constexpr int kThreads = 320;
 constexpr int kEpiWarps = 8;
 constexpr int kEpiGroups = 2;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned long long kWaitLimitNs = 100000000ull;   // 0.1 s: far beyond any legitimate wait
 constexpr int kMaxStages = 8;
 constexpr int kMaxBufs = 4;
 constexpr int kLuts = 6;                 // magnitude 1, then 4, 8, 16, 32, 64
@@ -71,15 +71,19 @@ struct Params {
     int pdl;            // launched with programmatic dependent launch
 };
 
+// Bounded wait on an mbarrier phase.  The clock is read only every 1024 polls (a
+// poll that finds the phase incomplete already suspends the thread for a while), so
+// that a wait which ends within microseconds never pays for a timer read.
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    unsigned long long t0 = ptx::globaltimer();
+    unsigned long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 0) {
+        if ((i & 1023u) == 0) {
             if (*abort_flag) return false;
-            if (ptx::globaltimer() - t0 > kWaitLimitNs) {
+            const unsigned long long now = ptx::globaltimer();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) {
                 *abort_flag = 1;
                 raise_status(PROM_ERR_TIMEOUT);
                 return false;
@@ -129,8 +133,8 @@ __device__ __forceinline__ void put_row(uint8_t *dst, const uint32_t (&out)[NC /
     }
 }
 
-// NC accumulator columns of this thread's row: one mad.hi and one shift per
-// value, saturating pack, halve.
+// NC accumulator columns of this thread's row: the high word of a 64-bit
+// multiply-add (rounding term in the addend), one shift, saturating pack, halve.
 template <int NC>
 __device__ __forceinline__ void epi_fast(uint32_t taddr, const int *__restrict__ cm, int shmax,
                                          uint8_t *dst, bool wide)
@@ -139,14 +143,15 @@ __device__ __forceinline__ void epi_fast(uint32_t taddr, const int *__restrict__
     tmem_ld<NC>(taddr, v);
     ptx::tmem_wait_ld();
     uint32_t out[NC / 4];
-    const int r = 1 << shmax;
+    const long long r64 = 1ll << (32 + shmax);   // rounding term, in the addend of the 64-bit product
+    const int sh = 32 + shmax;
 #pragma unroll
     for (int c = 0; c < NC; c += 4) {
         const int4 mu = *reinterpret_cast<const int4 *>(cm + c);
-        const int q0 = ptx::mad_hi((int)v[c], mu.x, r) >> shmax;
-        const int q1 = ptx::mad_hi((int)v[c + 1], mu.y, r) >> shmax;
-        const int q2 = ptx::mad_hi((int)v[c + 2], mu.z, r) >> shmax;
-        const int q3 = ptx::mad_hi((int)v[c + 3], mu.w, r) >> shmax;
+        const int q0 = (int)(((long long)(int)v[c] * mu.x + r64) >> sh);
+        const int q1 = (int)(((long long)(int)v[c + 1] * mu.y + r64) >> sh);
+        const int q2 = (int)(((long long)(int)v[c + 2] * mu.z + r64) >> sh);
+        const int q3 = (int)(((long long)(int)v[c + 3] * mu.w + r64) >> sh);
         uint32_t w = ptx::pack_sat_u8(q3, q2, 0u);
         w = ptx::pack_sat_u8(q1, q0, w);
         out[c / 4] = (w >> 1) & 0x7F7F7F7Fu;
@@ -520,7 +525,10 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         } else {
             // ---- epilogue ---------------------------------------------------------------
             const int q = warp & 3;                     // TMEM lane quarter of this warp
-            const int grp = (warp - 2) >> 2;            // epilogue group: units grp, grp+2, ..
+            // Unit u goes to group u % 2 and accumulator u % nbuf; nbuf is even, so a group meets
+            // each of its accumulators in cyclic order and never waits on a barrier that is more
+            // than one phase away.
+            const int grp = (warp - 2) >> 2;
             uint8_t *slab = smem + p.off_out + (size_t)(warp - 2) * 32 * p.nt;
             uint8_t *my_row = slab + lane * p.nt;
             const uint32_t slab_addr = ptx::smem_u32(slab);

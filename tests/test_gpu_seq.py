@@ -107,3 +107,51 @@ def test_config2_full_size_sampled_rows(oracle):
             ref = y.clone()
         else:
             assert torch.equal(y, ref)
+
+
+def test_every_layer_shape_many_tiles_per_cta(oracle):
+    """Each MobileNetV2 layer shape at a row count that gives every CTA several
+    tiles, so that the rings of activation stages and accumulators wrap many
+    times: the tensor-core variant against the one-thread-per-output kernel on
+    the whole tensor, and against the oracle on sampled rows."""
+    table = synth.mobilenetv2_pointwise_layers()
+    seen = set()
+    m = 128 * 148 * 4 + 78
+    rows = np.unique(np.concatenate([np.arange(0, 300), np.arange(m - 300, m),
+                                     np.random.default_rng(1).integers(0, m, 1500)]))
+    for i, l in enumerate(table):
+        if (l.cin, l.cout) in seen:
+            continue
+        seen.add((l.cin, l.cout))
+        x = synth.act_post_relu6(200 + i, (m, l.cin), device="cuda")
+        lay = synth.make_layer(200 + i, l.cin, l.cout, 0.5)
+        wp = binding.pack_ternary(lay["w"].cuda())
+        rq = binding.make_requant(lay["bias"].cuda(), lay["mult"].cuda(), lay["shift"].cuda())
+        y_tc = torch.full((m, l.cout), -3, dtype=torch.int8, device="cuda")
+        y_nv = torch.full((m, l.cout), -4, dtype=torch.int8, device="cuda")
+        binding.pw_conv_i8(x, wp, l.cout, rq, y=y_tc, variant="tc")
+        binding.pw_conv_i8(x, wp, l.cout, rq, y=y_nv, variant="naive")
+        torch.cuda.synchronize()
+        assert binding.last_device_status() == binding.PROM_OK, l
+        assert torch.equal(y_tc, y_nv), l
+        idx = torch.from_numpy(rows).cuda()
+        want = oracle_y(oracle, x[idx].cpu(), lay)
+        assert first_mismatch(y_tc[idx].cpu().numpy(), want) is None, l
+
+
+def test_config3_full_size_sequence(oracle):
+    """The benchmark's own launch: all 34 layers at batch 128.  The library's
+    choice of variants against the plain kernel on the whole output, and the
+    oracle on the first two images (images are independent)."""
+    table = synth.mobilenetv2_pointwise_layers()
+    host, seq = build_sequence(synth.BASE_SEED + 3, table)
+    x0 = synth.act_post_relu6(synth.BASE_SEED + 3, (128, 112, 112, 32), device="cuda")
+    ws = torch.empty((seq.workspace_bytes(128, 112, 112),), dtype=torch.uint8, device="cuda")
+    y_auto = binding.pw_layer_seq(seq, x0, ws, variant="auto").clone()
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == binding.PROM_OK
+    y_naive = binding.pw_layer_seq(seq, x0, ws, variant="naive")
+    torch.cuda.synchronize()
+    assert torch.equal(y_auto, y_naive)
+    want = oracle.layer_seq(host, x0[:2].cpu().numpy())
+    assert np.array_equal(y_auto[:2].cpu().numpy(), want)
