@@ -74,11 +74,13 @@ struct Params {
 // Bounded wait on an mbarrier phase.  The clock is read only every 1024 polls (a
 // poll that finds the phase incomplete already suspends the thread for a while), so
 // that a wait which ends within microseconds never pays for a timer read.
+template <bool BACKOFF = false>
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
     unsigned long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
+        if constexpr (BACKOFF) __nanosleep(20);      // whole warps wait here: poll gently
         if ((i & 1023u) == 0) {
             if (*abort_flag) return false;
             const unsigned long long now = ptx::globaltimer();
@@ -446,28 +448,37 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     const int loads_per_tile = p.share_x ? 1 : p.subs_per_cta * p.kc;
 
     if (!bad_consts) {
+        // The two single-thread roles below run beside many busy epilogue warps, so every
+        // instruction on their per-unit path costs tens of cycles: ring positions, phases and
+        // descriptors are advanced by additions, never recomputed with divisions.
         if (warp == 0) {
             // ---- TMA producer ----------------------------------------------------
             if (lane == 0) {
-                uint32_t it = 0;
+                uint32_t s = 0, ph = 0, issued = 0;
+                uint32_t dst = smem_base, bfull = bar_full, bempty = bar_empty;
+                const int cx_end = p.share_x ? p.cw : p.kc * p.cw;
                 bool ok = true;
-                for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers)
-                    for (int l = 0; l < loads_per_tile; ++l, ++it) {
-                        const int chunk = p.share_x ? 0 : l % p.kc;
-                        const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
-                        if (!wait_bar(bar_empty + 8 * s, ph ^ 1u, flags)) { ok = false; break; }
-                        ptx::mbar_expect_tx(bar_full + 8 * s, p.tx_bytes);
-                        const uint32_t dst = smem_base + s * stage_bytes;
-                        if (p.x3d)
-                            ptx::tma_load_3d(dst, &xmap, chunk * p.cw, 0, mt * p.box_r,
-                                             bar_full + 8 * s);
-                        else
-                            ptx::tma_load_2d(dst, &xmap, chunk * p.cw, mt * p.tm, bar_full + 8 * s);
+                for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers) {
+                    const int c_row = p.x3d ? mt * p.box_r : mt * p.tm;
+                    int cx = 0;
+                    for (int l = 0; l < loads_per_tile; ++l) {
+                        if (!wait_bar(bempty, ph ^ 1u, flags)) { ok = false; break; }
+                        ptx::mbar_expect_tx(bfull, p.tx_bytes);
+                        if (p.x3d) ptx::tma_load_3d(dst, &xmap, cx, 0, c_row, bfull);
+                        else ptx::tma_load_2d(dst, &xmap, cx, c_row, bfull);
+                        ++issued;
+                        cx += p.cw;
+                        if (cx == cx_end) cx = 0;
+                        ++s; dst += stage_bytes; bfull += 8; bempty += 8;
+                        if (s == (uint32_t)p.stages) {
+                            s = 0; ph ^= 1u; dst = smem_base; bfull = bar_full; bempty = bar_empty;
+                        }
                     }
+                }
                 if (!ok) {
                     // let the copies already issued land before the CTA goes away
-                    const uint32_t first = it > (uint32_t)p.stages ? it - p.stages : 0;
-                    for (uint32_t j = first; j < it; ++j) {
+                    const uint32_t first = issued > (uint32_t)p.stages ? issued - p.stages : 0;
+                    for (uint32_t j = first; j < issued; ++j) {
                         const unsigned long long t0 = ptx::globaltimer();
                         while (!ptx::mbar_try_wait(bar_full + 8 * (j % p.stages),
                                                    (j / p.stages) & 1u) &&
@@ -478,45 +489,52 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         } else if (warp == 1) {
             // ---- MMA issuer ---------------------------------------------------------
             if (lane == 0) {
-                uint32_t it = 0, unit = 0;
                 bool ok = true;
-                const uint32_t w_addr = ptx::smem_u32(w_smem);
-                const uint32_t wb_addr = ptx::smem_u32(wbias_smem);
-                const uint64_t ac_desc = smem_desc(ptx::smem_u32(aconst_smem), 32u);
-                for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers)
-                    for (int ls = 0; ls < p.subs_per_cta && ok; ++ls, ++unit) {
-                        const uint32_t b = unit % p.nbuf, tph = (unit / p.nbuf) & 1u;
-                        if (!wait_bar(bar_tempty + 8 * b, tph ^ 1u, flags)) { ok = false; break; }
+                // descriptors: constant high word, low word = (address >> 4) | LBO field
+                const uint64_t d_cw = smem_desc(0u, cw), d_32 = smem_desc(0u, 32u);
+                const uint32_t a_lo0 = smem_base >> 4, a_step = stage_bytes >> 4;
+                const uint32_t b_lo0 = ptx::smem_u32(w_smem) >> 4, b_step = ((uint32_t)p.nt_pad * cw) >> 4;
+                const uint32_t wb_lo0 = ptx::smem_u32(wbias_smem) >> 4, wb_step = ((uint32_t)p.nt_pad * 32u) >> 4;
+                const uint64_t ac_desc = d_32 | (uint64_t)(ptx::smem_u32(aconst_smem) >> 4);
+                const int ks_full = p.cw >> 5;
+                uint32_t s = 0, ph = 0, a_lo = a_lo0, bfull = bar_full, bempty = bar_empty;
+                uint32_t b = 0, tph = 0, d_tmem = tmem_base, btfull = bar_tfull, btempty = bar_tempty;
+                for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers) {
+                    uint32_t b_lo = b_lo0, wb_lo = wb_lo0;
+                    for (int ls = 0; ls < p.subs_per_cta && ok; ++ls) {
+                        if (!wait_bar(btempty, tph ^ 1u, flags)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
-                        const uint32_t d_tmem = tmem_base + b * p.nt_pad;
                         uint32_t acc = 0;
                         for (int chunk = 0; chunk < p.kc; ++chunk) {
-                            const uint32_t s = it % p.stages, ph = (it / p.stages) & 1u;
                             if (!p.share_x || ls == 0) {
-                                if (!wait_bar(bar_full + 8 * s, ph, flags)) { ok = false; break; }
+                                if (!wait_bar(bfull, ph, flags)) { ok = false; break; }
                                 ptx::tc_fence_after_sync();
                             }
-                            const uint32_t a_addr = smem_base + s * stage_bytes;
-                            const uint32_t b_addr =
-                                w_addr + (uint32_t)((ls * p.kc + chunk) * p.nt_pad) * cw;
-                            const int nks = (chunk == p.kc - 1) ? p.ksteps_last : (p.cw >> 5);
+                            const int nks = (chunk == p.kc - 1) ? p.ksteps_last : ks_full;
                             for (int ks = 0; ks < nks; ++ks) {
-                                ptx::mma_i8(d_tmem, smem_desc(a_addr + 32 * ks, cw),
-                                            smem_desc(b_addr + 32 * ks, cw), idesc, acc);
+                                ptx::mma_i8(d_tmem, d_cw | (uint64_t)(a_lo + 2 * ks),
+                                            d_cw | (uint64_t)(b_lo + 2 * ks), idesc, acc);
                                 acc = 1;
                             }
+                            b_lo += b_step;
                             if (!p.share_x || ls == p.subs_per_cta - 1) {
-                                ptx::mma_commit(bar_empty + 8 * s);
-                                ++it;
+                                ptx::mma_commit(bempty);
+                                ++s; a_lo += a_step; bfull += 8; bempty += 8;
+                                if (s == (uint32_t)p.stages) {
+                                    s = 0; ph ^= 1u; a_lo = a_lo0; bfull = bar_full; bempty = bar_empty;
+                                }
                             }
                         }
                         if (!ok) break;
-                        if (fast)
-                            ptx::mma_i8(d_tmem, ac_desc,
-                                        smem_desc(wb_addr + (uint32_t)(ls * p.nt_pad) * 32u, 32u),
-                                        idesc, 1u);
-                        ptx::mma_commit(bar_tfull + 8 * b);
+                        if (fast) ptx::mma_i8(d_tmem, ac_desc, d_32 | (uint64_t)wb_lo, idesc, 1u);
+                        wb_lo += wb_step;
+                        ptx::mma_commit(btfull);
+                        ++b; d_tmem += p.nt_pad; btfull += 8; btempty += 8;
+                        if (b == (uint32_t)p.nbuf) {
+                            b = 0; tph ^= 1u; d_tmem = tmem_base; btfull = bar_tfull; btempty = bar_tempty;
+                        }
                     }
+                }
                 // every MMA has finished before tensor memory is released
                 ptx::mma_commit(bar_drain);
                 const unsigned long long t0 = ptx::globaltimer();
@@ -532,55 +550,60 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             uint8_t *slab = smem + p.off_out + (size_t)(warp - 2) * 32 * p.nt;
             uint8_t *my_row = slab + lane * p.nt;
             const uint32_t slab_addr = ptx::smem_u32(slab);
-            uint32_t unit = 0;
+            const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
             bool ok = true;
-            for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers)
-                for (int ls = 0; ls < p.subs_per_cta && ok; ++ls, ++unit) {
-                    if ((int)(unit & 1u) != grp) continue;
-                    const uint32_t b = unit % p.nbuf, tph = (unit / p.nbuf) & 1u;
-                    if (!wait_bar(bar_tfull + 8 * b, tph, flags)) { ok = false; break; }
-                    ptx::tc_fence_after_sync();
-                    // the previous bulk store must have read the slab before it is rewritten
-                    ptx::bulk_wait_read0();
-                    __syncwarp();
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * p.nt_pad;
-                    const int *cms = cmult + ls * p.nt_pad;
-                    if (fast) epi_subtile<true>(p, taddr, cms, nullptr, shmax, my_row);
-                    else epi_subtile<false>(p, taddr, cms, cbs + ls * p.nt_pad, shmax, my_row);
-                    ptx::tc_fence_before_sync();
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
-                    const long long row0 = (long long)mt * p.tm + q * 32;
-                    const long long lim = p.m_rows - row0;
-                    int rows_valid = p.tm - q * 32;
-                    if (lim < rows_valid) rows_valid = (int)lim;
-                    if (rows_valid > 32) rows_valid = 32;
-                    if (!p.store_2d) {
-                        // one subtile spans the row: the slab is one contiguous range of Y
-                        if (lane == 0 && rows_valid > 0) {
-                            const uint32_t bytes = (uint32_t)(rows_valid * p.nf);
-                            const uint32_t whole = bytes & ~15u;      // bulk copies move 16-byte granules
-                            if (whole) {
-                                ptx::bulk_store(p.y + row0 * p.nf, slab_addr, whole);
-                                ptx::bulk_commit();
-                            }
-                            if (bytes & 15u)                          // odd last row of an 8-multiple width
-                                *reinterpret_cast<uint2 *>(p.y + row0 * p.nf + whole) =
-                                    *reinterpret_cast<const uint2 *>(slab + whole);
-                        }
-                    } else if (rows_valid == 32) {
-                        if (lane == 0) {
-                            ptx::tma_store_2d(&ymap, (g + ls * p.groups) * p.nt, (int)row0, slab_addr);
+            int mt = worker, ls = grp;                  // this group's first unit
+            while (ls >= p.subs_per_cta) { ls -= p.subs_per_cta; mt += nworkers; }
+            uint32_t b = (uint32_t)grp, tph = 0;
+            while (mt < p.n_mtiles && ok) {
+                if (!wait_bar<true>(bar_tfull + 8 * b, tph, flags)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
+                // the previous bulk store must have read the slab before it is rewritten
+                ptx::bulk_wait_read0();
+                __syncwarp();
+                const uint32_t taddr = t_lane + b * p.nt_pad;
+                const int *cms = cmult + ls * p.nt_pad;
+                if (fast) epi_subtile<true>(p, taddr, cms, nullptr, shmax, my_row);
+                else epi_subtile<false>(p, taddr, cms, cbs + ls * p.nt_pad, shmax, my_row);
+                ptx::tc_fence_before_sync();
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
+                const long long row0 = (long long)mt * p.tm + q * 32;
+                const long long lim = p.m_rows - row0;
+                int rows_valid = p.tm - q * 32;
+                if (lim < rows_valid) rows_valid = (int)lim;
+                if (rows_valid > 32) rows_valid = 32;
+                if (!p.store_2d) {
+                    // one subtile spans the row: the slab is one contiguous range of Y
+                    if (lane == 0 && rows_valid > 0) {
+                        const uint32_t bytes = (uint32_t)(rows_valid * p.nf);
+                        const uint32_t whole = bytes & ~15u;      // bulk copies move 16-byte granules
+                        if (whole) {
+                            ptx::bulk_store(p.y + row0 * p.nf, slab_addr, whole);
                             ptx::bulk_commit();
                         }
-                    } else if (lane < rows_valid) {
-                        // a partial slab (short tile or end of the matrix) leaves row by row
-                        ptx::bulk_store(p.y + (row0 + lane) * p.nf + (g + ls * p.groups) * p.nt,
-                                        slab_addr + (uint32_t)(lane * p.nt), (uint32_t)p.nt);
+                        if (bytes & 15u)                          // odd last row of an 8-multiple width
+                            *reinterpret_cast<uint2 *>(p.y + row0 * p.nf + whole) =
+                                *reinterpret_cast<const uint2 *>(slab + whole);
+                    }
+                } else if (rows_valid == 32) {
+                    if (lane == 0) {
+                        ptx::tma_store_2d(&ymap, (g + ls * p.groups) * p.nt, (int)row0, slab_addr);
                         ptx::bulk_commit();
                     }
+                } else if (lane < rows_valid) {
+                    // a partial slab (short tile or end of the matrix) leaves row by row
+                    ptx::bulk_store(p.y + (row0 + lane) * p.nf + (g + ls * p.groups) * p.nt,
+                                    slab_addr + (uint32_t)(lane * p.nt), (uint32_t)p.nt);
+                    ptx::bulk_commit();
                 }
+                // this group's next unit: two further on
+                ls += kEpiGroups;
+                while (ls >= p.subs_per_cta) { ls -= p.subs_per_cta; mt += nworkers; }
+                b += kEpiGroups;
+                if (b >= (uint32_t)p.nbuf) { b -= p.nbuf; tph ^= 1u; }
+            }
             ptx::bulk_wait_all();
         }
     }
