@@ -208,6 +208,12 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     if (stages > cap) stages = cap;
     if (stages > tc::kMaxStages) stages = tc::kMaxStages;
     if (stages < 2) return false;
+    // the packed weights of the CTA are copied into the activation stages before these are used
+    {
+        const size_t rowb = (size_t)(cin + 3) / 4;
+        const size_t packed = fold > 1 ? (size_t)cout * rowb : (size_t)subs * nt * rowb;
+        if (packed > (size_t)stages * stage_bytes) return false;
+    }
 
     p.m_rows = rows; p.k0 = cin; p.n0 = cout; p.fold = fold; p.kf = kf; p.nf = nf;
     p.tm = tm; p.n_mtiles = (int)n_mtiles; p.nt = nt; p.nt_pad = nt_pad;

@@ -95,6 +95,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *m, 
 }
 
 
+// Plain byte range global -> shared, completion counted on an mbarrier; both addresses
+// 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *gsrc, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(gsrc), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 // ---- bulk (TMA) stores: shared -> global, tracked in per-thread bulk groups -----------
 // Plain byte range; both addresses 16-byte aligned, size a multiple of 16.
 __device__ __forceinline__ void bulk_store(void *gdst, uint32_t src, uint32_t bytes)

@@ -44,6 +44,7 @@ constexpr int kLuts = 6;                 // magnitude 1, then 4, 8, 16, 32, 64
 constexpr int kAConstBytes = 128 * 32;
 constexpr int kBiasHiDigits = 30;        // A-const row: 1, 1, then 30 x 127
 constexpr int kBiasMax = 127 * 127 * kBiasHiDigits;
+constexpr int kNoColumn = -1000;        // marks a padding column (no int8 shift has this value)
 
 struct Params {
     long long m_rows;   // rows of the folded problem
@@ -229,7 +230,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     const uint32_t bar_tfull = bar_empty + 8 * kMaxStages;
     const uint32_t bar_tempty = bar_tfull + 8 * kMaxBufs;
     const uint32_t bar_drain = bar_tempty + 8 * kMaxBufs;
-    constexpr int kBarSlots = 2 * kMaxStages + 2 * kMaxBufs + 1;
+    const uint32_t bar_wload = bar_drain + 8;
+    constexpr int kBarSlots = 2 * kMaxStages + 2 * kMaxBufs + 2;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + kBarSlots);
     volatile int *flags = reinterpret_cast<volatile int *>(bars + kBarSlots + 1);
     // flags[0] abort, flags[1] shmin, flags[2] shmax, flags[3] bad constants, flags[4] slow path
@@ -242,6 +244,11 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     const uint32_t stage_bytes = 128u * cw;
 
     // ---- prologue: nothing here depends on the previous kernel's output -------------
+    // Thread 0 sets up the barriers and starts the bulk copy of this CTA's packed (2-bit)
+    // weights into the not yet used activation stages; meanwhile every thread requests the
+    // constants of its channels and builds the code tables.  Three block-wide syncs in all.
+    const int rowb = (p.k0 + 3) >> 2;
+    const uint8_t *wq = smem;                    // packed weights: rows of rowb bytes
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             ptx::mbar_init(bar_full + 8 * s, 1);
@@ -252,78 +259,109 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             ptx::mbar_init(bar_tempty + 8 * b, kEpiWarps / kEpiGroups);
         }
         ptx::mbar_init(bar_drain, 1);
+        ptx::mbar_init(bar_wload, 1);
         ptx::mbar_init_fence();
         flags[0] = 0; flags[1] = 31; flags[2] = 0; flags[3] = 0; flags[4] = 0;
+        if (p.fold > 1) {
+            // small layer: the whole packed matrix, indexed by channel
+            const uint32_t bytes = (uint32_t)(p.n0 * rowb);
+            ptx::mbar_expect_tx(bar_wload, bytes);
+            ptx::bulk_load(smem_base, p.w_packed, bytes, bar_wload);
+        } else {
+            // the rows of each resident subtile, subtile after subtile
+            const uint32_t bytes = (uint32_t)(p.nt * rowb);
+            ptx::mbar_expect_tx(bar_wload, bytes * (uint32_t)p.subs_per_cta);
+            for (int ls = 0; ls < p.subs_per_cta; ++ls)
+                ptx::bulk_load(smem_base + (uint32_t)ls * bytes,
+                               p.w_packed + (size_t)(g + ls * p.groups) * bytes, bytes, bar_wload);
+        }
         ptx::tma_prefetch_desc(&xmap);
         if (p.store_2d) ptx::tma_prefetch_desc(&ymap);
     }
-    __syncthreads();
     if (warp == 1) ptx::tmem_alloc(ptx::smem_u32((const void *)tmem_slot), (uint32_t)p.tmem_cols);
 
-    // constants of the resident channels: range check, shift span
-    {
-        int mn = 31, mx = 0, bad = 0;
-        for (int i = threadIdx.x; i < ncols_res; i += kThreads) {
+    // constants of up to kConstPerThread resident channels per thread, requested early
+    constexpr int kConstPerThread = 4;
+    int cb_[kConstPerThread], cm_[kConstPerThread], cs_[kConstPerThread];
+#pragma unroll
+    for (int u = 0; u < kConstPerThread; ++u) {
+        const int i = u * kThreads + (int)threadIdx.x;
+        cb_[u] = 0; cm_[u] = 0; cs_[u] = kNoColumn;         // padding column, or none
+        if (i < ncols_res) {
             const int ls = i / p.nt_pad, c = i - ls * p.nt_pad;
             const int nfold = (g + ls * p.groups) * p.nt + c;
-            int b = 0, mu = 0, sh = 0;
             if (c < p.nt && nfold < p.nf) {
                 const int n = nfold % p.n0;
-                b = __ldg(p.bias + n); mu = __ldg(p.mult + n); sh = __ldg(p.shift + n);
+                cb_[u] = __ldg(p.bias + n); cm_[u] = __ldg(p.mult + n); cs_[u] = __ldg(p.shift + n);
+            }
+        }
+    }
+    // code tables: byte of four 2-bit codes -> four int8 of magnitude 1, 4, 8, .., 64
+    for (int i = threadIdx.x; i < kLuts * 256; i += kThreads) {
+        const uint32_t t = (uint32_t)i >> 8, byte = (uint32_t)i & 255u;
+        const uint32_t mag = t == 0 ? 1u : (2u << t), neg = 256u - mag;
+        uint32_t w4 = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t code = (byte >> (2 * e)) & 3u;
+            const uint32_t val = code == 1u ? mag : (code == 3u ? neg : 0u);
+            w4 |= val << (8 * e);
+        }
+        lut[i] = w4;
+    }
+    // the constant A block of the bias step: bytes 0,1 = 1, bytes 2..31 = 127
+    for (int i = threadIdx.x; i < 128 * 2; i += kThreads) {
+        const uint32_t r = (uint32_t)i >> 1, j = (uint32_t)i & 1u;
+        const uint4 val = j == 0 ? make_uint4(0x7F7F0101u, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu)
+                                 : make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+        *reinterpret_cast<uint4 *>(aconst_smem + swz_offset(r, j, 32u)) = val;
+    }
+    __syncthreads();                                        // barriers and flags are set up
+
+    // range check, shift span, and whether every channel can take the fast epilogue: with
+    // the largest weight magnitude (2^6) |acc + bias| * 2^6 must stay below 2^31 and the
+    // scaled bias within the digit range
+    {
+        int mn = 31, mx = 0, bad = 0, slow = 0;
+        auto take = [&](int i, int b, int mu, int sh) {
+            if (sh != kNoColumn) {
                 if (!requant_ok(b, mu, sh)) { bad = 1; b = 0; mu = 0; sh = 0; }
                 mn = min(mn, sh); mx = max(mx, sh);
+                const long long ab = b < 0 ? -(long long)b : b;
+                if ((((long long)128 * p.k0 + ab) << 6) >= (1ll << 31) || (ab << 6) > kBiasMax) slow = 1;
+            } else {
+                sh = 0;
             }
             cmult[i] = mu;
             cbs[i] = make_int2(b, sh);
+        };
+#pragma unroll
+        for (int u = 0; u < kConstPerThread; ++u) {
+            const int i = u * kThreads + (int)threadIdx.x;
+            if (i < ncols_res) take(i, cb_[u], cm_[u], cs_[u]);
+        }
+        for (int i = kConstPerThread * kThreads + (int)threadIdx.x; i < ncols_res; i += kThreads) {
+            const int ls = i / p.nt_pad, c = i - ls * p.nt_pad;
+            const int nfold = (g + ls * p.groups) * p.nt + c;
+            int b = 0, mu = 0, sh = kNoColumn;
+            if (c < p.nt && nfold < p.nf) {
+                const int n = nfold % p.n0;
+                b = __ldg(p.bias + n); mu = __ldg(p.mult + n); sh = __ldg(p.shift + n);
+            }
+            take(i, b, mu, sh);
         }
         if (bad) flags[3] = 1;
+        if (slow) flags[4] = 1;
         if (mn <= mx) {
             atomicMin((int *)&flags[1], mn);
             atomicMax((int *)&flags[2], mx);
-        }
-        // code tables: byte of four 2-bit codes -> four int8 of magnitude 1, 4, 8, .., 64
-        for (int i = threadIdx.x; i < kLuts * 256; i += kThreads) {
-            const uint32_t t = (uint32_t)i >> 8, byte = (uint32_t)i & 255u;
-            const uint32_t mag = t == 0 ? 1u : (2u << t), neg = 256u - mag;
-            uint32_t word = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const uint32_t code = (byte >> (2 * e)) & 3u;
-                const uint32_t val = code == 1u ? mag : (code == 3u ? neg : 0u);
-                word |= val << (8 * e);
-            }
-            lut[i] = word;
-        }
-        // the constant A block of the bias step: bytes 0,1 = 1, bytes 2..31 = 127
-        for (int i = threadIdx.x; i < 128 * 2; i += kThreads) {
-            const uint32_t r = (uint32_t)i >> 1, j = (uint32_t)i & 1u;
-            const uint4 val = j == 0 ? make_uint4(0x7F7F0101u, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu)
-                                     : make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
-            *reinterpret_cast<uint4 *>(aconst_smem + swz_offset(r, j, 32u)) = val;
         }
     }
     __syncthreads();
     const int shmax = flags[2];
     const bool bad_consts = flags[3] != 0;
-    {
-        const bool span_ok = (p.act_min == 0 && p.act_max == 127) && (shmax - flags[1] <= 4) &&
-                             shmax <= 24;
-        int slow = span_ok ? 0 : 1;
-        if (span_ok)
-            for (int i = threadIdx.x; i < ncols_res; i += kThreads) {
-                const int ls = i / p.nt_pad, c = i - ls * p.nt_pad;
-                if (c >= p.nt || (g + ls * p.groups) * p.nt + c >= p.nf) continue;   // padding
-                const int2 bs = cbs[i];
-                const int lg = 2 + shmax - bs.y;
-                const long long ab = bs.x < 0 ? -(long long)bs.x : bs.x;
-                // |acc + bias| * 2^lg must stay below 2^31, the scaled bias within the digit range
-                if ((((long long)128 * p.k0 + ab) << lg) >= (1ll << 31) || (ab << lg) > kBiasMax)
-                    slow = 1;
-            }
-        if (slow) flags[4] = 1;
-    }
-    __syncthreads();
-    const bool fast = flags[4] == 0;
+    const bool fast = flags[4] == 0 && p.act_min == 0 && p.act_max == 127 && shmax - flags[1] <= 4 &&
+                      shmax <= 24;
 
     // bias digits of the resident channels (fast path): row n of a 32-byte-swizzled block
     if (fast)
@@ -351,81 +389,64 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 make_uint4(wd[4], wd[5], wd[6], wd[7]);
         }
 
-    // expand the resident weights into the K-major swizzled operand layout
+    // expand the resident weights from the packed copy into the K-major swizzled operand
+    // layout: one table look-up per byte of four codes
     {
-        const int rowb = (p.k0 + 3) >> 2;
         const bool quick = (p.k0 & 15) == 0;
         const int cpr = p.cw >> 4;                        // 16-byte pieces per row
         const int cpr_log2 = cpr == 8 ? 3 : (cpr == 4 ? 2 : 1);
         const int per_blk = p.nt_pad * cpr;
         const int nblk = p.subs_per_cta * p.kc;
         uint32_t invalid = 0;
-        for (int blk = 0; blk < nblk; ++blk) {
+        const bool have_w = wait_bar<true>(bar_wload, 0u, flags);
+        for (int blk = 0; have_w && blk < nblk; ++blk) {
             const int ls = blk / p.kc, chunk = blk - ls * p.kc;
             const int sub = g + ls * p.groups;
             uint8_t *dst_blk = w_smem + (size_t)blk * p.nt_pad * cw;
             const int jmax = (chunk == p.kc - 1) ? p.ksteps_last * 2 : cpr;   // pieces ever read
-            for (int base = 0; base < per_blk; base += 4 * kThreads) {
-                uint32_t word[4];
-                int tsel[4];
-                // loads first, so that they are in flight together
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int idx = base + u * kThreads + (int)threadIdx.x;
-                    word[u] = 0; tsel[u] = -1;
-                    if (idx >= per_blk) continue;
-                    const int n = idx >> cpr_log2, j = idx & (cpr - 1);
-                    if (j >= jmax) continue;
-                    tsel[u] = -2;                                  // write zeros
-                    const int nfold = sub * p.nt + n, kbase = chunk * p.cw + j * 16;
-                    if (n >= p.nt || nfold >= p.nf || kbase >= p.kf) continue;
-                    const int2 bs = cbs[ls * p.nt_pad + n];
-                    const int t = fast ? 1 + shmax - bs.y : 0;
-                    if (quick) {
-                        const int pn = nfold / p.n0, pk = kbase / p.k0;
-                        if (pn != pk) continue;                    // off the block diagonal
-                        const int n_ch = nfold - pn * p.n0, k = kbase - pk * p.k0;
-                        word[u] = __ldg(reinterpret_cast<const uint32_t *>(
-                            p.w_packed + (size_t)n_ch * rowb + (k >> 2)));
-                        tsel[u] = t;
-                    } else {
-                        tsel[u] = 16 + t;                          // element by element below
+            for (int idx = threadIdx.x; idx < per_blk; idx += kThreads) {
+                const int n = idx >> cpr_log2, j = idx & (cpr - 1);
+                if (j >= jmax) continue;
+                const int nfold = sub * p.nt + n, kbase = chunk * p.cw + j * 16;
+                uint4 val = make_uint4(0, 0, 0, 0);
+                if (n < p.nt && nfold < p.nf && kbase < p.kf) {
+                    const int t = fast ? 1 + shmax - cbs[ls * p.nt_pad + n].y : 0;
+                    int pn = 0, pk = 0;                    // diagonal block of the folded weights
+                    if (p.fold > 1) {
+                        while ((pn + 1) * p.n0 <= nfold) ++pn;
+                        while ((pk + 1) * p.k0 <= kbase) ++pk;
                     }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (tsel[u] == -1) continue;
-                    const int idx = base + u * kThreads + (int)threadIdx.x;
-                    const int n = idx >> cpr_log2, j = idx & (cpr - 1);
-                    uint4 val = make_uint4(0, 0, 0, 0);
-                    if (tsel[u] >= 16) {
-                        const int t = tsel[u] - 16;
+                    // row of this channel in the packed copy
+                    const int row = p.fold > 1 ? nfold - pn * p.n0 : ls * p.nt + n;
+                    if (quick) {
+                        if (pn == pk) {
+                            const uint32_t w = *reinterpret_cast<const uint32_t *>(
+                                wq + (size_t)row * rowb + ((kbase - pk * p.k0) >> 2));
+                            invalid |= (w >> 1) & ~w & 0x55555555u;
+                            const uint32_t *tb = lut + t * 256;
+                            val.x = tb[w & 0xFFu];
+                            val.y = tb[(w >> 8) & 0xFFu];
+                            val.z = tb[(w >> 16) & 0xFFu];
+                            val.w = tb[w >> 24];
+                        }
+                    } else {
+                        // cin is 8 modulo 16: a piece may straddle two diagonal blocks
                         const uint32_t mag = t == 0 ? 1u : (2u << t), neg = 256u - mag;
-                        const int nfold = sub * p.nt + n, kbase = chunk * p.cw + j * 16;
-                        const int pn = nfold / p.n0, n_ch = nfold - pn * p.n0;
                         uint32_t wd[4] = {0, 0, 0, 0};
                         for (int e = 0; e < 16; ++e) {
                             const int kk = kbase + e;
                             if (kk >= p.kf) break;
-                            const int pk = kk / p.k0, k = kk - pk * p.k0;
-                            if (pk != pn) continue;
-                            int wv = weight_at(p.w_packed, rowb, n_ch, k);
+                            const int pke = kk / p.k0, k = kk - pke * p.k0;
+                            if (pke != pn) continue;
+                            int wv = weight_at(wq, rowb, row, k);
                             if (wv == -2) { invalid = 1; wv = 0; }
                             const uint32_t byte = wv == 0 ? 0u : (wv > 0 ? mag : neg);
                             wd[e >> 2] |= byte << (8 * (e & 3));
                         }
                         val = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-                    } else if (tsel[u] >= 0) {
-                        const uint32_t w = word[u];
-                        invalid |= (w >> 1) & ~w & 0x55555555u;
-                        const uint32_t *tb = lut + tsel[u] * 256;
-                        val.x = tb[w & 0xFFu];
-                        val.y = tb[(w >> 8) & 0xFFu];
-                        val.z = tb[(w >> 16) & 0xFFu];
-                        val.w = tb[w >> 24];
                     }
-                    *reinterpret_cast<uint4 *>(dst_blk + swz_offset((uint32_t)n, (uint32_t)j, cw)) = val;
                 }
+                *reinterpret_cast<uint4 *>(dst_blk + swz_offset((uint32_t)n, (uint32_t)j, cw)) = val;
             }
         }
         if (invalid) raise_status(PROM_ERR_BAD_WEIGHT);
