@@ -3,7 +3,9 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <array>
 #include <atomic>
+#include <map>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -61,6 +63,7 @@ struct Conv {
     int8_t *y;
     cudaStream_t st;
     bool pdl;           // chain to the previous kernel with programmatic dependent launch
+    bool pdl_next;      // the next kernel of the sequence chains to this one
 };
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -181,7 +184,9 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
 
     // tensor memory: two CTAs share the 512 columns, or one takes them all
     int tmem_cols;
-    if (occ == 2) {
+    const bool half = occ != 1;     // occ 2: two CTAs of this kernel per SM; occ 3: one, leaving
+                                    // the other half of the SM to the next kernel's prologue
+    if (half) {
         if (2 * nt_pad > 256) return false;
         tmem_cols = 256;
     } else {
@@ -198,8 +203,8 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     const size_t wbias_bytes = (size_t)subs * nt_pad * 32;
     const size_t out_bytes = (size_t)tc::kEpiWarps * 32 * nt;
     const size_t fixed = w_bytes + wbias_bytes + tc::kAConstBytes + round_up((int)out_bytes, 128) +
-                         (size_t)ncols * 12 + tc::kLuts * 1024 + 256 + 1024 /* alignment slack */;
-    const size_t budget = occ == 2 ? (size_t)((d.smem_total - 2 * 1024) / 2) : (size_t)d.smem_optin;
+                         (size_t)ncols * 12 + 16 + 256 + tc::kLuts * 1024 + 256 + 1024 /* alignment slack */;
+    const size_t budget = half ? (size_t)((d.smem_total - 2 * 1024) / 2) : (size_t)d.smem_optin;
     if (budget > (size_t)d.smem_optin || fixed + 2 * stage_bytes > budget) return false;
     int stages = (int)((budget - fixed) / stage_bytes);
     const int share_x = (kc == 1 && subs > 1) ? 1 : 0;
@@ -226,13 +231,18 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     p.x3d = x3d; p.box_r = box_r;
     p.tx_bytes = x3d ? (uint32_t)(cw * map.wo * box_r) : (uint32_t)stage_bytes;
 
+    // shared-memory layout; [off_w, off_hdr + 16) is the CTA's prepared image
     uint32_t off = (uint32_t)(stages * stage_bytes);
     p.off_w = off; off += (uint32_t)w_bytes;
     p.off_wbias = off; off += (uint32_t)wbias_bytes;
-    p.off_aconst = off; off += tc::kAConstBytes;
-    p.off_out = off; off += (uint32_t)round_up((int)out_bytes, 128);
     p.off_mult = off; off += (uint32_t)ncols * 4;
     p.off_bs = off; off += (uint32_t)ncols * 8;
+    p.off_hdr = off; off += 16;
+    p.image_bytes = off - p.off_w;
+    p.image_stride = (p.image_bytes + 255u) & ~255u;
+    off = (off + 255u) & ~255u;
+    p.off_aconst = off; off += tc::kAConstBytes;
+    p.off_out = off; off += (uint32_t)round_up((int)out_bytes, 128);
     p.off_lut = off; off += tc::kLuts * 1024;
     p.off_bars = off; off += 256;
     pl.smem = (size_t)off + 1024;
@@ -240,7 +250,8 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
         pl.smem = (size_t)d.smem_total / 2;       // keep a second CTA (and its TMEM request) off the SM
     if (pl.smem > (size_t)d.smem_optin) return false;
 
-    const long long slots = (long long)d.sms * occ;
+    const int per_sm = occ == 2 ? 2 : 1;
+    const long long slots = (long long)d.sms * per_sm;
     long long workers = slots / groups;
     if (workers < 1) workers = 1;
     if (workers > n_mtiles) workers = n_mtiles;
@@ -249,7 +260,7 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     // rough time model (microseconds) used only to rank candidate plans
     const double rounds = (double)((n_mtiles + workers - 1) / workers);
     const double ctas_per_sm = (double)pl.grid / d.sms < 1.0 ? 1.0
-                               : ((double)pl.grid / d.sms > occ ? occ : (double)pl.grid / d.sms);
+                               : ((double)pl.grid / d.sms > per_sm ? per_sm : (double)pl.grid / d.sms);
     const double epi_rate = 30e3 / ctas_per_sm;              // outputs per microsecond per CTA
     const double load_rate = 70e3 / ctas_per_sm;             // bytes per microsecond per CTA
     const double t_epi = (double)tm * nt / epi_rate;
@@ -267,8 +278,8 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
 
 // Picks fold, subtile width, channel groups and occupancy.  Returns false when
 // the tensor-core variant cannot run this shape.
-static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
-                          TcPlan &best)
+static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
+                           TcPlan &best)
 {
     if (m <= 0 || (cin & 7) || (cout & 7)) return false;
     int fold = 1;
@@ -290,8 +301,9 @@ static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, con
         for (int groups = 1; groups <= n_sub; ++groups) {
             if (n_sub % groups) continue;
             if (g_tune.groups > 0 && groups != g_tune.groups) continue;
-            for (int occ = 2; occ >= 1; --occ) {
+            for (int occ = 3; occ >= 1; --occ) {
                 if (g_tune.occ > 0 && occ != g_tune.occ) continue;
+                if (g_tune.occ == 0 && occ == 3) continue;      // only on request for now
                 TcPlan pl;
                 if (!tc_fill_plan(m, cin, cout, map, d, fold, nt, groups, occ, g_tune.stages, pl))
                     continue;
@@ -300,6 +312,32 @@ static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, con
         }
     }
     return found;
+}
+
+
+// The search above costs tens of microseconds; its result depends only on the shape, the
+// device and the tuning override, so it is remembered.
+static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
+                          TcPlan &best)
+{
+    struct Entry { bool ok; TcPlan pl; };
+    static std::mutex mu;
+    static std::map<std::array<long long, 14>, Entry> cache;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const std::array<long long, 14> key = {m, cin, cout, map.stride, map.ho, map.wo, map.hin, map.win,
+                                           g_tune.fold, g_tune.nt, g_tune.groups, g_tune.occ,
+                                           g_tune.stages, dev};
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = cache.find(key);
+    if (it == cache.end()) {
+        Entry e;
+        e.ok = tc_search_plan(m, cin, cout, map, d, e.pl);
+        if (cache.size() > 4096) cache.clear();
+        it = cache.emplace(key, e).first;
+    }
+    if (it->second.ok) best = it->second.pl;
+    return it->second.ok;
 }
 
 static bool tc_make_maps(const Conv &c, TcPlan &pl)
@@ -346,25 +384,34 @@ static bool tc_make_maps(const Conv &c, TcPlan &pl)
     return true;
 }
 
-static prom_status launch_tc(const Conv &c)
+static prom_status tc_set_attr(const DeviceInfo &d)
 {
-    DeviceInfo d = device_info();
-    if (!d.ok) return PROM_ERR_CUDA;
-    TcPlan pl;
-    if (!tc_shape_plan(c.m, c.cin, c.cout, c.map, d, pl)) return PROM_ERR_UNSUPPORTED;
-    if (!tc_make_maps(c, pl)) return PROM_ERR_CUDA;
-    tc::Params &p = pl.p;
-    p.w_packed = c.w; p.bias = c.rq.bias; p.mult = c.rq.mult; p.shift = c.rq.shift;
-    p.act_min = c.rq.act_min; p.act_max = c.rq.act_max; p.y = c.y; p.pdl = c.pdl ? 1 : 0;
-
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
         attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tc::tc_prep_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            d.smem_optin);
     });
-    if (attr_err != cudaSuccess) return PROM_ERR_CUDA;
+    return attr_err == cudaSuccess ? PROM_OK : PROM_ERR_CUDA;
+}
 
+// Fills in the pointers of a planned layer (image: prepared operands, or null).
+static void tc_bind(const Conv &c, TcPlan &pl, uint8_t *image)
+{
+    tc::Params &p = pl.p;
+    p.w_packed = c.w; p.bias = c.rq.bias; p.mult = c.rq.mult; p.shift = c.rq.shift;
+    p.act_min = c.rq.act_min; p.act_max = c.rq.act_max; p.y = c.y; p.pdl = c.pdl ? 1 : 0;
+    p.pdl_next = c.pdl_next ? 1 : 0;
+    p.image = image;
+}
+
+static prom_status tc_launch_planned(const Conv &c, TcPlan &pl)
+{
+    if (!tc_make_maps(c, pl)) return PROM_ERR_CUDA;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)pl.grid);
@@ -378,9 +425,20 @@ static prom_status launch_tc(const Conv &c)
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
-    cudaError_t e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel, pl.xmap, pl.ymap, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel, pl.xmap, pl.ymap, pl.p);
     ++g_launches;
     return cuda_status(e);
+}
+
+static prom_status launch_tc(const Conv &c)
+{
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    TcPlan pl;
+    if (!tc_shape_plan(c.m, c.cin, c.cout, c.map, d, pl)) return PROM_ERR_UNSUPPORTED;
+    if (tc_set_attr(d) != PROM_OK) return PROM_ERR_CUDA;
+    tc_bind(c, pl, nullptr);
+    return tc_launch_planned(c, pl);
 }
 
 static bool tc_supported(const Conv &c)
@@ -451,6 +509,23 @@ static void seq_regions(const prom_layer *layers, int n, const SeqShape &s, size
     }
 }
 
+// Bytes of prepared-operand images a sequence wants in its workspace (0 for layers the
+// tensor-core variant cannot run).
+static size_t seq_image_bytes(const prom_layer *layers, int n, const SeqShape &s, const DeviceInfo &d,
+                              std::vector<size_t> *offsets)
+{
+    size_t total = 0;
+    for (int i = 0; i < n; ++i) {
+        TcPlan pl;
+        size_t bytes = 0;
+        if (tc_shape_plan(s.m[i], layers[i].cin, layers[i].cout, s.map[i], d, pl))
+            bytes = round256((size_t)pl.p.groups * pl.p.image_stride);
+        if (offsets) offsets->push_back(bytes ? total : (size_t)-1);
+        total += bytes;
+    }
+    return total;
+}
+
 static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, int batch, int h0,
                            int w0, void *ws, size_t ws_bytes, int8_t *y_out, prom_variant variant,
                            cudaStream_t st)
@@ -472,24 +547,72 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
         if (e != PROM_OK) return e;
         if (!aligned16(layers[i].w_packed)) return PROM_ERR_ALIGN;
     }
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+
+    // plan: which layers run on the tensor cores, and where their prepared operands go
+    const bool want_tc = variant == PROM_VARIANT_TC || variant == PROM_VARIANT_AUTO;
+    std::vector<Conv> conv(n);
+    std::vector<TcPlan> plan(n);
+    std::vector<char> is_tc(n, 0);
+    std::vector<size_t> img_off;
+    size_t img_total = want_tc ? seq_image_bytes(layers, n, s, d, &img_off) : 0;
+    // the images are an optimisation: a workspace without room for them still works
+    uint8_t *img_base = nullptr;
+    if (img_total > 0 && ws && ws_bytes >= round256(ra + rb) + img_total)
+        img_base = static_cast<uint8_t *>(ws) + round256(ra + rb);
     const int8_t *cur = x0;
     long long in_rows = (long long)batch * h0 * w0;
     for (int i = 0; i < n; ++i) {
-        Conv c;
+        Conv &c = conv[i];
         c.x = cur; c.m = s.m[i]; c.cin = layers[i].cin; c.cout = layers[i].cout;
         c.map = s.map[i]; c.in_rows = in_rows;
         c.w = layers[i].w_packed; c.rq = layers[i].rq;
         c.y = (i == n - 1) ? y_out : reg[i & 1];
         c.st = st;
         c.pdl = i > 0;
-        prom_status e = run_conv(c, variant);
-        if (e != PROM_OK) return e;
+        c.pdl_next = i + 1 < n;
+        if (want_tc && c.m > 0 && tc_shape_plan(c.m, c.cin, c.cout, c.map, d, plan[i])) {
+            is_tc[i] = 1;
+            tc_bind(c, plan[i], img_base && img_off[i] != (size_t)-1 ? img_base + img_off[i] : nullptr);
+        } else if (variant == PROM_VARIANT_TC && c.m > 0) {
+            return PROM_ERR_UNSUPPORTED;
+        }
         cur = c.y;
         in_rows = c.m;
     }
+    if (want_tc && tc_set_attr(d) != PROM_OK) return PROM_ERR_CUDA;
+
+    // one launch prepares the operands of every tensor-core layer
+    if (img_base) {
+        int i = 0;
+        while (i < n) {
+            tc::PrepTable t;
+            memset(&t, 0, sizeof(t));
+            size_t smem = 0;
+            int ctas = 0;
+            for (; i < n && t.n < tc::kMaxPrepLayers; ++i) {
+                if (!is_tc[i]) continue;
+                t.first[t.n] = ctas;
+                t.layer[t.n] = plan[i].p;
+                ctas += plan[i].p.groups;
+                if (plan[i].smem > smem) smem = plan[i].smem;
+                ++t.n;
+            }
+            if (t.n == 0) break;
+            t.first[t.n] = ctas;
+            tc::tc_prep_kernel<<<ctas, tc::kThreads, smem, st>>>(t);
+            ++g_launches;
+            if (cudaGetLastError() != cudaSuccess) return PROM_ERR_CUDA;
+        }
+    }
+
+    for (int i = 0; i < n; ++i) {
+        prom_status e = is_tc[i] ? tc_launch_planned(conv[i], plan[i]) : run_conv(conv[i], variant);
+        if (e != PROM_OK) return e;
+    }
     return PROM_OK;
 }
-
 
 // ---- the add/sub variant on built-in scratch (no allocation anywhere) --------------------
 // The index lists of the add/sub variant normally live in a buffer the library
@@ -565,6 +688,7 @@ prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin, const uint8
     c.w = w_packed_dev; c.rq = *rq; c.y = y_dev;
     c.st = static_cast<cudaStream_t>(cuda_stream);
     c.pdl = false;
+    c.pdl_next = false;
     return run_conv(c, variant);
 }
 
@@ -584,6 +708,7 @@ prom_status prom_pw_conv_i8_acc32(const int8_t *x_dev, int64_t m, int cin,
     c.y = nullptr;
     c.st = static_cast<cudaStream_t>(cuda_stream);
     c.pdl = false;
+    c.pdl_next = false;
     return launch_naive(c, acc_dev);
 }
 
@@ -616,7 +741,9 @@ size_t prom_layer_seq_workspace_bytes(const prom_layer *layers, int n, int batch
     if (!seq_shapes(layers, n, batch, h0, w0, s)) return 0;
     size_t a, b;
     seq_regions(layers, n, s, a, b);
-    return a + b;
+    DeviceInfo d = device_info();
+    const size_t img = d.ok ? seq_image_bytes(layers, n, s, d, nullptr) : 0;
+    return img ? round256(a + b) + img : a + b;
 }
 
 prom_status prom_pw_layer_seq(const prom_layer *layers, int n, const int8_t *x0_dev, int batch,
@@ -634,11 +761,10 @@ size_t prom_layer_seq_host_workspace_bytes(const prom_layer *layers, int n, int 
 {
     SeqShape s;
     if (!seq_shapes(layers, n, batch, h0, w0, s)) return 0;
-    size_t a, b;
-    seq_regions(layers, n, s, a, b);
+    const size_t core = round256(prom_layer_seq_workspace_bytes(layers, n, batch, h0, w0));
     size_t xin = round256((size_t)batch * h0 * w0 * layers[0].cin);
     size_t yout = round256((size_t)s.m[n - 1] * layers[n - 1].cout);
-    return a + b + xin + yout;
+    return core + xin + yout;
 }
 
 prom_status prom_pw_layer_seq_host(const prom_layer *layers, int n, const int8_t *x0_host,
@@ -650,18 +776,17 @@ prom_status prom_pw_layer_seq_host(const prom_layer *layers, int n, const int8_t
     if (!aligned16(workspace_dev)) return PROM_ERR_ALIGN;
     SeqShape s;
     if (!seq_shapes(layers, n, batch, h0, w0, s)) return PROM_ERR_SHAPE;
-    size_t a, b;
-    seq_regions(layers, n, s, a, b);
+    const size_t core = round256(prom_layer_seq_workspace_bytes(layers, n, batch, h0, w0));
     size_t xin_raw = (size_t)batch * h0 * w0 * layers[0].cin;
     size_t yout_raw = (size_t)s.m[n - 1] * layers[n - 1].cout;
     size_t xin = round256(xin_raw), yout = round256(yout_raw);
-    if (workspace_bytes < a + b + xin + yout) return PROM_ERR_WORKSPACE;
+    if (workspace_bytes < core + xin + yout) return PROM_ERR_WORKSPACE;
     int8_t *base = static_cast<int8_t *>(workspace_dev);
-    int8_t *xd = base + a + b, *yd = xd + xin;
+    int8_t *xd = base + core, *yd = xd + xin;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (cudaMemcpyAsync(xd, x0_host, xin_raw, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return PROM_ERR_CUDA;
-    prom_status e = run_seq(layers, n, xd, batch, h0, w0, base, a + b, yd, variant, st);
+    prom_status e = run_seq(layers, n, xd, batch, h0, w0, base, core, yd, variant, st);
     if (e != PROM_OK) return e;
     return cuda_status(cudaMemcpyAsync(y_out_host, yd, yout_raw, cudaMemcpyDeviceToHost, st));
 }

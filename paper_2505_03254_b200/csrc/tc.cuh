@@ -63,13 +63,20 @@ struct Params {
     int store_2d;       // 0: rows of a slab are contiguous in Y (one subtile), 1: tensor-map store
     int x3d, box_r;     // 3-D activation map (strided input); rows of dim 2 per tile
     uint32_t tx_bytes;
-    uint32_t off_w, off_wbias, off_aconst, off_out, off_mult, off_bs, off_lut, off_bars;
+    uint32_t off_w, off_wbias, off_mult, off_bs, off_hdr, off_aconst, off_out, off_lut, off_bars;
+    // A CTA's prepared operands (expanded weights, bias digits, multipliers, {bias, shift},
+    // header) are one contiguous range of shared memory, [off_w, off_hdr + 16).  When `image`
+    // is set it holds that range for every channel group, image_stride bytes apart, written
+    // by tc_prep_kernel; the convolution kernel then copies it in instead of building it.
+    uint8_t *image;
+    uint32_t image_bytes, image_stride;
     const uint8_t *w_packed;
     const int32_t *bias, *mult;
     const int8_t *shift;
     int act_min, act_max;
     int8_t *y;
     int pdl;            // launched with programmatic dependent launch
+    int pdl_next;       // the next kernel in the stream is launched that way
 };
 
 // Bounded wait on an mbarrier phase.  The clock is read only every 1024 polls (a
@@ -207,58 +214,74 @@ __device__ __forceinline__ void epi_subtile(const Params &p, uint32_t taddr, con
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
-tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
-               const Params p)
+// Where the parts of a CTA's shared memory are.
+struct View {
+    uint8_t *smem;
+    uint32_t smem_base;
+    uint8_t *w_smem, *wbias_smem, *aconst_smem;
+    int *cmult;          // mult per resident column
+    int2 *cbs;           // {bias, shift} per resident column
+    int *hdr;            // {shmax, fast epilogue, bad constants, 0}
+    uint32_t *lut;       // [kLuts][256]
+    volatile int *flags; // [0] abort, [1] shmin, [2] shmax, [3] bad constants, [4] slow path
+    uint32_t bar_wload;
+};
+
+__device__ __forceinline__ View make_view(const Params &p, uint8_t *smem, uint64_t *bars)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t smem_base = ptx::smem_u32(smem);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-
-    uint8_t *w_smem = smem + p.off_w;
-    uint8_t *wbias_smem = smem + p.off_wbias;
-    uint8_t *aconst_smem = smem + p.off_aconst;
-    int *cmult = reinterpret_cast<int *>(smem + p.off_mult);        // mult per resident column
-    int2 *cbs = reinterpret_cast<int2 *>(smem + p.off_bs);          // {bias, shift} per column
-    uint32_t *lut = reinterpret_cast<uint32_t *>(smem + p.off_lut); // [kLuts][256]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + p.off_bars);
-    // barrier slots: full[kMaxStages], empty[kMaxStages], tfull[kMaxBufs], tempty[kMaxBufs], drain
-    const uint32_t bar_full = ptx::smem_u32(bars);
-    const uint32_t bar_empty = bar_full + 8 * kMaxStages;
-    const uint32_t bar_tfull = bar_empty + 8 * kMaxStages;
-    const uint32_t bar_tempty = bar_tfull + 8 * kMaxBufs;
-    const uint32_t bar_drain = bar_tempty + 8 * kMaxBufs;
-    const uint32_t bar_wload = bar_drain + 8;
+    View v;
+    v.smem = smem;
+    v.smem_base = ptx::smem_u32(smem);
+    v.w_smem = smem + p.off_w;
+    v.wbias_smem = smem + p.off_wbias;
+    v.aconst_smem = smem + p.off_aconst;
+    v.cmult = reinterpret_cast<int *>(smem + p.off_mult);
+    v.cbs = reinterpret_cast<int2 *>(smem + p.off_bs);
+    v.hdr = reinterpret_cast<int *>(smem + p.off_hdr);
+    v.lut = reinterpret_cast<uint32_t *>(smem + p.off_lut);
     constexpr int kBarSlots = 2 * kMaxStages + 2 * kMaxBufs + 2;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + kBarSlots);
-    volatile int *flags = reinterpret_cast<volatile int *>(bars + kBarSlots + 1);
-    // flags[0] abort, flags[1] shmin, flags[2] shmax, flags[3] bad constants, flags[4] slow path
+    v.flags = reinterpret_cast<volatile int *>(bars + kBarSlots + 1);
+    v.bar_wload = ptx::smem_u32(bars) + 8 * (kBarSlots - 1);
+    return v;
+}
 
-    const int g = blockIdx.x % p.groups;
-    const int worker = blockIdx.x / p.groups;
-    const int nworkers = gridDim.x / p.groups;
+// The constant A block of the bias step: bytes 0,1 = 1, bytes 2..31 = 127.
+__device__ __forceinline__ void build_aconst(uint8_t *aconst_smem)
+{
+    for (int i = threadIdx.x; i < 128 * 2; i += kThreads) {
+        const uint32_t r = (uint32_t)i >> 1, j = (uint32_t)i & 1u;
+        const uint4 val = j == 0 ? make_uint4(0x7F7F0101u, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu)
+                                 : make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
+        *reinterpret_cast<uint4 *>(aconst_smem + swz_offset(r, j, 32u)) = val;
+    }
+}
+
+// Builds the prepared operands of channel group g in shared memory: requantisation
+// constants checked and stored, the fast/exact decision, bias digits, and the 2-bit weights
+// expanded into the K-major swizzled int8 operand layout.  All kThreads threads take part
+// (three block-wide syncs inside); on return the header is written but not yet synchronised.
+// Thread 0 starts the bulk copy of the group's packed weights into the not yet used
+// activation stages; meanwhile every thread requests the constants of its channels and
+// builds the code tables.
+__device__ __forceinline__ void build_image(const Params &p, const int g, const View &vw)
+{
+    uint8_t *const smem = vw.smem;
+    const uint32_t smem_base = vw.smem_base;
+    uint8_t *const w_smem = vw.w_smem, *const wbias_smem = vw.wbias_smem;
+    int *const cmult = vw.cmult;
+    int2 *const cbs = vw.cbs;
+    int *const hdr = vw.hdr;
+    uint32_t *const lut = vw.lut;
+    volatile int *const flags = vw.flags;
+    const uint32_t bar_wload = vw.bar_wload;
     const int ncols_res = p.subs_per_cta * p.nt_pad;
     const uint32_t cw = (uint32_t)p.cw;
-    const uint32_t stage_bytes = 128u * cw;
-
-    // ---- prologue: nothing here depends on the previous kernel's output -------------
     // Thread 0 sets up the barriers and starts the bulk copy of this CTA's packed (2-bit)
     // weights into the not yet used activation stages; meanwhile every thread requests the
     // constants of its channels and builds the code tables.  Three block-wide syncs in all.
     const int rowb = (p.k0 + 3) >> 2;
     const uint8_t *wq = smem;                    // packed weights: rows of rowb bytes
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(bar_full + 8 * s, 1);
-            ptx::mbar_init(bar_empty + 8 * s, 1);
-        }
-        for (int b = 0; b < p.nbuf; ++b) {
-            ptx::mbar_init(bar_tfull + 8 * b, 1);
-            ptx::mbar_init(bar_tempty + 8 * b, kEpiWarps / kEpiGroups);
-        }
-        ptx::mbar_init(bar_drain, 1);
         ptx::mbar_init(bar_wload, 1);
         ptx::mbar_init_fence();
         flags[0] = 0; flags[1] = 31; flags[2] = 0; flags[3] = 0; flags[4] = 0;
@@ -275,10 +298,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 ptx::bulk_load(smem_base + (uint32_t)ls * bytes,
                                p.w_packed + (size_t)(g + ls * p.groups) * bytes, bytes, bar_wload);
         }
-        ptx::tma_prefetch_desc(&xmap);
-        if (p.store_2d) ptx::tma_prefetch_desc(&ymap);
     }
-    if (warp == 1) ptx::tmem_alloc(ptx::smem_u32((const void *)tmem_slot), (uint32_t)p.tmem_cols);
 
     // constants of up to kConstPerThread resident channels per thread, requested early
     constexpr int kConstPerThread = 4;
@@ -308,13 +328,6 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             w4 |= val << (8 * e);
         }
         lut[i] = w4;
-    }
-    // the constant A block of the bias step: bytes 0,1 = 1, bytes 2..31 = 127
-    for (int i = threadIdx.x; i < 128 * 2; i += kThreads) {
-        const uint32_t r = (uint32_t)i >> 1, j = (uint32_t)i & 1u;
-        const uint4 val = j == 0 ? make_uint4(0x7F7F0101u, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu)
-                                 : make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
-        *reinterpret_cast<uint4 *>(aconst_smem + swz_offset(r, j, 32u)) = val;
     }
     __syncthreads();                                        // barriers and flags are set up
 
@@ -452,16 +465,91 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         if (invalid) raise_status(PROM_ERR_BAD_WEIGHT);
         if (bad_consts && threadIdx.x == 0) raise_status(PROM_ERR_BAD_REQUANT);
     }
+    if (threadIdx.x == 0) {
+        hdr[0] = shmax; hdr[1] = fast ? 1 : 0; hdr[2] = bad_consts ? 1 : 0; hdr[3] = 0;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
+               const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t smem_base = ptx::smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    uint8_t *w_smem = smem + p.off_w;
+    uint8_t *wbias_smem = smem + p.off_wbias;
+    uint8_t *aconst_smem = smem + p.off_aconst;
+    int *cmult = reinterpret_cast<int *>(smem + p.off_mult);        // mult per resident column
+    int2 *cbs = reinterpret_cast<int2 *>(smem + p.off_bs);          // {bias, shift} per column
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + p.off_bars);
+    // barrier slots: full[kMaxStages], empty[kMaxStages], tfull[kMaxBufs], tempty[kMaxBufs], drain
+    const uint32_t bar_full = ptx::smem_u32(bars);
+    const uint32_t bar_empty = bar_full + 8 * kMaxStages;
+    const uint32_t bar_tfull = bar_empty + 8 * kMaxStages;
+    const uint32_t bar_tempty = bar_tfull + 8 * kMaxBufs;
+    const uint32_t bar_drain = bar_tempty + 8 * kMaxBufs;
+    const uint32_t bar_wload = bar_drain + 8;
+    constexpr int kBarSlots = 2 * kMaxStages + 2 * kMaxBufs + 2;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + kBarSlots);
+    volatile int *flags = reinterpret_cast<volatile int *>(bars + kBarSlots + 1);
+    // flags[0] abort, flags[1] shmin, flags[2] shmax, flags[3] bad constants, flags[4] slow path
+
+    const int g = blockIdx.x % p.groups;
+    const int worker = blockIdx.x / p.groups;
+    const int nworkers = gridDim.x / p.groups;
+    const uint32_t cw = (uint32_t)p.cw;
+    const uint32_t stage_bytes = 128u * cw;
+
+    // Let the next kernel of the stream start its own prologue as soon as there is room for
+    // it; it waits for this grid to finish before it touches activations.
+    if (p.pdl_next) ptx::grid_dep_launch();
+
+    // ---- prologue: nothing here depends on the previous kernel's output -------------
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            ptx::mbar_init(bar_full + 8 * s, 1);
+            ptx::mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < p.nbuf; ++b) {
+            ptx::mbar_init(bar_tfull + 8 * b, 1);
+            ptx::mbar_init(bar_tempty + 8 * b, kEpiWarps / kEpiGroups);
+        }
+        ptx::mbar_init(bar_drain, 1);
+        ptx::tma_prefetch_desc(&xmap);
+        if (p.store_2d) ptx::tma_prefetch_desc(&ymap);
+    }
+    if (warp == 1) ptx::tmem_alloc(ptx::smem_u32((const void *)tmem_slot), (uint32_t)p.tmem_cols);
+    const View vw = make_view(p, smem, bars);
+    build_aconst(aconst_smem);
+    if (p.image) {
+        // prepared by tc_prep_kernel: one bulk copy
+        if (threadIdx.x == 0) {
+            ptx::mbar_init(bar_wload, 1);
+            ptx::mbar_init_fence();
+            flags[0] = 0;
+            ptx::mbar_expect_tx(bar_wload, p.image_bytes);
+            ptx::bulk_load(smem_base + p.off_w, p.image + (size_t)g * p.image_stride, p.image_bytes,
+                           bar_wload);
+        }
+        __syncthreads();
+        wait_bar<true>(bar_wload, 0u, flags);
+    } else {
+        build_image(p, g, vw);
+    }
     ptx::fence_proxy_async_smem();
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    const int shmax = vw.hdr[0];
+    const bool fast = vw.hdr[1] != 0;
+    const bool bad_consts = vw.hdr[2] != 0;
 
-    if (p.pdl) {
-        ptx::grid_dep_launch();
-        ptx::grid_dep_wait();
-    }
+    if (p.pdl) ptx::grid_dep_wait();
 
     // instruction descriptor: s8 x s8 -> s32, both K-major, M = 128, N = nt_pad
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.nt_pad >> 3) << 17) |
@@ -635,6 +723,39 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
+}
+
+
+// Prepared operands for a whole layer sequence in one launch: CTA b builds the image of
+// (layer, channel group) = the b-th entry of the table and writes it to that layer's
+// `image` buffer.  Shared-memory offsets are those of the layer's convolution launch.
+constexpr int kMaxPrepLayers = 48;
+struct PrepTable {
+    int n;
+    int first[kMaxPrepLayers + 1];     // first CTA of each layer; first[n] = grid size
+    Params layer[kMaxPrepLayers];
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_prep_kernel(const __grid_constant__ PrepTable t)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    int l = 0;
+    while (l + 1 < t.n && (int)blockIdx.x >= t.first[l + 1]) ++l;
+    const Params &p = t.layer[l];
+    const int g = (int)blockIdx.x - t.first[l];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + p.off_bars);
+    const View vw = make_view(p, smem, bars);
+    build_image(p, g, vw);
+    ptx::fence_proxy_async_smem();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        ptx::bulk_store(p.image + (size_t)g * p.image_stride, vw.smem_base + p.off_w, p.image_bytes);
+        ptx::bulk_commit();
+        ptx::bulk_wait_all();
     }
 }
 
