@@ -510,6 +510,17 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
 
     // ---- prologue: nothing here depends on the previous kernel's output -------------
     if (threadIdx.x == 0) {
+        if (p.image) {
+            // prepared by tc_prep_kernel: one bulk copy, started before anything else
+            ptx::mbar_init(bar_wload, 1);
+            ptx::mbar_init_fence();
+            ptx::mbar_expect_tx(bar_wload, p.image_bytes);
+            ptx::bulk_load(smem_base + p.off_w, p.image + (size_t)g * p.image_stride, p.image_bytes,
+                           bar_wload);
+            flags[0] = 0;
+        }
+        ptx::tma_prefetch_desc(&xmap);
+        if (p.store_2d) ptx::tma_prefetch_desc(&ymap);
         for (int s = 0; s < p.stages; ++s) {
             ptx::mbar_init(bar_full + 8 * s, 1);
             ptx::mbar_init(bar_empty + 8 * s, 1);
@@ -519,22 +530,12 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             ptx::mbar_init(bar_tempty + 8 * b, kEpiWarps / kEpiGroups);
         }
         ptx::mbar_init(bar_drain, 1);
-        ptx::tma_prefetch_desc(&xmap);
-        if (p.store_2d) ptx::tma_prefetch_desc(&ymap);
+        ptx::mbar_init_fence();
     }
     if (warp == 1) ptx::tmem_alloc(ptx::smem_u32((const void *)tmem_slot), (uint32_t)p.tmem_cols);
     const View vw = make_view(p, smem, bars);
     build_aconst(aconst_smem);
     if (p.image) {
-        // prepared by tc_prep_kernel: one bulk copy
-        if (threadIdx.x == 0) {
-            ptx::mbar_init(bar_wload, 1);
-            ptx::mbar_init_fence();
-            flags[0] = 0;
-            ptx::mbar_expect_tx(bar_wload, p.image_bytes);
-            ptx::bulk_load(smem_base + p.off_w, p.image + (size_t)g * p.image_stride, p.image_bytes,
-                           bar_wload);
-        }
         __syncthreads();
         wait_bar<true>(bar_wload, 0u, flags);
     } else {
@@ -713,7 +714,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 b += kEpiGroups;
                 if (b >= (uint32_t)p.nbuf) { b -= p.nbuf; tph ^= 1u; }
             }
-            ptx::bulk_wait_all();
+            // the stores complete with the grid; only their reads of the slab must be over
+            ptx::bulk_wait_read0();
         }
     }
 
