@@ -257,21 +257,26 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     if (workers > n_mtiles) workers = n_mtiles;
     pl.grid = (int)(workers * groups);
 
-    // rough time model (microseconds) used only to rank candidate plans
+    // Rough time model (microseconds), used only to rank candidate plans; the constants come
+    // from timing the kernel on a B200.  A CTA pays a start-up that grows with the operands it
+    // brings in, then streams its units at the rate the epilogue warps sustain, and ends with
+    // the latency of its last unit (one warp draining nt columns, then the store).
     const double rounds = (double)((n_mtiles + workers - 1) / workers);
     const double ctas_per_sm = (double)pl.grid / d.sms < 1.0 ? 1.0
                                : ((double)pl.grid / d.sms > per_sm ? per_sm : (double)pl.grid / d.sms);
-    const double epi_rate = 30e3 / ctas_per_sm;              // outputs per microsecond per CTA
-    const double load_rate = 70e3 / ctas_per_sm;             // bytes per microsecond per CTA
+    const double epi_rate = 36e3 / ctas_per_sm;              // outputs per microsecond per CTA
+    const double load_rate = 60e3 / ctas_per_sm;             // bytes per microsecond per CTA
     const double t_epi = (double)tm * nt / epi_rate;
     const double t_load = (double)kc * tm * (kf < cw ? kf : cw) / load_rate;
-    const double t_unit_first = (t_epi > t_load ? t_epi : t_load) + 0.15;
-    const double t_unit_next = share_x ? t_epi + 0.15 : t_unit_first;
-    const double pieces = (double)ncols * kc * (cw / 16);
-    const double prologue = 1.5 + pieces * 20.0 / 32.0 / (1.2 / ctas_per_sm) / 1900.0;
-    const double t_cta = prologue + rounds * (t_unit_first + (subs - 1) * t_unit_next) + 1.5;
-    const double bytes = (double)m * cin * (share_x || groups == 1 ? 1.0 : 1.0) + (double)m * cout;
-    const double t_mem = bytes / 6.0e6;
+    const double t_first = (t_epi > t_load ? t_epi : t_load) + 0.1;
+    const double t_next = share_x ? t_epi + 0.1 : t_first;
+    const double startup = 1.2 + (double)p.image_bytes / 80e3 * ctas_per_sm;
+    const double fill = 1.0 + 0.1 * kc;                      // first load, first MMA
+    const double last = 0.45 * ((nt + 31) / 32) + 0.8;       // draining the last accumulator, store
+    const double t_cta = startup + fill + rounds * (t_first + (subs - 1) * t_next) + last +
+                         (per_sm == 1 ? 0.6 : 0.0);          // one CTA per SM overlaps less
+    const double t_mem = ((double)m * cin * (groups == 1 ? 1.0 : 1.0 + 0.15 * (groups - 1)) +
+                          (double)m * cout) / 5.5e6;
     pl.est_us = t_cta > t_mem ? t_cta : t_mem;
     return true;
 }
