@@ -145,7 +145,7 @@ def build_network(seed, synth, binding=None, device=None):
 def run_reference(args):
     """The CPU oracle, as it stands, on the host cores: each step is the whole
     34-layer sequence over a bounded number of images."""
-    rank = int(os.environ.get("RANK", "0"))
+    rank, _, _ = rank_info()
     if rank != 0:
         return 0
     from oracle import prom_oracle
@@ -185,6 +185,29 @@ def run_reference(args):
     return 0
 
 
+# --------------------------------------------------------------------------- ranks
+def rank_info():
+    """(rank, local_rank, world_size) from the launcher's environment."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def max_over_ranks(ms, device="cuda"):
+    """The slowest rank's time: every multi-GPU number is the max over ranks."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(images_per_rank_per_step, steps, world, ms):
+    """Aggregate images/s of the job: all ranks' images over the slowest rank's time."""
+    return world * images_per_rank_per_step * steps / (ms * 1e-3)
+
+
 # --------------------------------------------------------------------------- GPU arm
 def time_region(torch, fn, steps, dist_on):
     """Times `steps` calls of fn with CUDA events on the current stream, bracketed
@@ -203,12 +226,7 @@ def time_region(torch, fn, steps, dist_on):
     torch.cuda.synchronize()
     if dist_on:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
-    if dist_on:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    return ms
+    return max_over_ranks(e0.elapsed_time(e1))
 
 
 def cold_time_us(torch, fn, flush, iters=20, warm=3):
@@ -233,9 +251,7 @@ def run_gpu(args):
     import torch.distributed as dist
     from paper_2505_03254_b200 import binding, build, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = rank_info()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
     torch.cuda.set_device(local)
@@ -260,8 +276,25 @@ def run_gpu(args):
     y = torch.empty((BATCH, 7, 7, 1280), dtype=torch.int8, device="cuda")
     variant = args.variant
 
-    def step():
+    side = torch.cuda.Stream()
+
+    def step_plain():
         binding.pw_layer_seq(seq, x0, ws, y_out=y, variant=variant)
+
+    l0 = binding.launch_count()
+    step_plain()
+    launches_per_step = binding.launch_count() - l0
+    torch.cuda.synchronize()
+    graph = None
+    if not args.no_graph:
+        # the step's launches (one prep kernel + one kernel per layer) captured once and replayed
+        with torch.cuda.stream(side):
+            binding.pw_layer_seq(seq, x0, ws, y_out=y, variant=variant, stream=side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            binding.pw_layer_seq(seq, x0, ws, y_out=y, variant=variant, stream=side)
+    step = graph.replay if graph is not None else step_plain
 
     sampler = ClockSampler(local)
     for _ in range(max(args.warmup, 3)):
@@ -272,11 +305,11 @@ def run_gpu(args):
 
     # ---- device-resident timing ------------------------------------------------
     sampler.start()
-    l0 = binding.launch_count()
     ms = time_region(torch, step, args.steps, dist_on)
-    launches = binding.launch_count() - l0
+    launches = launches_per_step * args.steps
     ms_per_step = ms / args.steps
-    value = world * BATCH * args.steps / (ms * 1e-3)
+    value = whole_job_value(BATCH, args.steps, world, ms)
+    ms_plain = time_region(torch, step_plain, min(args.steps, 200), dist_on) / min(args.steps, 200)
 
     # ---- end to end: pinned host input -> device -> sequence -> host output ------
     x0_host = x0.cpu().pin_memory()
@@ -292,7 +325,7 @@ def run_gpu(args):
     e2e_steps = args.steps
     ms_e2e = time_region(torch, step_e2e, e2e_steps, dist_on)
     sampler.stop()
-    e2e_value = world * BATCH * e2e_steps / (ms_e2e * 1e-3)
+    e2e_value = whole_job_value(BATCH, e2e_steps, world, ms_e2e)
     same = bool(torch.equal(y_host, y.cpu()))
     del ws_host
 
@@ -324,9 +357,12 @@ def run_gpu(args):
                                f"chained, batch {BATCH} per GPU, post-ReLU6 int8 NHWC input "
                                f"[{BATCH},112,112,32], P(0)=0.5 ternary weights",
                    "variant": variant, "seed": seed,
+                   "launch": ("CUDA graph of the step's kernels, replayed" if graph is not None
+                              else "plain launches"),
                    "l2": "no flush: a step moves 877 MB through buffers of up to 154 MB (> 126 MB L2)",
                    "parallelism": f"batch sharded over {world} GPU(s), no collective"},
         "gops": step_ops / (ms_per_step * 1e-3) / 1e9,
+        "ms_per_step_plain_launches": ms_plain,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x0_host.numel()),
                 "d2h_bytes_per_step": int(y_host.numel()), "ms_per_step": ms_e2e / e2e_steps,
                 "matches_device_run": same},
@@ -511,6 +547,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", default="auto", choices=["auto", "tc", "naive"])
+    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
