@@ -33,6 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio on B200 (4.5 : 2.25)
 FLUSH_BYTES = 512 << 20       # > 2x the 126 MB L2
+NCU_TRAFFIC_PER_LAUNCH = 15.29e6
 
 
 # --------------------------------------------------------------------------- helpers
@@ -342,7 +343,10 @@ def run_gpu(args):
     achieved = step_bytes / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "tc_conv_kernel", "achieved": achieved,
                 "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
-                "peak_source": pk["source"], "traffic": None,
+                "peak_source": pk["source"],
+                # dram read + write bytes per tc_conv_kernel launch (average over the step's 34
+                # launches) from the ncu capture summarised in profiles/; None once the kernel changes
+                "traffic": NCU_TRAFFIC_PER_LAUNCH,
                 "launches_per_step": launches / args.steps,
                 "bytes_per_launch": step_bytes / (launches / args.steps),
                 "us_per_launch": ms_per_step * 1e3 / (launches / args.steps),
