@@ -126,6 +126,18 @@ __device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&v)[NC])
     else ptx::tmem_ld_x8(taddr, v);
 }
 
+// Once a warp has read the last columns of an accumulator into registers it hands the
+// accumulator back (one arrival per warp), so that the next MMA overlaps the arithmetic
+// on those registers.  bar == 0: not the last columns.
+__device__ __forceinline__ void release_acc(uint32_t bar)
+{
+    if (bar) {
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(bar);
+    }
+}
+
 // Rows of the staging slab are nt bytes apart: 16-byte aligned only when nt is a
 // multiple of 16 (`wide`), 8-byte aligned otherwise.
 template <int NC>
@@ -147,11 +159,12 @@ __device__ __forceinline__ void put_row(uint8_t *dst, const uint32_t (&out)[NC /
 // multiply-add (rounding term in the addend), one shift, saturating pack, halve.
 template <int NC>
 __device__ __forceinline__ void epi_fast(uint32_t taddr, const int *__restrict__ cm, int shmax,
-                                         uint8_t *dst, bool wide)
+                                         uint8_t *dst, bool wide, uint32_t release_bar)
 {
     uint32_t v[NC];
     tmem_ld<NC>(taddr, v);
     ptx::tmem_wait_ld();
+    release_acc(release_bar);
     uint32_t out[NC / 4];
     const long long r64 = 1ll << (32 + shmax);   // rounding term, in the addend of the 64-bit product
     const int sh = 32 + shmax;
@@ -173,11 +186,12 @@ __device__ __forceinline__ void epi_fast(uint32_t taddr, const int *__restrict__
 template <int NC>
 __device__ __forceinline__ void epi_exact(uint32_t taddr, const int *__restrict__ cm,
                                           const int2 *__restrict__ cbs, int lo, int hi, uint8_t *dst,
-                                          bool wide)
+                                          bool wide, uint32_t release_bar)
 {
     uint32_t v[NC];
     tmem_ld<NC>(taddr, v);
     ptx::tmem_wait_ld();
+    release_acc(release_bar);
     uint32_t out[NC / 4];
 #pragma unroll
     for (int c = 0; c < NC; c += 4) {
@@ -195,22 +209,27 @@ __device__ __forceinline__ void epi_exact(uint32_t taddr, const int *__restrict_
 
 template <bool FAST>
 __device__ __forceinline__ void epi_subtile(const Params &p, uint32_t taddr, const int *cm,
-                                            const int2 *cbs, int shmax, uint8_t *dst_row)
+                                            const int2 *cbs, int shmax, uint8_t *dst_row,
+                                            uint32_t bar_release)
 {
     const bool wide = (p.nt & 15) == 0;
+    const int tail = p.nt & 31;          // columns after the last full chunk of 32
     int c = 0;
     for (; c + 32 <= p.nt; c += 32) {
-        if constexpr (FAST) epi_fast<32>(taddr + c, cm + c, shmax, dst_row + c, wide);
-        else epi_exact<32>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide);
+        const uint32_t rel = (tail == 0 && c + 32 == p.nt) ? bar_release : 0u;
+        if constexpr (FAST) epi_fast<32>(taddr + c, cm + c, shmax, dst_row + c, wide, rel);
+        else epi_exact<32>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, rel);
     }
     if (c + 16 <= p.nt) {
-        if constexpr (FAST) epi_fast<16>(taddr + c, cm + c, shmax, dst_row + c, wide);
-        else epi_exact<16>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide);
+        const uint32_t rel = (c + 16 == p.nt) ? bar_release : 0u;
+        if constexpr (FAST) epi_fast<16>(taddr + c, cm + c, shmax, dst_row + c, wide, rel);
+        else epi_exact<16>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, rel);
         c += 16;
     }
     if (c + 8 <= p.nt) {
-        if constexpr (FAST) epi_fast<8>(taddr + c, cm + c, shmax, dst_row + c, wide);
-        else epi_exact<8>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide);
+        if constexpr (FAST) epi_fast<8>(taddr + c, cm + c, shmax, dst_row + c, wide, bar_release);
+        else epi_exact<8>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide,
+                          bar_release);
     }
 }
 
@@ -673,12 +692,11 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 __syncwarp();
                 const uint32_t taddr = t_lane + b * p.nt_pad;
                 const int *cms = cmult + ls * p.nt_pad;
-                if (fast) epi_subtile<true>(p, taddr, cms, nullptr, shmax, my_row);
-                else epi_subtile<false>(p, taddr, cms, cbs + ls * p.nt_pad, shmax, my_row);
-                ptx::tc_fence_before_sync();
+                const uint32_t bar_rel = bar_tempty + 8 * b;
+                if (fast) epi_subtile<true>(p, taddr, cms, nullptr, shmax, my_row, bar_rel);
+                else epi_subtile<false>(p, taddr, cms, cbs + ls * p.nt_pad, shmax, my_row, bar_rel);
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(bar_tempty + 8 * b);
                 const long long row0 = (long long)mt * p.tm + q * 32;
                 const long long lim = p.m_rows - row0;
                 int rows_valid = p.tm - q * 32;
