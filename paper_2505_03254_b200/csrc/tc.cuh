@@ -528,27 +528,28 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     if (p.pdl_next) ptx::grid_dep_launch();
 
     // ---- prologue: nothing here depends on the previous kernel's output -------------
-    if (threadIdx.x == 0) {
-        if (p.image) {
-            // prepared by tc_prep_kernel: one bulk copy, started before anything else
-            ptx::mbar_init(bar_wload, 1);
-            ptx::mbar_init_fence();
-            ptx::mbar_expect_tx(bar_wload, p.image_bytes);
-            ptx::bulk_load(smem_base + p.off_w, p.image + (size_t)g * p.image_stride, p.image_bytes,
-                           bar_wload);
-            flags[0] = 0;
+    if (threadIdx.x == 0 && p.image) {
+        // prepared by tc_prep_kernel: one bulk copy, started before anything else
+        ptx::mbar_init(bar_wload, 1);
+        ptx::mbar_init_fence();
+        ptx::mbar_expect_tx(bar_wload, p.image_bytes);
+        ptx::bulk_load(smem_base + p.off_w, p.image + (size_t)g * p.image_stride, p.image_bytes,
+                       bar_wload);
+        flags[0] = 0;
+    }
+    if (warp == 0) {
+        // the pipeline's barriers, one lane each
+        if (lane < p.stages) {
+            ptx::mbar_init(bar_full + 8 * lane, 1);
+            ptx::mbar_init(bar_empty + 8 * lane, 1);
+        } else if (lane >= 16 && lane < 16 + p.nbuf) {
+            ptx::mbar_init(bar_tfull + 8 * (lane - 16), 1);
+            ptx::mbar_init(bar_tempty + 8 * (lane - 16), kEpiWarps / kEpiGroups);
+        } else if (lane == 31) {
+            ptx::mbar_init(bar_drain, 1);
+            ptx::tma_prefetch_desc(&xmap);
+            if (p.store_2d) ptx::tma_prefetch_desc(&ymap);
         }
-        ptx::tma_prefetch_desc(&xmap);
-        if (p.store_2d) ptx::tma_prefetch_desc(&ymap);
-        for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(bar_full + 8 * s, 1);
-            ptx::mbar_init(bar_empty + 8 * s, 1);
-        }
-        for (int b = 0; b < p.nbuf; ++b) {
-            ptx::mbar_init(bar_tfull + 8 * b, 1);
-            ptx::mbar_init(bar_tempty + 8 * b, kEpiWarps / kEpiGroups);
-        }
-        ptx::mbar_init(bar_drain, 1);
         ptx::mbar_init_fence();
     }
     if (warp == 1) ptx::tmem_alloc(ptx::smem_u32((const void *)tmem_slot), (uint32_t)p.tmem_cols);
@@ -569,8 +570,6 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     const bool fast = vw.hdr[1] != 0;
     const bool bad_consts = vw.hdr[2] != 0;
 
-    if (p.pdl) ptx::grid_dep_wait();
-
     // instruction descriptor: s8 x s8 -> s32, both K-major, M = 128, N = nt_pad
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.nt_pad >> 3) << 17) |
                            ((128u >> 4) << 24);
@@ -587,6 +586,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 uint32_t dst = smem_base, bfull = bar_full, bempty = bar_empty;
                 const int cx_end = p.share_x ? p.cw : p.kc * p.cw;
                 bool ok = true;
+                // Only this thread reads what the previous kernel wrote; everything else in the
+                // CTA follows from its loads, so it alone waits for that kernel to finish.
+                if (p.pdl) ptx::grid_dep_wait();
                 for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers) {
                     const int c_row = p.x3d ? mt * p.box_r : mt * p.tm;
                     int cx = 0;
