@@ -265,9 +265,9 @@ __device__ __forceinline__ View make_view(const Params &p, uint8_t *smem, uint64
 }
 
 // The constant A block of the bias step: bytes 0,1 = 1, bytes 2..31 = 127.
-__device__ __forceinline__ void build_aconst(uint8_t *aconst_smem)
+__device__ __forceinline__ void build_aconst(uint8_t *aconst_smem, int tid, int nthreads)
 {
-    for (int i = threadIdx.x; i < 128 * 2; i += kThreads) {
+    for (int i = tid; i < 128 * 2; i += nthreads) {
         const uint32_t r = (uint32_t)i >> 1, j = (uint32_t)i & 1u;
         const uint4 val = j == 0 ? make_uint4(0x7F7F0101u, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu)
                                  : make_uint4(0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu);
@@ -554,21 +554,37 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     }
     if (warp == 1) ptx::tmem_alloc(ptx::smem_u32((const void *)tmem_slot), (uint32_t)p.tmem_cols);
     const View vw = make_view(p, smem, bars);
-    build_aconst(aconst_smem);
-    if (p.image) {
-        __syncthreads();
-        wait_bar<true>(bar_wload, 0u, flags);
+    // With a prepared image, warp 0 (the producer) does not take part in the rest of the
+    // prologue: it announces the barriers and goes straight to its loads, which need neither
+    // weights nor constants, while the other nine warps wait for the image.
+    const bool split = p.image != nullptr;
+    if (split) {
+        if (warp == 0) {
+            __syncwarp();
+            ptx::named_arrive(1, kThreads);
+        } else {
+            build_aconst(aconst_smem, (int)threadIdx.x - 32, kThreads - 32);
+            ptx::named_sync(1, kThreads);
+            wait_bar<true>(bar_wload, 0u, flags);
+            ptx::fence_proxy_async_smem();
+            ptx::tc_fence_before_sync();
+            ptx::named_sync(2, kThreads - 32);
+            ptx::tc_fence_after_sync();
+        }
     } else {
+        build_aconst(aconst_smem, (int)threadIdx.x, kThreads);
         build_image(p, g, vw);
+        ptx::fence_proxy_async_smem();
+        ptx::tc_fence_before_sync();
+        __syncthreads();
+        ptx::tc_fence_after_sync();
     }
-    ptx::fence_proxy_async_smem();
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
-    const int shmax = vw.hdr[0];
-    const bool fast = vw.hdr[1] != 0;
-    const bool bad_consts = vw.hdr[2] != 0;
+    const bool solo = split && warp == 0;        // has not seen the image or tensor memory
+    const uint32_t tmem_base = solo ? 0u : *tmem_slot;
+    const int shmax = solo ? 0 : vw.hdr[0];
+    const bool fast = solo ? false : vw.hdr[1] != 0;
+    const bool bad_consts = solo ? false : vw.hdr[2] != 0;
+    if (bad_consts && threadIdx.x == 32) flags[0] = 1;      // stops the producer too
 
     // instruction descriptor: s8 x s8 -> s32, both K-major, M = 128, N = nt_pad
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.nt_pad >> 3) << 17) |
