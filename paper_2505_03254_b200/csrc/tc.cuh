@@ -590,6 +590,10 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.nt_pad >> 3) << 17) |
                            ((128u >> 4) << 24);
     const int loads_per_tile = p.share_x ? 1 : p.subs_per_cta * p.kc;
+    // One load per unit (one K chunk, one subtile): the k-th unit uses stage k % stages, and the
+    // epilogue, which learns of the MMA's completion anyway, frees that stage for the producer;
+    // this spares the MMA thread one of its four tcgen05 instructions per unit.
+    const bool epi_frees = p.kc == 1 && p.subs_per_cta == 1;
 
     if (!bad_consts) {
         // The two single-thread roles below run beside many busy epilogue warps, so every
@@ -646,6 +650,34 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 const int ks_full = p.cw >> 5;
                 uint32_t s = 0, ph = 0, a_lo = a_lo0, bfull = bar_full, bempty = bar_empty;
                 uint32_t b = 0, tph = 0, d_tmem = tmem_base, btfull = bar_tfull, btempty = bar_tempty;
+                if (epi_frees) {
+                    // One load, one accumulator per tile: the shortest path this thread can take.
+                    // It competes for issue slots with the epilogue warps, so what it executes
+                    // per tile is what bounds the tile rate of streaming layers.
+                    const uint64_t b_desc = d_cw | (uint64_t)b_lo0, wb_desc = d_32 | (uint64_t)wb_lo0;
+                    const uint32_t a_end = a_lo0 + (uint32_t)p.stages * a_step;
+                    const uint32_t bfull_end = bar_full + 8u * (uint32_t)p.stages;
+                    const uint32_t btfull_end = bar_tfull + 8u * (uint32_t)p.nbuf;
+                    const uint32_t tempty_off = bar_tempty - bar_tfull;
+                    const int nks = p.ksteps_last;
+                    int left = (p.n_mtiles - worker + nworkers - 1) / nworkers;
+                    for (; left > 0 && ok; --left) {
+                        if (!ptx::mbar_try_wait(btfull + tempty_off, tph ^ 1u) &&
+                            !wait_bar(btfull + tempty_off, tph ^ 1u, flags)) { ok = false; break; }
+                        if (!ptx::mbar_try_wait(bfull, ph) && !wait_bar(bfull, ph, flags)) { ok = false; break; }
+                        ptx::tc_fence_after_sync();
+                        ptx::mma_i8(d_tmem, d_cw | (uint64_t)a_lo, b_desc, idesc, 0u);
+                        for (int ks = 1; ks < nks; ++ks)
+                            ptx::mma_i8(d_tmem, d_cw | (uint64_t)(a_lo + 2 * ks), b_desc + 2 * ks, idesc, 1u);
+                        if (fast) ptx::mma_i8(d_tmem, ac_desc, wb_desc, idesc, 1u);
+                        ptx::mma_commit(btfull);
+                        a_lo += a_step; bfull += 8;
+                        if (bfull == bfull_end) { ph ^= 1u; a_lo = a_lo0; bfull = bar_full; }
+                        d_tmem += p.nt_pad; btfull += 8;
+                        if (btfull == btfull_end) { tph ^= 1u; d_tmem = tmem_base; btfull = bar_tfull; }
+                    }
+                    (void)a_end;
+                } else
                 for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers) {
                     uint32_t b_lo = b_lo0, wb_lo = wb_lo0;
                     for (int ls = 0; ls < p.subs_per_cta && ok; ++ls) {
@@ -665,7 +697,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                             }
                             b_lo += b_step;
                             if (!p.share_x || ls == p.subs_per_cta - 1) {
-                                ptx::mma_commit(bempty);
+                                if (!epi_frees) ptx::mma_commit(bempty);
                                 ++s; a_lo += a_step; bfull += 8; bempty += 8;
                                 if (s == (uint32_t)p.stages) {
                                     s = 0; ph ^= 1u; a_lo = a_lo0; bfull = bar_full; bempty = bar_empty;
@@ -702,8 +734,14 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             int mt = worker, ls = grp;                  // this group's first unit
             while (ls >= p.subs_per_cta) { ls -= p.subs_per_cta; mt += nworkers; }
             uint32_t b = (uint32_t)grp, tph = 0;
+            uint32_t st = (uint32_t)grp % (uint32_t)p.stages;    // stage of this group's unit (epi_frees)
             while (mt < p.n_mtiles && ok) {
                 if (!wait_bar<true>(bar_tfull + 8 * b, tph, flags)) { ok = false; break; }
+                if (epi_frees) {
+                    if (q == 0 && lane == 0) ptx::mbar_arrive(bar_empty + 8 * st);
+                    st += kEpiGroups;
+                    if (st >= (uint32_t)p.stages) st -= p.stages;
+                }
                 ptx::tc_fence_after_sync();
                 // the previous bulk store must have read the slab before it is rewritten
                 ptx::bulk_wait_read0();
