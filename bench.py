@@ -34,6 +34,7 @@ FALLBACK_BF16_TFLOPS = 1590.0
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio on B200 (4.5 : 2.25)
 FLUSH_BYTES = 512 << 20       # > 2x the 126 MB L2
 NCU_TRAFFIC_PER_LAUNCH = 15.29e6
+MULHI_LANES_PER_CLK_SM = 31.6   # mul.hi.s32 issue rate measured on B200 (independent chains, all SMs)
 
 
 # --------------------------------------------------------------------------- helpers
@@ -352,6 +353,14 @@ def run_gpu(args):
                 "us_per_launch": ms_per_step * 1e3 / (launches / args.steps),
                 "step_roofline_us": sum(roof_us),
                 "step_roofline_frac": sum(roof_us) / (ms_per_step * 1e3)}
+
+    # second roof of the requantising epilogue: one 32-bit high multiply per output, an
+    # instruction the SM retires at 31.6 lanes per clock (measured), i.e. a quarter of the fp32 rate
+    step_outputs = sum(m * l.cout for m, l in zip(ms_layers, table))
+    alu_peak = 148 * MULHI_LANES_PER_CLK_SM * 1.965e9
+    roofline["epilogue_alu"] = {"bound": "alu", "achieved": step_outputs / (ms_per_step * 1e-3),
+                                "peak": alu_peak, "unit": "outputs/s",
+                                "frac": step_outputs / (ms_per_step * 1e-3) / alu_peak}
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -150,8 +150,14 @@ prom_status prom_pw_conv_i8_host(const int8_t *x_host, int64_t m, int cin,
  * [batch][h0][w0][layers[0].cin]; the result y_out_dev is
  * [batch][h][w][layers[n-1].cout] with h, w divided by every in_stride.
  * Intermediate activations live in the caller's workspace (two ping-pong
- * regions); prom_layer_seq_workspace_bytes gives the size needed (0 on a
- * shape error).  `variant` applies to every layer (AUTO picks per layer). */
+ * regions), followed by the prepared operands of the tensor-core layers
+ * (expanded weights, bias digits, constants; rebuilt by one small kernel at
+ * the start of every call, so the call stays stateless);
+ * prom_layer_seq_workspace_bytes gives the size needed (0 on a shape error).
+ * A workspace that only holds the two activation regions still works, more
+ * slowly.  `variant` applies to every layer (AUTO picks per layer).  The
+ * kernels of one call are chained with programmatic dependent launch and can
+ * be captured into a CUDA graph. */
 size_t prom_layer_seq_workspace_bytes(const prom_layer *layers, int n,
                                       int batch, int h0, int w0);
 prom_status prom_pw_layer_seq(const prom_layer *layers, int n,
@@ -212,14 +218,16 @@ prom_status prom_last_device_status(void *cuda_stream);
  * streams, this process); used by the benchmark to count launches. */
 uint64_t prom_launch_count(void);
 
-/* Tuning aid for the TC variant: forces the row fold, the subtile width, the
- * number of output-channel groups, CTAs per SM (1 or 2) and the depth of the
- * activation ring of later calls; 0 leaves a choice to the library.  A forced
- * combination that does not fit makes TC report PROM_ERR_UNSUPPORTED.  Results
- * never depend on the plan.  Not thread-safe.  prom_debug_tc_plan_query
- * writes the plan the library would use for a plain [m][cin] x [cout] layer
- * ({fold, nt, groups, grid, stages, accumulators, shared bytes, chunk bytes,
- * estimate in 1/100 us}) and returns 1, or returns 0 if TC cannot run it. */
+/* Tuning aid for the TC variant: forces the row fold (1, 2, 4, 8), the subtile
+ * width, the number of output-channel groups, the way CTAs share an SM (1: one
+ * CTA with all of tensor memory; 2: two CTAs of the kernel per SM; 3: one
+ * half-sized CTA per SM) and the depth of the activation ring of later calls;
+ * 0 leaves a choice to the library.  A forced combination that does not fit
+ * makes TC report PROM_ERR_UNSUPPORTED.  Results never depend on the plan.  Not
+ * thread-safe.  prom_debug_tc_plan_query writes the plan the library would
+ * use for a plain [m][cin] x [cout] layer ({fold, nt, groups, grid, stages,
+ * accumulators, shared bytes, chunk bytes, estimate in 1/100 us}) and returns
+ * 1, or returns 0 if TC cannot run it. */
 void prom_debug_tc_plan(int fold, int nt, int groups, int occ, int stages);
 int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
 

@@ -274,7 +274,7 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     const double fill = 1.0 + 0.1 * kc;                      // first load, first MMA
     const double last = 0.45 * ((nt + 31) / 32) + 0.8;       // draining the last accumulator, store
     const double t_cta = startup + fill + rounds * (t_first + (subs - 1) * t_next) + last +
-                         (per_sm == 1 ? 0.6 : 0.0);          // one CTA per SM overlaps less
+                         (occ == 1 ? 2.5 : 0.0);   // a CTA that fills its SM keeps the next kernel out
     const double t_mem = ((double)m * cin * (groups == 1 ? 1.0 : 1.0 + 0.15 * (groups - 1)) +
                           (double)m * cout) / 5.5e6;
     pl.est_us = t_cta > t_mem ? t_cta : t_mem;
