@@ -165,8 +165,10 @@ def pack_ternary(w: torch.Tensor, stream=None) -> torch.Tensor:
 
 def make_requant(bias: torch.Tensor, mult: torch.Tensor, shift: torch.Tensor,
                  act_min: int = 0, act_max: int = 127) -> PromRequant:
-    return PromRequant(_dev(bias, torch.int32, "bias"), _dev(mult, torch.int32, "mult"),
-                       _dev(shift, torch.int8, "shift"), int(act_min), int(act_max))
+    rq = PromRequant(_dev(bias, torch.int32, "bias"), _dev(mult, torch.int32, "mult"),
+                     _dev(shift, torch.int8, "shift"), int(act_min), int(act_max))
+    rq._keep = (bias, mult, shift)      # the struct holds raw pointers: keep the tensors alive
+    return rq
 
 
 def pw_conv_i8(x: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequant,
