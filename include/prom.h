@@ -118,7 +118,8 @@ prom_status prom_pack_ternary(const int8_t *w_dev, int cout, int cin,
  *   x_dev        [m][cin]  int8, dense rows, 16-byte aligned base
  *   w_packed_dev 2-bit weights of [cout][cin], 16-byte aligned base
  *   y_dev        [m][cout] int8, 16-byte aligned base, must not overlap x_dev
- * m >= 0 (m == 0 is a no-op), 1 <= cin <= 4096, 1 <= cout <= 4096.
+ * m >= 0 (m == 0 is a no-op for which x_dev and y_dev may be NULL), 1 <= cin <= 4096,
+ * 1 <= cout <= 4096.
  * TC needs cin % 8 == 0 and cout % 8 == 0 (and even m when cin or cout is not
  * a multiple of 16); SMALLK needs cin % 4 == 0 and cin <= 64; ADDSUB and NAIVE
  * take any shape.  An explicit variant that cannot run the shape returns

@@ -684,6 +684,9 @@ prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin, const uint8
                             int cout, const prom_requant *rq, int8_t *y_dev, prom_variant variant,
                             void *cuda_stream)
 {
+    // an empty matrix has no rows to read or write: its pointers may be anything
+    if (m == 0 && cin >= 1 && cin <= 4096 && cout >= 1 && cout <= 4096 && w_packed_dev && rq)
+        return check_requant(rq);
     prom_status s = check_conv(x_dev, m, cin, w_packed_dev, cout, rq, y_dev);
     if (s != PROM_OK) return s;
     Conv c;

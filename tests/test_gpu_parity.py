@@ -177,3 +177,36 @@ def test_host_buffer_entry_point(oracle):
     binding.pw_conv_i8_host(xh, wp, cout, rq, yh, ws)
     torch.cuda.synchronize()
     assert first_mismatch(yh.numpy(), oracle_y(oracle, x, lay)) is None
+
+
+def test_empty_and_single_row(oracle):
+    """m = 0 is a no-op that touches nothing; m = 1 and m = 2 are the smallest tiles."""
+    x, lay = make_case(22, 4, 32, 48)
+    xd, wp, consts = to_device(x, lay)
+    rq = binding.make_requant(*consts)
+    y = torch.full((0, 48), 7, dtype=torch.int8, device="cuda")
+    for variant in ["auto", "tc", "smallk", "addsub", "naive"]:
+        binding.pw_conv_i8(xd[:0], wp, 48, rq, y=y, variant=variant)
+    for rows in (1, 2):
+        want = oracle_y(oracle, x[:rows], lay)
+        for variant in ["auto", "smallk", "addsub", "naive"]:
+            got = run_variant(xd[:rows].contiguous(), wp, consts, 48, variant)
+            assert first_mismatch(got, want) is None, (rows, variant)
+
+
+def test_largest_channel_counts(oracle):
+    """Cin = Cout = 4096, the largest the interface accepts (weights 16 M ternary values)."""
+    m, c = 260, 4096
+    x = synth.act_uniform_i8(23, (m, c))
+    lay = synth.make_layer(23, c, c, 0.5)
+    xd, wp, consts = to_device(x, lay)
+    rows = np.array([0, 1, 127, 128, 129, 259])
+    want = oracle_y(oracle, x[rows], lay)
+    ref = None
+    for variant in ["tc", "naive"]:
+        got = run_variant(xd, wp, consts, c, variant)
+        assert first_mismatch(got[rows], want) is None, variant
+        if ref is None:
+            ref = got
+        else:
+            assert np.array_equal(got, ref)

@@ -155,3 +155,72 @@ def test_config3_full_size_sequence(oracle):
     assert torch.equal(y_auto, y_naive)
     want = oracle.layer_seq(host, x0[:2].cpu().numpy())
     assert np.array_equal(y_auto[:2].cpu().numpy(), want)
+
+
+def test_sequence_with_small_workspace_and_mixed_variants(oracle):
+    """The prepared-operand images are an optimisation: a workspace that only
+    holds the two activation regions gives the same bytes.  The second half
+    mixes in layers the tensor-core variant refuses (Cin = 20, Cout = 12), which
+    AUTO runs on other kernels inside the same chained call."""
+    table = synth.mobilenetv2_pointwise_layers(h0=32, w0=32)[:12]
+    host, seq = build_sequence(41, table)
+    x0 = synth.act_post_relu6(41, (4, 32, 32, 32))
+    want = oracle.layer_seq(host, x0.numpy())
+    full = seq.workspace_bytes(4, 32, 32)
+    regions = 0
+    h = w = 32
+    sizes = []
+    for l in table:
+        h //= l.in_stride; w //= l.in_stride
+        sizes.append((4 * h * w * l.cout + 255) // 256 * 256)
+    regions = max(sizes[0:-1:2]) + max(sizes[1:-1:2])
+    assert regions < full
+    for nbytes in (full, regions):
+        ws = torch.empty((nbytes,), dtype=torch.uint8, device="cuda")
+        y = binding.pw_layer_seq(seq, x0.cuda(), ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(y.cpu().numpy(), want), nbytes
+
+    shapes = [(32, 64, 1), (64, 20, 1), (20, 12, 1), (12, 48, 2), (48, 16, 1)]
+    host, dev = [], []
+    for i, (cin, cout, stride) in enumerate(shapes):
+        d = synth.make_layer(42, cin, cout, 0.5, index=i + 1)
+        host.append(dict(cin=cin, cout=cout, in_stride=stride, w=d["w"].numpy(), bias=d["bias"].numpy(),
+                         mult=d["mult"].numpy(), shift=d["shift"].numpy()))
+        dev.append(dict(cin=cin, cout=cout, in_stride=stride, w_packed=binding.pack_ternary(d["w"].cuda()),
+                        bias=d["bias"].cuda(), mult=d["mult"].cuda(), shift=d["shift"].cuda()))
+    seq2 = binding.LayerSeq(dev)
+    x0 = synth.act_post_relu6(42, (3, 16, 16, 32))
+    ws = torch.empty((max(16, seq2.workspace_bytes(3, 16, 16)),), dtype=torch.uint8, device="cuda")
+    y = binding.pw_layer_seq(seq2, x0.cuda(), ws, variant="auto")
+    torch.cuda.synchronize()
+    assert np.array_equal(y.cpu().numpy(), oracle.layer_seq(host, x0.numpy()))
+    with pytest.raises(binding.PromError) as e:
+        binding.pw_layer_seq(seq2, x0.cuda(), ws, variant="tc")
+    assert e.value.code == binding.PROM_ERR_UNSUPPORTED
+
+
+def test_sequence_twice_and_in_a_cuda_graph(oracle):
+    """Two calls in a row reuse the workspace (the images are rebuilt each time),
+    and a captured call replays to the same bytes."""
+    table = synth.mobilenetv2_pointwise_layers(h0=32, w0=32)
+    host, seq = build_sequence(43, table)
+    x0 = synth.act_post_relu6(43, (2, 32, 32, 32)).cuda()
+    want = oracle.layer_seq(host, x0.cpu().numpy())
+    ws = torch.empty((seq.workspace_bytes(2, 32, 32),), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    y = torch.zeros(want.shape, dtype=torch.int8, device="cuda")
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
+    torch.cuda.synchronize()
+    assert np.array_equal(y.cpu().numpy(), want)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
+    for _ in range(3):
+        y.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(y.cpu().numpy(), want)
+    assert binding.last_device_status() == binding.PROM_OK
