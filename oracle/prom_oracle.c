@@ -32,6 +32,7 @@
  * arithmetic for the requantiser, hand-built ties, and byte tables for the
  * 2-bit codes.  No function in this file is "parity unpinned".
  */
+#include <math.h>
 #include <stdint.h>
 #include <stddef.h>
 #include <stdlib.h>
@@ -266,5 +267,61 @@ int prom_ref_layer_seq(int n, const int *cin, const int *cout, const int *in_str
         cur = dst;
         h = ho; wd = wo;
     }
+    return 0;
+}
+
+/* ---- ternary absmean quantiser (the step before the path) ---------------- */
+/*
+ * Paper, Section 3.1, Eq. 1-3, and the pointwise branch of the quantiser in
+ * Figure 10: per output channel i
+ *     alpha_i = mean_j |W[i][j]|
+ *     W-hat[i][j] = max(-1, min(1, round(W[i][j] / alpha_i)))
+ * Readings taken where the paper is at odds with itself: the division guard
+ * is the figure's (the mean is clamped from below by eps = 1e-5) rather than
+ * Eq. 3's (eps added to the mean); `round` is the framework's, i.e. ties go
+ * to the even integer, so a ratio of exactly 0.5 gives 0 and 1.5 gives 2 -> 1.
+ * The paper fixes no summation order; mean and ratio are taken in binary64 so
+ * that the order cannot matter at the precision of the float32 inputs.
+ * w: [cout][cin] float32; q: [cout][cin] in {-1,0,+1}; alpha: [cout].
+ */
+void prom_ref_quantize_ternary(const float *w, int cout, int cin, double eps,
+                               int8_t *q, double *alpha)
+{
+    for (int i = 0; i < cout; ++i) {
+        double sum = 0.0;
+        for (int j = 0; j < cin; ++j) sum += fabs((double)w[(long)i * cin + j]);
+        double mean = sum / (double)cin;
+        alpha[i] = mean;
+        double scale = 1.0 / (mean < eps ? eps : mean);
+        for (int j = 0; j < cin; ++j) {
+            double r = nearbyint((double)w[(long)i * cin + j] * scale);   /* ties to even */
+            if (r > 1.0) r = 1.0;
+            if (r < -1.0) r = -1.0;
+            q[(long)i * cin + j] = (int8_t)r;
+        }
+    }
+}
+
+/*
+ * The fixed-point pair that stands for a real per-channel scale (the paper
+ * scales by alpha and the activation scales in floating point, Figure 12; the
+ * build's contract wants mult in [2^30, 2^31) and a right shift): the shift is
+ * the one that puts scale * 2^(31+shift) into [2^30, 2^31], and mult is that
+ * number rounded to nearest (a result of 2^31 is renormalised to 2^30 with the
+ * shift one smaller).  Returns 0, or -1 when scale is not positive or the
+ * shift would leave [0, 31].
+ */
+int prom_ref_requant_from_scale(double scale, int32_t *mult, int *shift)
+{
+    if (!(scale > 0.0) || isinf(scale)) return -1;
+    int sh = 0;
+    double v = scale * 2147483648.0;            /* scale * 2^31 */
+    while (v >= 2147483648.0) { v /= 2.0; --sh; }
+    while (v < 1073741824.0) { v *= 2.0; ++sh; if (sh > 64) return -1; }
+    double m = floor(v + 0.5);
+    if (m >= 2147483648.0) { m = 1073741824.0; --sh; }
+    if (sh < 0 || sh > 31) return -1;
+    *mult = (int32_t)m;
+    *shift = sh;
     return 0;
 }

@@ -25,7 +25,7 @@ def build(force: bool = False) -> str:
         return _LIB
     tmp = _LIB + f".tmp{os.getpid()}"
     subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-shared", "-fPIC",
-                           "-Wall", "-o", tmp, _SRC])
+                           "-Wall", "-o", tmp, _SRC, "-lm"])
     os.replace(tmp, _LIB)
     return _LIB
 
@@ -56,6 +56,10 @@ def lib():
             C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
             C.POINTER(i8p), C.POINTER(i32p), C.POINTER(i32p), C.POINTER(i8p),
             C.c_int, C.c_int, i8p, C.c_int, C.c_int, C.c_int, i8p]
+        L.prom_ref_quantize_ternary.argtypes = [C.POINTER(C.c_float), C.c_int, C.c_int, C.c_double,
+                                                i8p, C.POINTER(C.c_double)]
+        L.prom_ref_requant_from_scale.restype = C.c_int
+        L.prom_ref_requant_from_scale.argtypes = [C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_int)]
         _lib = L
     return _lib
 
@@ -186,3 +190,23 @@ def layer_seq(layers, x0, act_min=0, act_max=127) -> np.ndarray:
     if rc != 0:
         raise ValueError("layer sequence does not chain")
     return y
+
+
+def quantize_ternary(w, eps: float = 1e-5):
+    """Absmean ternary quantiser (paper Eq. 1-3 / Figure 10).  w: float32 [cout, cin].
+    Returns (q int8 [cout, cin] in {-1,0,+1}, alpha float64 [cout])."""
+    w = _c(w, np.float32)
+    cout, cin = w.shape
+    q = np.empty((cout, cin), dtype=np.int8)
+    alpha = np.empty((cout,), dtype=np.float64)
+    lib().prom_ref_quantize_ternary(_p(w, C.c_float), cout, cin, float(eps), _p(q, C.c_int8),
+                                    _p(alpha, C.c_double))
+    return q, alpha
+
+
+def requant_from_scale(scale: float):
+    """(mult, shift) with mult in [2^30, 2^31) and mult * 2^-(31+shift) nearest to scale."""
+    m, s = C.c_int32(), C.c_int()
+    if lib().prom_ref_requant_from_scale(float(scale), C.byref(m), C.byref(s)) != 0:
+        raise ValueError("scale cannot be represented with a shift in [0, 31]")
+    return int(m.value), int(s.value)
