@@ -387,6 +387,7 @@ def run_gpu(args):
     if rank == 0 and world == 1 and not args.no_detail:
         out["layers"] = per_layer_detail(torch, binding, synth, table, dev, seed, bw, p_i8, variant)
         out["single_layer"] = single_layer_configs(torch, binding, synth, bw, p_i8)
+        out["quantizer"] = quantizer_timing(torch, binding, table, bw)
         cold_us = sum(r["us"] for r in out["layers"])
         roofline["sum_layer_cold_us"] = cold_us
         roofline["sum_layer_cold_frac"] = sum(roof_us) / cold_us
@@ -435,6 +436,22 @@ def per_layer_detail(torch, binding, synth, table, dev, seed, bw, p_i8, variant)
                      "roof_us": round(roof, 2), "frac": round(roof / med, 3)})
         del x, yy
     return rows
+
+
+def quantizer_timing(torch, binding, table, bw):
+    """The step before the path (off the timed step): float weights of all 34 layers ->
+    alpha and 2-bit ternary codes, one launch per layer, L2 flushed before the batch."""
+    import math
+    g = torch.Generator(device="cuda").manual_seed(1)
+    ws = [torch.randn((l.cout, l.cin), generator=g, device="cuda") * math.sqrt(2.0 / l.cout) for l in table]
+    flush = torch.empty((FLUSH_BYTES,), dtype=torch.uint8, device="cuda")
+    fn = lambda: [binding.quantize_ternary(w) for w in ws]
+    med, mn = cold_time_us(torch, fn, flush, iters=10)
+    nbytes = sum(4 * w.numel() + (w.shape[0] * ((w.shape[1] + 3) // 4)) + 4 * w.shape[0] for w in ws)
+    return {"workload": "float32 weights of the 34 layers (2.1 M) -> alpha + 2-bit codes, 34 launches",
+            "us": round(med, 2), "us_min": round(mn, 2), "bytes": nbytes,
+            "gbs": round(nbytes / med / 1e3, 1), "roof_us": round(nbytes / bw * 1e6, 2),
+            "frac": round(nbytes / bw * 1e6 / med, 4)}
 
 
 def single_layer_configs(torch, binding, synth, bw, p_i8):

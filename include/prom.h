@@ -113,6 +113,26 @@ prom_status prom_pack_ternary(const int8_t *w_dev, int cout, int cin,
                               uint8_t *packed_dev, size_t packed_bytes,
                               void *cuda_stream);
 
+/* The step before the path: quantises float weights w_dev[cout][cin] to ternary
+ * and writes them in the 2-bit form straight away (Section 3.1, Eq. 1-3;
+ * Figure 10, pointwise branch): alpha_i = mean_j |W[i][j]|,
+ * W-hat = clip(round(W / max(alpha_i, 1e-5)), -1, 1), ties to the even integer
+ * as the framework's round does, the division guarded as in the figure (Eq. 3
+ * adds the epsilon instead).  alpha_dev (cout floats, may be NULL) receives the
+ * per-channel scales, by which the paper multiplies the integer result
+ * afterwards.  Asynchronous on `cuda_stream`; a NaN weight sets
+ * PROM_ERR_BAD_WEIGHT in the device status word. */
+prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin,
+                                  uint8_t *packed_dev, size_t packed_bytes,
+                                  float *alpha_dev, void *cuda_stream);
+
+/* Host helper: the fixed-point pair for a real per-channel scale (alpha_i times
+ * the activation scales and whatever BatchNorm folds in; Figure 12 divides by
+ * these in floating point): mult in [2^30, 2^31) and shift in [0, 31] with
+ * mult * 2^-(31+shift) the nearest such number to `scale`.  0 < scale < 1;
+ * PROM_ERR_BAD_REQUANT when the shift would leave its range. */
+prom_status prom_requant_from_scale(double scale, int32_t *mult, int8_t *shift);
+
 /* One ternary pointwise convolution with fused requantisation (Section 3.1,
  * inference form; formula at the top of this file).
  *   x_dev        [m][cin]  int8, dense rows, 16-byte aligned base

@@ -28,6 +28,7 @@ EXPORTS = [
     "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
     "prom_launch_count", "prom_shutdown", "prom_status_string",
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
+    "prom_quantize_ternary", "prom_requant_from_scale",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -87,6 +88,10 @@ def lib():
         L.prom_debug_tc_plan.argtypes = [i32, i32, i32, i32, i32]
         L.prom_debug_tc_plan_query.restype = i32
         L.prom_debug_tc_plan_query.argtypes = [i64, i32, i32, C.POINTER(C.c_int)]
+        L.prom_quantize_ternary.restype = i32
+        L.prom_quantize_ternary.argtypes = [vp, i32, i32, vp, sz, vp, vp]
+        L.prom_requant_from_scale.restype = i32
+        L.prom_requant_from_scale.argtypes = [C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_int8)]
         L.prom_last_device_status.restype = i32
         L.prom_last_device_status.argtypes = [vp]
         L.prom_launch_count.restype = C.c_uint64
@@ -161,6 +166,25 @@ def pack_ternary(w: torch.Tensor, stream=None) -> torch.Tensor:
     _check(lib().prom_pack_ternary(_dev(w, torch.int8, "w"), cout, cin, out.data_ptr(),
                                    out.numel(), _stream(stream)), "prom_pack_ternary")
     return out
+
+
+def quantize_ternary(w: torch.Tensor, want_alpha: bool = True, stream=None):
+    """prom_quantize_ternary: device float32 [cout, cin] -> (packed uint8 [cout, ceil(cin/4)],
+    alpha float32 [cout] or None)."""
+    cout, cin = w.shape
+    packed = torch.empty((cout, (cin + 3) // 4), dtype=torch.uint8, device=w.device)
+    alpha = torch.empty((cout,), dtype=torch.float32, device=w.device) if want_alpha else None
+    _check(lib().prom_quantize_ternary(_dev(w, torch.float32, "w"), cout, cin, packed.data_ptr(),
+                                       packed.numel(), alpha.data_ptr() if want_alpha else None,
+                                       _stream(stream)), "prom_quantize_ternary")
+    return packed, alpha
+
+
+def requant_from_scale(scale: float):
+    """prom_requant_from_scale: (mult, shift) for a real scale in (0, 1)."""
+    m, s = C.c_int32(), C.c_int8()
+    _check(lib().prom_requant_from_scale(float(scale), C.byref(m), C.byref(s)), "prom_requant_from_scale")
+    return int(m.value), int(s.value)
 
 
 def make_requant(bias: torch.Tensor, mult: torch.Tensor, shift: torch.Tensor,

@@ -7,6 +7,7 @@
 #include <atomic>
 #include <map>
 #include <cstdio>
+#include <cmath>
 #include <cstring>
 #include <mutex>
 #include <unordered_map>
@@ -19,6 +20,7 @@
 #include "tc.cuh"
 #include "smallk.cuh"
 #include "addsub.cuh"
+#include "quantize.cuh"
 
 namespace prom {
 
@@ -678,6 +680,36 @@ prom_status prom_pack_ternary(const int8_t *w_dev, int cout, int cin, uint8_t *p
         return PROM_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return PROM_ERR_CUDA;
     return host_bad ? PROM_ERR_BAD_WEIGHT : PROM_OK;
+}
+
+prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin, uint8_t *packed_dev,
+                                  size_t packed_bytes, float *alpha_dev, void *cuda_stream)
+{
+    if (!w_dev || !packed_dev) return PROM_ERR_NULL;
+    if (cout < 1 || cin < 1 || cout > 4096 || cin > 4096) return PROM_ERR_SHAPE;
+    if (packed_bytes < prom_packed_bytes(cout, cin)) return PROM_ERR_WORKSPACE;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    const int grid = cout < d.sms * 8 ? cout : d.sms * 8;
+    quant::quantize_ternary_kernel<<<grid, quant::kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        w_dev, cout, cin, 1e-5, packed_dev, alpha_dev);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+prom_status prom_requant_from_scale(double scale, int32_t *mult, int8_t *shift)
+{
+    if (!mult || !shift) return PROM_ERR_NULL;
+    if (!(scale > 0.0) || scale >= 1.0) return PROM_ERR_BAD_REQUANT;
+    // scale = f * 2^(e+1) with f in [0.5, 1): mult = round(f * 2^31), shift = -(e+1)
+    int e = ilogb(scale);                        // floor(log2(scale)), <= -1
+    int sh = -(e + 1);
+    double m = nearbyint(scalbn(scale, 31 + sh));
+    if (m >= 2147483648.0) { m = 1073741824.0; --sh; }
+    if (sh < 0 || sh > 31) return PROM_ERR_BAD_REQUANT;
+    *mult = (int32_t)m;
+    *shift = (int8_t)sh;
+    return PROM_OK;
 }
 
 prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin, const uint8_t *w_packed_dev,

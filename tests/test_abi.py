@@ -84,3 +84,21 @@ def test_layer_seq_shape_checks(lib):
     assert lib.prom_pw_layer_seq(arr, 3, A, 2, 7, 8, A, 1 << 20, A, 0, None) == binding.PROM_ERR_SHAPE
     assert lib.prom_pw_layer_seq(arr, 3, A, 2, 8, 8, A, 16, A, 0, None) == binding.PROM_ERR_WORKSPACE
     assert lib.prom_pw_layer_seq(arr, 3, None, 2, 8, 8, A, 1 << 20, A, 0, None) == binding.PROM_ERR_NULL
+
+
+def test_requant_from_scale_matches_the_oracle(lib, oracle):
+    """Host-only helper: same (mult, shift) as the oracle's definition on random and
+    boundary scales, and the documented refusals."""
+    import numpy as np
+    rng = np.random.default_rng(5)
+    scales = list(2.0 ** rng.uniform(-31.9, -0.001, size=3000))
+    scales += [0.5, 0.25, 2.0 ** -32 * 1.5, 2.0 ** -13, (1 - 2.0 ** -33) * 2.0 ** -9]
+    for sc in scales:
+        assert binding.requant_from_scale(sc) == oracle.requant_from_scale(sc), sc
+    # refused by both: not positive, not below one, rounding up to one, or too small for shift 31
+    for bad in (0.0, -0.5, 1.0, 7.0, 1 - 2.0 ** -40, 2.0 ** -40, float("nan")):
+        with pytest.raises(binding.PromError) as e:
+            binding.requant_from_scale(bad)
+        assert e.value.code == binding.PROM_ERR_BAD_REQUANT
+        with pytest.raises(ValueError):
+            oracle.requant_from_scale(bad)
