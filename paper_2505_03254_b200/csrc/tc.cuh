@@ -167,14 +167,14 @@ __device__ __forceinline__ void epi_fast(uint32_t taddr, const int *__restrict__
     release_acc(release_bar);
     uint32_t out[NC / 4];
     const long long r64 = 1ll << (32 + shmax);   // rounding term, in the addend of the 64-bit product
-    const int sh = 32 + shmax;
 #pragma unroll
     for (int c = 0; c < NC; c += 4) {
         const int4 mu = *reinterpret_cast<const int4 *>(cm + c);
-        const int q0 = (int)(((long long)(int)v[c] * mu.x + r64) >> sh);
-        const int q1 = (int)(((long long)(int)v[c + 1] * mu.y + r64) >> sh);
-        const int q2 = (int)(((long long)(int)v[c + 2] * mu.z + r64) >> sh);
-        const int q3 = (int)(((long long)(int)v[c + 3] * mu.w + r64) >> sh);
+        // high word first (a shift by the constant 32), then the 32-bit shift
+        const int q0 = (int)(((long long)(int)v[c] * mu.x + r64) >> 32) >> shmax;
+        const int q1 = (int)(((long long)(int)v[c + 1] * mu.y + r64) >> 32) >> shmax;
+        const int q2 = (int)(((long long)(int)v[c + 2] * mu.z + r64) >> 32) >> shmax;
+        const int q3 = (int)(((long long)(int)v[c + 3] * mu.w + r64) >> 32) >> shmax;
         uint32_t w = ptx::pack_sat_u8(q3, q2, 0u);
         w = ptx::pack_sat_u8(q1, q0, w);
         out[c / 4] = (w >> 1) & 0x7F7F7F7Fu;
