@@ -140,6 +140,7 @@ struct TcPlan {
     tc::Params p;
     CUtensorMap xmap, ymap;
     int grid = 0;
+    int per_sm = 2;        // CTAs of the launch that share an SM (picks the kernel build)
     size_t smem = 0;
     double est_us = 0;
 };
@@ -182,18 +183,14 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     const long long rows = m / fold;
     if ((nf & 15) && (tm & 1)) return false;     // slabs of the 1-D store start on 16-byte granules
     const long long n_mtiles = (rows + tm - 1) / tm;
-    if (n_mtiles > 0x7fffffff) return false;
+    if (rows + 256 >= (1ll << 31)) return false;   // row coordinates are 32-bit in the kernel
 
-    // tensor memory: two CTAs share the 512 columns, or one takes them all
-    int tmem_cols;
-    const bool half = occ != 1;     // occ 2: two CTAs of this kernel per SM; occ 3: one, leaving
-                                    // the other half of the SM to the next kernel's prologue
-    if (half) {
-        if (2 * nt_pad > 256) return false;
-        tmem_cols = 256;
-    } else {
-        tmem_cols = 512;
-    }
+    // tensor memory: the CTAs of an SM share its 512 columns
+    // occ 1: one CTA with all of the SM; occ 2: two CTAs; occ 3: one CTA on half an SM, leaving
+    // the other half to the next kernel's prologue; occ 4: three CTAs
+    const int share = occ == 1 ? 1 : (occ == 4 ? 3 : 2);
+    const int tmem_cols = share == 1 ? 512 : (share == 2 ? 256 : 128);
+    if (2 * nt_pad > tmem_cols) return false;
     // accumulator ring: an even length, so that each of the two epilogue groups keeps to its own
     // accumulators
     if (tmem_cols / nt_pad < 2) return false;
@@ -206,7 +203,8 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     const size_t out_bytes = (size_t)tc::kEpiWarps * 32 * nt;
     const size_t fixed = w_bytes + wbias_bytes + tc::kAConstBytes + round_up((int)out_bytes, 128) +
                          (size_t)ncols * 12 + 16 + 256 + tc::kLuts * 1024 + 256 + 1024 /* alignment slack */;
-    const size_t budget = half ? (size_t)((d.smem_total - 2 * 1024) / 2) : (size_t)d.smem_optin;
+    const size_t budget = share == 1 ? (size_t)d.smem_optin
+                                     : (size_t)((d.smem_total - share * 1024) / share);
     if (budget > (size_t)d.smem_optin || fixed + 2 * stage_bytes > budget) return false;
     int stages = (int)((budget - fixed) / stage_bytes);
     const int share_x = (kc == 1 && subs > 1) ? 1 : 0;
@@ -252,7 +250,8 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
         pl.smem = (size_t)d.smem_total / 2;       // keep a second CTA (and its TMEM request) off the SM
     if (pl.smem > (size_t)d.smem_optin) return false;
 
-    const int per_sm = occ == 2 ? 2 : 1;
+    const int per_sm = occ == 2 ? 2 : (occ == 4 ? 3 : 1);
+    pl.per_sm = per_sm;
     const long long slots = (long long)d.sms * per_sm;
     long long workers = slots / groups;
     if (workers < 1) workers = 1;
@@ -308,9 +307,9 @@ static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, co
         for (int groups = 1; groups <= n_sub; ++groups) {
             if (n_sub % groups) continue;
             if (g_tune.groups > 0 && groups != g_tune.groups) continue;
-            for (int occ = 3; occ >= 1; --occ) {
+            for (int occ = 4; occ >= 1; --occ) {
                 if (g_tune.occ > 0 && occ != g_tune.occ) continue;
-                if (g_tune.occ == 0 && occ == 3) continue;      // only on request for now
+                if (g_tune.occ == 0 && occ >= 3) continue;      // only on request for now
                 TcPlan pl;
                 if (!tc_fill_plan(m, cin, cout, map, d, fold, nt, groups, occ, g_tune.stages, pl))
                     continue;
@@ -396,8 +395,12 @@ static prom_status tc_set_attr(const DeviceInfo &d)
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel,
+        attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<3>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            d.smem_optin);
         if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(tc::tc_prep_kernel,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -432,7 +435,9 @@ static prom_status tc_launch_planned(const Conv &c, TcPlan &pl)
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
-    cudaError_t e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel, pl.xmap, pl.ymap, pl.p);
+    cudaError_t e = pl.per_sm == 3
+                        ? cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<3>, pl.xmap, pl.ymap, pl.p)
+                        : cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2>, pl.xmap, pl.ymap, pl.p);
     ++g_launches;
     return cuda_status(e);
 }

@@ -155,33 +155,6 @@ __device__ __forceinline__ void put_row(uint8_t *dst, const uint32_t (&out)[NC /
     }
 }
 
-// NC accumulator columns of this thread's row: the high word of a 64-bit
-// multiply-add (rounding term in the addend), one shift, saturating pack, halve.
-template <int NC>
-__device__ __forceinline__ void epi_fast(uint32_t taddr, const int *__restrict__ cm, int shmax,
-                                         uint8_t *dst, bool wide, uint32_t release_bar)
-{
-    uint32_t v[NC];
-    tmem_ld<NC>(taddr, v);
-    ptx::tmem_wait_ld();
-    release_acc(release_bar);
-    uint32_t out[NC / 4];
-    const long long r64 = 1ll << (32 + shmax);   // rounding term, in the addend of the 64-bit product
-#pragma unroll
-    for (int c = 0; c < NC; c += 4) {
-        const int4 mu = *reinterpret_cast<const int4 *>(cm + c);
-        // high word first (a shift by the constant 32), then the 32-bit shift
-        const int q0 = (int)(((long long)(int)v[c] * mu.x + r64) >> 32) >> shmax;
-        const int q1 = (int)(((long long)(int)v[c + 1] * mu.y + r64) >> 32) >> shmax;
-        const int q2 = (int)(((long long)(int)v[c + 2] * mu.z + r64) >> 32) >> shmax;
-        const int q3 = (int)(((long long)(int)v[c + 3] * mu.w + r64) >> 32) >> shmax;
-        uint32_t w = ptx::pack_sat_u8(q3, q2, 0u);
-        w = ptx::pack_sat_u8(q1, q0, w);
-        out[c / 4] = (w >> 1) & 0x7F7F7F7Fu;
-    }
-    put_row<NC>(dst, out, wide);
-}
-
 // The 64-bit definition (any clamp, any shifts).
 template <int NC>
 __device__ __forceinline__ void epi_exact(uint32_t taddr, const int *__restrict__ cm,
@@ -207,30 +180,81 @@ __device__ __forceinline__ void epi_exact(uint32_t taddr, const int *__restrict_
     put_row<NC>(dst, out, wide);
 }
 
-template <bool FAST>
-__device__ __forceinline__ void epi_subtile(const Params &p, uint32_t taddr, const int *cm,
-                                            const int2 *cbs, int shmax, uint8_t *dst_row,
-                                            uint32_t bar_release)
+// NC accumulator columns of this thread's row, already in registers: the high word of a
+// 64-bit multiply-add (rounding term in the addend), one shift, saturating pack, halve.
+template <int NC>
+__device__ __forceinline__ void fast_piece(const uint32_t (&v)[NC], const int *__restrict__ cm,
+                                           long long r64, int shmax, uint8_t *dst, bool wide)
+{
+    uint32_t out[NC / 4];
+#pragma unroll
+    for (int c = 0; c < NC; c += 4) {
+        const int4 mu = *reinterpret_cast<const int4 *>(cm + c);
+        const int q0 = (int)(((long long)(int)v[c] * mu.x + r64) >> 32) >> shmax;
+        const int q1 = (int)(((long long)(int)v[c + 1] * mu.y + r64) >> 32) >> shmax;
+        const int q2 = (int)(((long long)(int)v[c + 2] * mu.z + r64) >> 32) >> shmax;
+        const int q3 = (int)(((long long)(int)v[c + 3] * mu.w + r64) >> 32) >> shmax;
+        uint32_t w = ptx::pack_sat_u8(q3, q2, 0u);
+        w = ptx::pack_sat_u8(q1, q0, w);
+        out[c / 4] = (w >> 1) & 0x7F7F7F7Fu;
+    }
+    put_row<NC>(dst, out, wide);
+}
+
+// The fast epilogue over one subtile, in chunks of CH (32 or 16), then 16 and 8 columns.  The
+// accumulator goes back to the MMA thread as soon as its last columns are in registers.
+template <int CH>
+__device__ __forceinline__ void epi_fast_subtile(const Params &p, uint32_t taddr, const int *cm,
+                                                 int shmax, uint8_t *dst_row, uint32_t bar_release)
 {
     const bool wide = (p.nt & 15) == 0;
-    const int tail = p.nt & 31;          // columns after the last full chunk of 32
+    const long long r64 = 1ll << (32 + shmax);   // rounding term, in the addend of the 64-bit product
+    const int tail = p.nt & (CH - 1);            // columns after the last full chunk
     int c = 0;
-    for (; c + 32 <= p.nt; c += 32) {
-        const uint32_t rel = (tail == 0 && c + 32 == p.nt) ? bar_release : 0u;
-        if constexpr (FAST) epi_fast<32>(taddr + c, cm + c, shmax, dst_row + c, wide, rel);
-        else epi_exact<32>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, rel);
+    for (; c + CH <= p.nt; c += CH) {
+        uint32_t v[CH];
+        tmem_ld<CH>(taddr + c, v);
+        ptx::tmem_wait_ld();
+        if (tail == 0 && c + CH == p.nt) release_acc(bar_release);
+        fast_piece<CH>(v, cm + c, r64, shmax, dst_row + c, wide);
     }
-    if (c + 16 <= p.nt) {
-        const uint32_t rel = (c + 16 == p.nt) ? bar_release : 0u;
-        if constexpr (FAST) epi_fast<16>(taddr + c, cm + c, shmax, dst_row + c, wide, rel);
-        else epi_exact<16>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, rel);
+    if (CH > 16 && c + 16 <= p.nt) {
+        uint32_t v[16];
+        ptx::tmem_ld_x16(taddr + c, v);
+        ptx::tmem_wait_ld();
+        if (c + 16 == p.nt) release_acc(bar_release);
+        fast_piece<16>(v, cm + c, r64, shmax, dst_row + c, wide);
         c += 16;
     }
     if (c + 8 <= p.nt) {
-        if constexpr (FAST) epi_fast<8>(taddr + c, cm + c, shmax, dst_row + c, wide, bar_release);
-        else epi_exact<8>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide,
-                          bar_release);
+        uint32_t v[8];
+        ptx::tmem_ld_x8(taddr + c, v);
+        ptx::tmem_wait_ld();
+        release_acc(bar_release);
+        fast_piece<8>(v, cm + c, r64, shmax, dst_row + c, wide);
     }
+}
+
+// The exact epilogue over one subtile, in chunks of CH (32 or 16), then 16 and 8 columns.
+template <int CH>
+__device__ __forceinline__ void epi_exact_subtile(const Params &p, uint32_t taddr, const int *cm,
+                                                  const int2 *cbs, uint8_t *dst_row,
+                                                  uint32_t bar_release)
+{
+    const bool wide = (p.nt & 15) == 0;
+    const int tail = p.nt & (CH - 1);    // columns after the last full chunk
+    int c = 0;
+    for (; c + CH <= p.nt; c += CH) {
+        const uint32_t rel = (tail == 0 && c + CH == p.nt) ? bar_release : 0u;
+        epi_exact<CH>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, rel);
+    }
+    if (CH > 16 && c + 16 <= p.nt) {
+        const uint32_t rel = (c + 16 == p.nt) ? bar_release : 0u;
+        epi_exact<16>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, rel);
+        c += 16;
+    }
+    if (c + 8 <= p.nt)
+        epi_exact<8>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, bar_release);
 }
 
 // Where the parts of a CTA's shared memory are.
@@ -489,7 +513,9 @@ __device__ __forceinline__ void build_image(const Params &p, const int g, const 
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+// MINB: CTAs of this kernel that share an SM (2 with 96 registers a thread, 3 with 64).
+template <int MINB>
+__global__ void __launch_bounds__(kThreads, MINB)
 tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
                const Params p)
 {
@@ -498,6 +524,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = ptx::smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int CH = MINB >= 3 ? 16 : 32;     // columns per tensor-memory load in the epilogue
 
     uint8_t *w_smem = smem + p.off_w;
     uint8_t *wbias_smem = smem + p.off_wbias;
@@ -721,6 +748,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             }
         } else {
             // ---- epilogue ---------------------------------------------------------------
+            // Everything a warp does per unit besides the arithmetic is a chain of dependent
+            // scalar instructions issued among many busy warps, tens of cycles each: positions,
+            // addresses and phases advance by additions, and a full slab takes the short path.
             const int q = warp & 3;                     // TMEM lane quarter of this warp
             // Unit u goes to group u % 2 and accumulator u % nbuf; nbuf is even, so a group meets
             // each of its accumulators in cyclic order and never waits on a barrier that is more
@@ -730,12 +760,27 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             uint8_t *my_row = slab + lane * p.nt;
             const uint32_t slab_addr = ptx::smem_u32(slab);
             const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+            const int subs = p.subs_per_cta;
+            const int m_rows = (int)p.m_rows;           // the planner keeps rows below 2^31
             bool ok = true;
-            int mt = worker, ls = grp;                  // this group's first unit
-            while (ls >= p.subs_per_cta) { ls -= p.subs_per_cta; mt += nworkers; }
+            int mt0 = worker, ls = grp;                 // this group's first unit
+            while (ls >= subs) { ls -= subs; mt0 += nworkers; }
+            // the next unit of the group is two further on: with one subtile per CTA that is two
+            // tiles on, otherwise two subtiles on and at most one step to the next tile
+            const int dls = subs == 1 ? 0 : kEpiGroups;
+            const int drow = subs == 1 ? kEpiGroups * nworkers * p.tm : 0, drow_wrap = nworkers * p.tm;
+            const bool whole_tile = p.tm - q * 32 >= 32;     // a tile gives this warp 32 rows
+            int row0 = mt0 * p.tm + q * 32;             // first row of this warp's slab
+            const int row_end = p.n_mtiles * p.tm + q * 32;
+            const uint32_t slab_bytes = 32u * (uint32_t)p.nf;
+            int col = (g + ls * p.groups) * p.nt;       // first column of the subtile
+            const int dcol = dls * p.groups * p.nt;
+            const bool store_2d = p.store_2d != 0;
+            // accumulators of this group: grp alone (two in the ring) or grp and grp + 2 (four)
+            const uint32_t btoggle = p.nbuf == 4 ? 2u : 0u;
             uint32_t b = (uint32_t)grp, tph = 0;
             uint32_t st = (uint32_t)grp % (uint32_t)p.stages;    // stage of this group's unit (epi_frees)
-            while (mt < p.n_mtiles && ok) {
+            while (row0 < row_end && ok) {
                 if (!wait_bar<true>(bar_tfull + 8 * b, tph, flags)) { ok = false; break; }
                 if (epi_frees) {
                     if (q == 0 && lane == 0) ptx::mbar_arrive(bar_empty + 8 * st);
@@ -749,44 +794,48 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 const uint32_t taddr = t_lane + b * p.nt_pad;
                 const int *cms = cmult + ls * p.nt_pad;
                 const uint32_t bar_rel = bar_tempty + 8 * b;
-                if (fast) epi_subtile<true>(p, taddr, cms, nullptr, shmax, my_row, bar_rel);
-                else epi_subtile<false>(p, taddr, cms, cbs + ls * p.nt_pad, shmax, my_row, bar_rel);
+                if (fast) epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
+                else epi_exact_subtile<CH>(p, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
-                const long long row0 = (long long)mt * p.tm + q * 32;
-                const long long lim = p.m_rows - row0;
-                int rows_valid = p.tm - q * 32;
-                if (lim < rows_valid) rows_valid = (int)lim;
-                if (rows_valid > 32) rows_valid = 32;
-                if (!p.store_2d) {
-                    // one subtile spans the row: the slab is one contiguous range of Y
-                    if (lane == 0 && rows_valid > 0) {
-                        const uint32_t bytes = (uint32_t)(rows_valid * p.nf);
-                        const uint32_t whole = bytes & ~15u;      // bulk copies move 16-byte granules
-                        if (whole) {
-                            ptx::bulk_store(p.y + row0 * p.nf, slab_addr, whole);
-                            ptx::bulk_commit();
-                        }
-                        if (bytes & 15u)                          // odd last row of an 8-multiple width
-                            *reinterpret_cast<uint2 *>(p.y + row0 * p.nf + whole) =
-                                *reinterpret_cast<const uint2 *>(slab + whole);
-                    }
-                } else if (rows_valid == 32) {
+                if (whole_tile && row0 + 32 <= m_rows) {
+                    // a whole slab: one copy
                     if (lane == 0) {
-                        ptx::tma_store_2d(&ymap, (g + ls * p.groups) * p.nt, (int)row0, slab_addr);
+                        if (store_2d) ptx::tma_store_2d(&ymap, col, row0, slab_addr);
+                        else ptx::bulk_store(p.y + (long long)row0 * p.nf, slab_addr, slab_bytes);
                         ptx::bulk_commit();
                     }
-                } else if (lane < rows_valid) {
-                    // a partial slab (short tile or end of the matrix) leaves row by row
-                    ptx::bulk_store(p.y + (row0 + lane) * p.nf + (g + ls * p.groups) * p.nt,
-                                    slab_addr + (uint32_t)(lane * p.nt), (uint32_t)p.nt);
-                    ptx::bulk_commit();
+                } else {
+                    // a short tile or the end of the matrix
+                    int rows_valid = p.tm - q * 32;
+                    if (m_rows - row0 < rows_valid) rows_valid = m_rows - row0;
+                    if (rows_valid > 32) rows_valid = 32;
+                    int8_t *yp = p.y + (long long)row0 * p.nf;
+                    if (!store_2d) {
+                        // one subtile spans the row: the slab is one contiguous range of Y
+                        if (lane == 0 && rows_valid > 0) {
+                            const uint32_t bytes = (uint32_t)(rows_valid * p.nf);
+                            const uint32_t whole = bytes & ~15u;      // bulk copies move 16-byte granules
+                            if (whole) {
+                                ptx::bulk_store(yp, slab_addr, whole);
+                                ptx::bulk_commit();
+                            }
+                            if (bytes & 15u)                          // odd last row of an 8-multiple width
+                                *reinterpret_cast<uint2 *>(yp + whole) =
+                                    *reinterpret_cast<const uint2 *>(slab + whole);
+                        }
+                    } else if (lane < rows_valid) {
+                        // the slab leaves row by row
+                        ptx::bulk_store(yp + (long long)lane * p.nf + col,
+                                        slab_addr + (uint32_t)(lane * p.nt), (uint32_t)p.nt);
+                        ptx::bulk_commit();
+                    }
                 }
-                // this group's next unit: two further on
-                ls += kEpiGroups;
-                while (ls >= p.subs_per_cta) { ls -= p.subs_per_cta; mt += nworkers; }
-                b += kEpiGroups;
-                if (b >= (uint32_t)p.nbuf) { b -= p.nbuf; tph ^= 1u; }
+                // this group's next unit and accumulator
+                ls += dls; row0 += drow; col += dcol;
+                if (ls >= subs) { ls -= subs; row0 += drow_wrap; col -= p.nf; }
+                b ^= btoggle;
+                if (b < (uint32_t)kEpiGroups) tph ^= 1u;
             }
             // the stores complete with the grid; only their reads of the slab must be over
             ptx::bulk_wait_read0();
