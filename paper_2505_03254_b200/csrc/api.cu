@@ -99,7 +99,14 @@ static int grid_for(long long work_items, int threads, int sms)
     return (int)blocks;
 }
 
-static prom_status cuda_status(cudaError_t e) { return e == cudaSuccess ? PROM_OK : PROM_ERR_CUDA; }
+// With PROM_VERBOSE set in the environment the CUDA error behind a PROM_ERR_CUDA goes to stderr.
+static prom_status cuda_status(cudaError_t e)
+{
+    if (e == cudaSuccess) return PROM_OK;
+    static const bool verbose = getenv("PROM_VERBOSE") != nullptr;
+    if (verbose) fprintf(stderr, "prom: CUDA error %d: %s\n", (int)e, cudaGetErrorString(e));
+    return PROM_ERR_CUDA;
+}
 
 // ---- naive -------------------------------------------------------------------------------
 static prom_status launch_naive(const Conv &c, int32_t *acc_out)
