@@ -126,10 +126,10 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def build_network(seed, synth, binding=None, device=None):
+def build_network(seed, synth, binding=None, device=None, width=1.0):
     """Layer table plus per-layer weights/constants: host arrays for the oracle,
     and (when a binding is given) packed device tensors for the library."""
-    table = synth.mobilenetv2_pointwise_layers()
+    table = synth.mobilenetv2_pointwise_layers(width=width)
     host, dev = [], []
     for i, l in enumerate(table):
         d = synth.make_layer(seed, l.cin, l.cout, 0.5, index=i + 1)
@@ -613,6 +613,54 @@ def run_single(args):
     return 0 if st == binding.PROM_OK else 1
 
 
+def run_widths(args):
+    """The chained sequence at other width multipliers (Section 5 sweeps 0.75x-2.0x): step
+    time, throughput and fraction of the summed per-layer roofline, each checked against the
+    CPU oracle on one image.  One JSON object; not the headline line."""
+    import torch
+    from paper_2505_03254_b200 import binding, build, synth
+    from oracle import prom_oracle
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(0)
+    build.build()
+    prom_oracle.build()
+    binding.lib()
+    pk = peaks()
+    p_i8 = INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12
+    bw = pk["hbm_gbs"] * 1e9
+    seed = synth.BASE_SEED + 3
+    rows = []
+    for width in [float(v) for v in args.widths.split(",")]:
+        table, host, dev = build_network(seed, synth, binding, "cuda", width=width)
+        seq = binding.LayerSeq(dev)
+        c0, c1 = table[0].cin, table[-1].cout
+        x0 = synth.act_post_relu6(seed, (BATCH, 112, 112, c0), device="cuda")
+        ws = torch.empty((seq.workspace_bytes(BATCH, 112, 112),), dtype=torch.uint8, device="cuda")
+        y = torch.empty((BATCH, 7, 7, c1), dtype=torch.int8, device="cuda")
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
+        for _ in range(5):
+            graph.replay()
+        steps = min(args.steps, 300)
+        ms = time_region(torch, graph.replay, steps, False) / steps
+        want = prom_oracle.layer_seq(host, x0[:1].cpu().numpy())
+        ok = bool((y[:1].cpu().numpy() == want).all()) and binding.last_device_status() == binding.PROM_OK
+        roof = sum(max(layer_bytes(BATCH * l.h * l.w, l.cin, l.cout) / bw,
+                       layer_ops(BATCH * l.h * l.w, l.cin, l.cout) / p_i8) for l in table) * 1e6
+        rows.append({"width": width, "ms_per_step": round(ms, 4), "images_per_s": round(BATCH / ms * 1e3, 1),
+                     "weights": sum(l.cin * l.cout for l in table), "step_roofline_us": round(roof, 1),
+                     "frac": round(roof / (ms * 1e3), 3), "parity_image_0": ok})
+        del graph, ws, x0, y
+    print(json.dumps({"widths": rows, "batch": BATCH, "unit": UNIT, "data": "synthetic"}))
+    return 0 if all(r["parity_image_0"] for r in rows) else 1
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -625,10 +673,13 @@ def main():
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
     ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
+    ap.add_argument("--widths", default=None, help="comma-separated width multipliers: time the sequence at each")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.widths:
+        return run_widths(args)
     if args.single:
         return run_single(args)
     if args.sweep:

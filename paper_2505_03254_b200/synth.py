@@ -150,15 +150,32 @@ MOBILENETV2_TCNS = [(1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 3, 2), (6, 64, 4, 2),
                     (6, 96, 3, 1), (6, 160, 3, 2), (6, 320, 1, 1)]
 
 
+def scaled_channels(channels: int, width: float, divisor: int = 8) -> int:
+    """Channel count under a width multiplier: the nearest multiple of `divisor`
+    (at least `divisor`), raised by one step where rounding would lose more than a
+    tenth of the scaled count.  This is the usual rule of MobileNet-family models."""
+    v = channels * width
+    c = max(divisor, int(v + divisor / 2) // divisor * divisor)
+    if c < 0.9 * v:
+        c += divisor
+    return c
+
+
 def mobilenetv2_pointwise_layers(stem_channels: int = 32, h0: int = 112, w0: int = 112,
-                                 head_channels: int = 1280) -> List[LayerShape]:
-    """Every 1x1 convolution of MobileNetV2 (width 1.0): per inverted-residual
-    block a ternary expand (omitted when t = 1) and a ternary project, then the
-    head convolution.  The block's stride sits in its depthwise convolution,
-    so the project after a stride-2 depthwise reads a subsampled input."""
+                                 head_channels: int = 1280, width: float = 1.0) -> List[LayerShape]:
+    """Every 1x1 convolution of MobileNetV2: per inverted-residual block a ternary
+    expand (omitted when t = 1) and a ternary project, then the head convolution.
+    The block's stride sits in its depthwise convolution, so the project after a
+    stride-2 depthwise reads a subsampled input.  `width` scales every channel count
+    (Section 5, Experiments: widths 0.75x to 2.0x); the head only grows, for widths above one."""
     layers: List[LayerShape] = []
     c, h, w = stem_channels, h0, w0
+    if width != 1.0:
+        c = scaled_channels(stem_channels, width)
+        head_channels = scaled_channels(head_channels, max(1.0, width))
     for bi, (t, cout, n, s) in enumerate(MOBILENETV2_TCNS, start=1):
+        if width != 1.0:
+            cout = scaled_channels(cout, width)
         for r in range(n):
             stride = s if r == 0 else 1
             hidden = c * t

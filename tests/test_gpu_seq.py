@@ -47,6 +47,49 @@ def test_mobilenetv2_sequence_small(oracle, variant, batch, hw):
     assert first_mismatch(y.cpu().numpy().reshape(-1, 1280), want.reshape(-1, 1280)) is None
 
 
+@pytest.mark.parametrize("width", [0.75, 1.4, 2.0])
+def test_mobilenetv2_sequence_width_multipliers(oracle, width):
+    """The widths the paper sweeps (Section 5: 0.75x to 2.0x): channel counts such as
+    72, 120, 136, 224, 448, 1344 and 2560, most of them not multiples of 32, some only of 8."""
+    table = synth.mobilenetv2_pointwise_layers(h0=32, w0=32, width=width)
+    host, seq = build_sequence(33, table)
+    x0 = synth.act_post_relu6(33, (2, 32, 32, table[0].cin))
+    ws = torch.empty((seq.workspace_bytes(2, 32, 32),), dtype=torch.uint8, device="cuda")
+    y = binding.pw_layer_seq(seq, x0.cuda(), ws)
+    torch.cuda.synchronize()
+    want = oracle.layer_seq(host, x0.numpy())
+    assert y.shape == want.shape
+    c = table[-1].cout
+    assert first_mismatch(y.cpu().numpy().reshape(-1, c), want.reshape(-1, c)) is None
+    assert binding.last_device_status() == binding.PROM_OK
+
+
+@pytest.mark.parametrize("width", [0.75, 1.4])
+def test_width_multiplier_layers_on_the_tensor_cores(oracle, width):
+    """Every distinct (Cin, Cout) of a scaled network as a single tensor-core call with
+    a ragged number of rows, where the tensor-core variant takes the shape."""
+    seen = set()
+    for l in synth.mobilenetv2_pointwise_layers(width=width):
+        if (l.cin, l.cout) in seen:
+            continue
+        seen.add((l.cin, l.cout))
+        m = 300
+        x = synth.act_uniform_i8(34, (m, l.cin))
+        lay = synth.make_layer(34, l.cin, l.cout, 0.5, index=len(seen))
+        want = oracle.conv_mul(x.numpy(), lay["w"].numpy(), lay["bias"].numpy(),
+                               lay["mult"].numpy(), lay["shift"].numpy())
+        wp = binding.pack_ternary(lay["w"].cuda())
+        rq = binding.make_requant(lay["bias"].cuda(), lay["mult"].cuda(), lay["shift"].cuda())
+        for variant in ("auto", "tc"):
+            try:
+                y = binding.pw_conv_i8(x.cuda(), wp, l.cout, rq, variant=variant)
+            except binding.PromError as e:
+                assert variant == "tc" and e.code == binding.PROM_ERR_UNSUPPORTED, (l, variant, e)
+                continue
+            torch.cuda.synchronize()
+            assert first_mismatch(y.cpu().numpy(), want) is None, (l.cin, l.cout, variant)
+
+
 def test_sequence_host_entry_point(oracle):
     table = synth.mobilenetv2_pointwise_layers(h0=32, w0=32)[:9]
     host, seq = build_sequence(32, table)

@@ -131,3 +131,24 @@ def test_layer_table_against_paper_figures():
     for a, b in zip(layers, layers[1:]):
         assert a.cout == b.cin
         assert b.h * b.in_stride == a.h
+
+
+def test_width_multiplier_tables():
+    """Width 1.0 is the plain table; scaled tables keep the block structure, channel counts
+    stay multiples of 8 and within a tenth of the scaled value, the head grows only above 1.0."""
+    base = synth.mobilenetv2_pointwise_layers()
+    assert synth.mobilenetv2_pointwise_layers(width=1.0) == base
+    assert [synth.scaled_channels(c, 0.75) for c in (16, 24, 32, 64, 96, 160, 320)] == \
+        [16, 24, 24, 48, 72, 120, 240]
+    assert synth.scaled_channels(24, 1.4) == 32 and synth.scaled_channels(320, 1.4) == 448
+    for width in (0.75, 1.25, 1.4, 2.0):
+        t = synth.mobilenetv2_pointwise_layers(width=width)
+        assert len(t) == len(base)
+        for a, b in zip(t, base):
+            assert (a.name, a.in_stride, a.h, a.w) == (b.name, b.in_stride, b.h, b.w)
+            assert a.cin % 8 == 0 and a.cout % 8 == 0
+            if "project" in a.name:
+                assert 0.9 * b.cout * width <= a.cout <= b.cout * width + 8
+        for prev, cur in zip(t, t[1:]):
+            assert cur.cin == prev.cout
+        assert t[-1].cout == (1280 if width <= 1.0 else synth.scaled_channels(1280, width))
