@@ -242,7 +242,8 @@ uint64_t prom_launch_count(void);
 /* Tuning aid for the TC variant: forces the row fold (1, 2, 4, 8), the subtile
  * width, the number of output-channel groups, the way CTAs share an SM (1: one
  * CTA with all of tensor memory; 2: two CTAs of the kernel per SM; 3: one
- * half-sized CTA per SM) and the depth of the activation ring of later calls;
+ * half-sized CTA per SM; 4: three CTAs per SM, on a build of the kernel with 64
+ * registers a thread) and the depth of the activation ring of later calls;
  * 0 leaves a choice to the library.  A forced combination that does not fit
  * makes TC report PROM_ERR_UNSUPPORTED.  Results never depend on the plan.  Not
  * thread-safe.  prom_debug_tc_plan_query writes the plan the library would
