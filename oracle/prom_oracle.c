@@ -325,3 +325,46 @@ int prom_ref_requant_from_scale(double scale, int32_t *mult, int *shift)
     *shift = sh;
     return 0;
 }
+
+/*
+ * Per-sample absmax quantisation of activations to 8 bits: paper, Section 3.1
+ * ("Activations", the two equations after Eq. 5, numbered 6 and 7 here) and the
+ * activation figure of the pseudocode appendix.  For sample i over all its
+ * channels and pixels
+ *     gamma_i = max |X[i][...]|
+ *     scale_i = 127 / max(gamma_i, eps)
+ *     X-hat[i][...] = max(-128, min(127, round(X[i][...] * scale_i)))
+ * Readings: the text's second equation divides by (gamma_i + eps) and leaves the
+ * 127 out, which would map every value into [-1, 1] before rounding; the figure
+ * multiplies by 127 / clamp(gamma_i, eps), and that is what is computed here.
+ * `round` is the framework's (ties to even).  The rounding decision is taken in
+ * binary32, the precision the paper's framework computes in: the quotient and
+ * the product are each one correctly rounded binary32 operation (volatile keeps
+ * the compiler from carrying extra precision or fusing them), so a second
+ * implementation that uses the same two operations must agree bit for bit.
+ * x: [batch][per_sample] float32 (any layout inside a sample: the maximum does
+ * not care); q: same shape, int8; gamma, scale: [batch].
+ */
+void prom_ref_quantize_act_absmax(const float *x, int batch, long per_sample, float eps,
+                                  int8_t *q, float *gamma, float *scale)
+{
+    for (int i = 0; i < batch; ++i) {
+        const float *xi = x + (long)i * per_sample;
+        float mx = 0.0f;
+        for (long j = 0; j < per_sample; ++j) {
+            float a = fabsf(xi[j]);
+            if (a > mx) mx = a;
+        }
+        gamma[i] = mx;
+        volatile float den = mx < eps ? eps : mx;
+        volatile float sc = 127.0f / den;
+        scale[i] = sc;
+        for (long j = 0; j < per_sample; ++j) {
+            volatile float prod = xi[j] * sc;
+            float r = nearbyintf(prod);                     /* ties to even */
+            if (r > 127.0f) r = 127.0f;
+            if (r < -128.0f) r = -128.0f;
+            q[(long)i * per_sample + j] = (int8_t)r;
+        }
+    }
+}

@@ -58,6 +58,8 @@ def lib():
             C.c_int, C.c_int, i8p, C.c_int, C.c_int, C.c_int, i8p]
         L.prom_ref_quantize_ternary.argtypes = [C.POINTER(C.c_float), C.c_int, C.c_int, C.c_double,
                                                 i8p, C.POINTER(C.c_double)]
+        L.prom_ref_quantize_act_absmax.argtypes = [C.POINTER(C.c_float), C.c_int, C.c_long, C.c_float,
+                                                   i8p, C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.prom_ref_requant_from_scale.restype = C.c_int
         L.prom_ref_requant_from_scale.argtypes = [C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_int)]
         _lib = L
@@ -210,3 +212,18 @@ def requant_from_scale(scale: float):
     if lib().prom_ref_requant_from_scale(float(scale), C.byref(m), C.byref(s)) != 0:
         raise ValueError("scale cannot be represented with a shift in [0, 31]")
     return int(m.value), int(s.value)
+
+
+def quantize_act_absmax(x, eps: float = 1e-5):
+    """Per-sample absmax quantiser of activations (paper Eq. 6-7 / the activation figure of
+    the pseudocode appendix).  x: float32 [batch, ...].  Returns (q int8 like x,
+    gamma float32 [batch] = max |x| per sample, scale float32 [batch] = 127 / max(gamma, eps))."""
+    x = _c(x, np.float32)
+    batch = x.shape[0]
+    per = int(np.prod(x.shape[1:])) if x.ndim > 1 else 1
+    q = np.empty(x.shape, dtype=np.int8)
+    gamma = np.empty((batch,), dtype=np.float32)
+    scale = np.empty((batch,), dtype=np.float32)
+    lib().prom_ref_quantize_act_absmax(_p(x, C.c_float), batch, C.c_long(per), C.c_float(eps),
+                                       _p(q, C.c_int8), _p(gamma, C.c_float), _p(scale, C.c_float))
+    return q, gamma, scale
