@@ -126,6 +126,26 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin,
                                   uint8_t *packed_dev, size_t packed_bytes,
                                   float *alpha_dev, void *cuda_stream);
 
+/* Per-sample absmax quantisation of float activations to int8: paper, Section 3.1
+ * ("Activations", Eq. 6-7) and the activation figure of the pseudocode appendix.  For each of
+ * the `batch` samples, over all `per_sample` values of the sample (any layout inside it),
+ *     gamma = max |x|,  scale = 127 / max(gamma, 1e-5),  q = clip(round(x * scale), -128, 127),
+ * round = ties to even.  The quotient and the product are single correctly rounded binary32
+ * operations, so q, gamma and scale are reproducible bit for bit.  Non-finite inputs are not
+ * supported (NaNs are ignored by the maximum and give an unspecified code).
+ *   x_dev      [batch][per_sample] float32, device, 16-byte aligned
+ *   q_dev      [batch][per_sample] int8, device, 16-byte aligned
+ *   gamma_dev, scale_dev  [batch] float32, device (Eq. 6's gamma and the factor applied)
+ * Asynchronous on the stream.  When per_sample is a multiple of 16 and a sample fits the
+ * shared memory of up to 8 SMs (per_sample <= about 450 000), each value is read from HBM
+ * once by a thread-block cluster per sample; otherwise two passes read it twice.
+ * Errors: PROM_ERR_NULL, PROM_ERR_SHAPE (batch < 0, per_sample < 1, batch > 65535 on the
+ * two-pass route), PROM_ERR_ALIGN, PROM_ERR_CUDA; a copy that does not land within 0.1 s sets
+ * PROM_ERR_TIMEOUT in prom_last_device_status.  batch == 0 is a no-op. */
+prom_status prom_quantize_act_absmax(const float *x_dev, int batch, int64_t per_sample,
+                                     int8_t *q_dev, float *gamma_dev, float *scale_dev,
+                                     void *cuda_stream);
+
 /* Host helper: the fixed-point pair for a real per-channel scale (alpha_i times
  * the activation scales and whatever BatchNorm folds in; Figure 12 divides by
  * these in floating point): mult in [2^30, 2^31) and shift in [0, 31] with

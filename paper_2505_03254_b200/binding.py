@@ -28,7 +28,7 @@ EXPORTS = [
     "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
     "prom_launch_count", "prom_shutdown", "prom_status_string",
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
-    "prom_quantize_ternary", "prom_requant_from_scale",
+    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -84,6 +84,9 @@ def lib():
         L.prom_pw_conv_i8_addsub_static.restype = i32
         L.prom_pw_conv_i8_addsub_static.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant),
                                                     vp, vp]
+        L.prom_quantize_act_absmax.restype = i32
+        L.prom_quantize_act_absmax.argtypes = [C.c_void_p, i32, i64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                               C.c_void_p]
         L.prom_debug_tc_plan.restype = None
         L.prom_debug_tc_plan.argtypes = [i32, i32, i32, i32, i32]
         L.prom_debug_tc_plan_query.restype = i32
@@ -139,6 +142,21 @@ def launch_count() -> int:
 
 def last_device_status(stream=None) -> int:
     return int(lib().prom_last_device_status(_stream(stream)))
+
+
+def quantize_act_absmax(x: torch.Tensor, stream=None):
+    """prom_quantize_act_absmax: float32 activations [batch, ...] on the device -> (q int8 like
+    x, gamma float32 [batch], scale float32 [batch])."""
+    if not x.is_cuda or x.dtype != torch.float32 or not x.is_contiguous():
+        raise ValueError("x must be a contiguous float32 CUDA tensor")
+    batch = x.shape[0]
+    per = x.numel() // batch if batch else 1
+    q = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+    gamma = torch.empty((batch,), dtype=torch.float32, device=x.device)
+    scale = torch.empty((batch,), dtype=torch.float32, device=x.device)
+    _check(lib().prom_quantize_act_absmax(x.data_ptr(), batch, per, q.data_ptr(), gamma.data_ptr(),
+                                          scale.data_ptr(), _stream(stream)), "prom_quantize_act_absmax")
+    return q, gamma, scale
 
 
 def debug_tc_plan(fold: int = 0, nt: int = 0, groups: int = 0, occ: int = 0, stages: int = 0) -> None:

@@ -20,6 +20,7 @@
 #include "tc.cuh"
 #include "smallk.cuh"
 #include "addsub.cuh"
+#include "actquant.cuh"
 #include "quantize.cuh"
 
 namespace prom {
@@ -705,6 +706,71 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin, uint8_t
     const int grid = cout < d.sms * 8 ? cout : d.sms * 8;
     quant::quantize_ternary_kernel<<<grid, quant::kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         w_dev, cout, cin, 1e-5, packed_dev, alpha_dev);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+prom_status prom_quantize_act_absmax(const float *x_dev, int batch, int64_t per_sample,
+                                     int8_t *q_dev, float *gamma_dev, float *scale_dev,
+                                     void *cuda_stream)
+{
+    if (batch < 0 || per_sample < 1 || per_sample > (1ll << 40)) return PROM_ERR_SHAPE;
+    if (batch == 0) return PROM_OK;
+    if (!x_dev || !q_dev || !gamma_dev || !scale_dev) return PROM_ERR_NULL;
+    if (!aligned16(x_dev) || !aligned16(q_dev)) return PROM_ERR_ALIGN;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const float eps = 1e-5f;
+
+    // fused route: the smallest cluster whose slices fit shared memory
+    const size_t room = (size_t)d.smem_optin - 4096;
+    int cluster = 0, slice = 0;
+    if (per_sample % 16 == 0) {
+        for (int c = 1; c <= actq::kMaxCluster; c *= 2) {
+            const long long s = ((per_sample + c - 1) / c + 15) / 16 * 16;
+            if ((size_t)s * 4 <= room) { cluster = c; slice = (int)s; break; }
+        }
+    }
+    if (cluster) {
+        static std::once_flag once;
+        static cudaError_t attr_err = cudaSuccess;
+        std::call_once(once, [&] {
+            attr_err = cudaFuncSetAttribute(actq::act_quant_cluster_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin - 4096);
+        });
+        if (attr_err != cudaSuccess) return cuda_status(attr_err);
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3((unsigned)((long long)batch * cluster));
+        cfg.blockDim = dim3(actq::kThreads);
+        cfg.dynamicSmemBytes = (size_t)slice * 4;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cluster;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, actq::act_quant_cluster_kernel, x_dev,
+                                           (long long)per_sample, slice, eps, q_dev, gamma_dev, scale_dev);
+        ++g_launches;
+        return cuda_status(e);
+    }
+
+    // two passes
+    if (cudaMemsetAsync(gamma_dev, 0, sizeof(float) * (size_t)batch, st) != cudaSuccess) return PROM_ERR_CUDA;
+    long long bx = (per_sample + actq::kThreads * 8 - 1) / (actq::kThreads * 8);
+    const long long cap = (long long)d.sms * 8 / batch + 1;
+    if (bx > cap) bx = cap;
+    if (bx < 1) bx = 1;
+    const dim3 grid((unsigned)bx, (unsigned)batch);
+    if (batch > 65535) return PROM_ERR_SHAPE;
+    actq::act_absmax_kernel<<<grid, actq::kThreads, 0, st>>>(x_dev, (long long)per_sample, gamma_dev);
+    ++g_launches;
+    actq::act_quant_kernel<<<grid, actq::kThreads, 0, st>>>(x_dev, (long long)per_sample, eps, gamma_dev, q_dev,
+                                                            scale_dev);
     ++g_launches;
     return cuda_status(cudaGetLastError());
 }
