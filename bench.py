@@ -431,6 +431,7 @@ def run_gpu(args):
         out["layers"] = per_layer_detail(torch, binding, synth, table, dev, seed, bw, p_i8, variant)
         out["single_layer"] = single_layer_configs(torch, binding, synth, bw, p_i8)
         out["quantizer"] = quantizer_timing(torch, binding, table, bw)
+        out["act_quantizer"] = act_quantizer_timing(torch, binding, bw)
         cold_us = sum(r["us"] for r in out["layers"])
         roofline["sum_layer_cold_us"] = cold_us
         roofline["sum_layer_cold_frac"] = sum(roof_us) / cold_us
@@ -495,6 +496,25 @@ def quantizer_timing(torch, binding, table, bw):
             "us": round(med, 2), "us_min": round(mn, 2), "bytes": nbytes,
             "gbs": round(nbytes / med / 1e3, 1), "roof_us": round(nbytes / bw * 1e6, 2),
             "frac": round(nbytes / bw * 1e6 / med, 4)}
+
+
+def act_quantizer_timing(torch, binding, bw):
+    """The step after the path in the paper's dataflow (off the timed step): per-sample absmax
+    quantisation of a float32 activation tensor of the first layer's input shape
+    [128,112,112,32] (205 MB > L2) to int8.  Algorithmic bytes: 4 read + 1 written per value."""
+    g = torch.Generator(device="cuda").manual_seed(2)
+    x = torch.randn((BATCH, 112, 112, 32), generator=g, device="cuda")
+    out = (torch.empty(x.shape, dtype=torch.int8, device="cuda"),
+           torch.empty((BATCH,), dtype=torch.float32, device="cuda"),
+           torch.empty((BATCH,), dtype=torch.float32, device="cuda"))
+    fn = lambda: binding.quantize_act_absmax(x, out=out)
+    for _ in range(3):
+        fn()
+    ms = time_region(torch, fn, 20, False) / 20
+    nbytes = 5 * x.numel() + 8 * BATCH
+    return {"workload": "float32 [128,112,112,32] -> int8 + per-sample gamma and scale, one launch",
+            "us": round(ms * 1e3, 2), "bytes": nbytes, "gbs": round(nbytes / ms / 1e6, 1),
+            "roof_us": round(nbytes / bw * 1e6, 2), "frac": round(nbytes / bw * 1e3 / ms, 4)}
 
 
 def single_layer_configs(torch, binding, synth, bw, p_i8):

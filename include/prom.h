@@ -136,9 +136,11 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin,
  *   x_dev      [batch][per_sample] float32, device, 16-byte aligned
  *   q_dev      [batch][per_sample] int8, device, 16-byte aligned
  *   gamma_dev, scale_dev  [batch] float32, device (Eq. 6's gamma and the factor applied)
- * Asynchronous on the stream.  When per_sample is a multiple of 16 and a sample fits the
- * shared memory of up to 8 SMs (per_sample <= about 450 000), each value is read from HBM
- * once by a thread-block cluster per sample; otherwise two passes read it twice.
+ * Asynchronous on the stream.  When per_sample is a multiple of 16 a thread-block cluster of
+ * up to 8 CTAs works on each sample and exchanges the maxima through distributed shared
+ * memory: if the sample fits the shared memory of 8 SMs (per_sample <= about 450 000) it is
+ * staged there and read from HBM once, larger samples are read twice (the second time from L2
+ * while it still holds them).  Other sizes take two kernels and read every value twice.
  * Errors: PROM_ERR_NULL, PROM_ERR_SHAPE (batch < 0, per_sample < 1, batch > 65535 on the
  * two-pass route), PROM_ERR_ALIGN, PROM_ERR_CUDA; a copy that does not land within 0.1 s sets
  * PROM_ERR_TIMEOUT in prom_last_device_status.  batch == 0 is a no-op. */

@@ -144,16 +144,22 @@ def last_device_status(stream=None) -> int:
     return int(lib().prom_last_device_status(_stream(stream)))
 
 
-def quantize_act_absmax(x: torch.Tensor, stream=None):
+def quantize_act_absmax(x: torch.Tensor, out=None, stream=None):
     """prom_quantize_act_absmax: float32 activations [batch, ...] on the device -> (q int8 like
-    x, gamma float32 [batch], scale float32 [batch])."""
+    x, gamma float32 [batch], scale float32 [batch]); `out` may carry the three tensors."""
     if not x.is_cuda or x.dtype != torch.float32 or not x.is_contiguous():
         raise ValueError("x must be a contiguous float32 CUDA tensor")
     batch = x.shape[0]
     per = x.numel() // batch if batch else 1
-    q = torch.empty(x.shape, dtype=torch.int8, device=x.device)
-    gamma = torch.empty((batch,), dtype=torch.float32, device=x.device)
-    scale = torch.empty((batch,), dtype=torch.float32, device=x.device)
+    if out is None:
+        q = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+        gamma = torch.empty((batch,), dtype=torch.float32, device=x.device)
+        scale = torch.empty((batch,), dtype=torch.float32, device=x.device)
+    else:
+        q, gamma, scale = out
+        if q.shape != x.shape or q.dtype != torch.int8 or not q.is_cuda or gamma.numel() != batch or \
+                scale.numel() != batch or gamma.dtype != torch.float32 or scale.dtype != torch.float32:
+            raise ValueError("out must be (int8 like x, float32 [batch], float32 [batch]) on the device")
     _check(lib().prom_quantize_act_absmax(x.data_ptr(), batch, per, q.data_ptr(), gamma.data_ptr(),
                                           scale.data_ptr(), _stream(stream)), "prom_quantize_act_absmax")
     return q, gamma, scale

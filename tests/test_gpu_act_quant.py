@@ -1,6 +1,7 @@
 """GPU parity of prom_quantize_act_absmax (paper Eq. 6-7) with the CPU oracle: codes, gamma
 and scale bit for bit (both sides take the decision in binary32 with the same two correctly
-rounded operations), on the fused cluster route and the two-pass route, ragged sizes included."""
+rounded operations), on the staged cluster route, the re-reading cluster route and the
+two-kernel route, ragged sizes included."""
 import numpy as np
 import pytest
 import torch
@@ -47,12 +48,13 @@ def test_fused_route(oracle, shape):
 
 
 @pytest.mark.parametrize("shape", [
-    (5, 7),                    # not a multiple of 16: two-pass route
+    (5, 7),                    # not a multiple of 16: two kernels (maxima, then codes)
     (3, 1001),
     (2, 7, 7, 1280 + 8),
-    (2, 160, 160, 24),         # 614 400 per sample: too large for a cluster's shared memory
+    (2, 160, 160, 24),         # 614 400 per sample: too large for a cluster's shared memory,
+    (3, 224, 224, 16),         # 802 816: the clusters read their slices twice instead
 ])
-def test_two_pass_route(oracle, shape):
+def test_other_routes(oracle, shape):
     _check(oracle, _input(12, shape))
 
 
