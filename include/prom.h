@@ -271,7 +271,8 @@ uint64_t prom_launch_count(void);
  * thread-safe.  prom_debug_tc_plan_query writes the plan the library would
  * use for a plain [m][cin] x [cout] layer ({fold, nt, groups, grid, stages,
  * accumulators, shared bytes, chunk bytes, estimate in 1/100 us}) and returns
- * 1, or returns 0 if TC cannot run it. */
+ * 1, or returns 0 if TC cannot run it.  Without a CUDA device it plans for a
+ * B200's nominal limits (148 SMs, 227 KB of shared memory per CTA). */
 void prom_debug_tc_plan(int fold, int nt, int groups, int occ, int stages);
 int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
 
