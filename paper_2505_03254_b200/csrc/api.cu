@@ -754,10 +754,26 @@ prom_status prom_quantize_act_absmax(const float *x_dev, int batch, int64_t per_
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         // as many clusters as are resident at once, each walking over its share of the samples
+        // (asked once per shape: the query costs tens of microseconds on the host)
+        static std::mutex mu;
+        static std::map<std::array<long long, 3>, int> known;
+        int dev = 0;
+        cudaGetDevice(&dev);
         int resident = 0;
-        if (cudaOccupancyMaxActiveClusters(&resident, actq::act_quant_cluster_kernel, &cfg) != cudaSuccess)
-            resident = 0;
-        cudaGetLastError();
+        {
+            std::lock_guard<std::mutex> lk(mu);
+            const std::array<long long, 3> key = {dev, cluster, slice};
+            auto it = known.find(key);
+            if (it == known.end()) {
+                if (cudaOccupancyMaxActiveClusters(&resident, actq::act_quant_cluster_kernel, &cfg) !=
+                    cudaSuccess)
+                    resident = 0;
+                cudaGetLastError();
+                known[key] = resident;
+            } else {
+                resident = it->second;
+            }
+        }
         if (resident > 0) {
             const int nclusters = resident < batch ? resident : batch;
             cfg.gridDim = dim3((unsigned)(nclusters * cluster));
@@ -787,10 +803,24 @@ prom_status prom_quantize_act_absmax(const float *x_dev, int batch, int64_t per_
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
+        static std::mutex mu;
+        static std::map<int, int> known;
+        int dev = 0;
+        cudaGetDevice(&dev);
         int resident = 0;
-        if (cudaOccupancyMaxActiveClusters(&resident, actq::act_quant_reread_kernel, &cfg) != cudaSuccess)
-            resident = 0;
-        cudaGetLastError();
+        {
+            std::lock_guard<std::mutex> lk(mu);
+            auto it = known.find(dev);
+            if (it == known.end()) {
+                if (cudaOccupancyMaxActiveClusters(&resident, actq::act_quant_reread_kernel, &cfg) !=
+                    cudaSuccess)
+                    resident = 0;
+                cudaGetLastError();
+                known[dev] = resident;
+            } else {
+                resident = it->second;
+            }
+        }
         if (resident > 0 && s * 4 <= (8ll << 20)) {
             const int nclusters = resident < batch ? resident : batch;
             cfg.gridDim = dim3((unsigned)(nclusters * c));
