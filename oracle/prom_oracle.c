@@ -368,3 +368,63 @@ void prom_ref_quantize_act_absmax(const float *x, int batch, long per_sample, fl
         }
     }
 }
+
+/*
+ * A pointwise layer in the paper's own inference dataflow (pseudocode appendix, the
+ * inference branch of the quantised convolution module, followed by the activation
+ * quantiser of the next module; Section 3.1, Eq. 6-7):
+ *     acc[m][o] = sum_k X-hat[m][k] * W-hat[o][k]                  (integers, exact)
+ *     y[m][o]   = acc[m][o] * alpha[o] * dq[b(m)]                  (dequantise)
+ *     gamma_y[b] = max_{m in sample b, o} |y[m][o]|
+ *     q[m][o]   = clip(round(y[m][o] * 127 / max(gamma_y[b], eps)), -128, 127)
+ * where X-hat was produced by the activation quantiser with per-sample maximum gamma_x[b],
+ * dq[b] = max(gamma_x[b], eps) / 127 is the reciprocal of its scale, and sample b owns rows
+ * [b * rows_per_sample, (b + 1) * rows_per_sample).
+ * Readings: the module divides by the weight scale (1 / alpha) and by the activation scale;
+ * here the result is multiplied by alpha and by dq, the same real numbers, so that each step
+ * is one binary32 rounding of a product; BatchNorm and PReLU, separate float modules in the
+ * paper, are not part of this function.  All float steps are single correctly rounded
+ * binary32 operations in the order written (volatile stops the compiler from fusing or
+ * widening), so that a second implementation with the same steps agrees bit for bit.
+ * y (optional): [m][cout] float32; q: [m][cout] int8; gamma_y, scale_y: [batch].
+ */
+void prom_ref_conv_dyn(const int8_t *x, int batch, long rows_per_sample, int cin,
+                       const int8_t *w, int cout, const float *alpha, const float *gamma_x,
+                       float eps, float *y_out, int8_t *q, float *gamma_y, float *scale_y)
+{
+    long m = (long)batch * rows_per_sample;
+    float *y = (float *)malloc(sizeof(float) * (size_t)m * (size_t)cout);
+    for (int b = 0; b < batch; ++b) {
+        volatile float gx = gamma_x[b] < eps ? eps : gamma_x[b];
+        volatile float dq = gx / 127.0f;
+        float mx = 0.0f;
+        for (long r = b * rows_per_sample; r < (b + 1) * rows_per_sample; ++r) {
+            for (int o = 0; o < cout; ++o) {
+                int32_t acc = 0;
+                for (int k = 0; k < cin; ++k)
+                    acc += (int32_t)x[r * cin + k] * (int32_t)w[(long)o * cin + k];
+                volatile float t = (float)acc;          /* exact: |acc| < 2^24 */
+                volatile float u = t * alpha[o];
+                volatile float v = u * dq;
+                y[r * cout + o] = v;
+                float a = fabsf(v);
+                if (a > mx) mx = a;
+            }
+        }
+        gamma_y[b] = mx;
+        volatile float den = mx < eps ? eps : mx;
+        volatile float sc = 127.0f / den;
+        scale_y[b] = sc;
+        for (long r = b * rows_per_sample; r < (b + 1) * rows_per_sample; ++r) {
+            for (int o = 0; o < cout; ++o) {
+                volatile float prod = y[r * cout + o] * sc;
+                float rr = nearbyintf(prod);
+                if (rr > 127.0f) rr = 127.0f;
+                if (rr < -128.0f) rr = -128.0f;
+                q[r * cout + o] = (int8_t)rr;
+            }
+        }
+    }
+    if (y_out) memcpy(y_out, y, sizeof(float) * (size_t)m * (size_t)cout);
+    free(y);
+}

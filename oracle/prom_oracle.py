@@ -60,6 +60,10 @@ def lib():
                                                 i8p, C.POINTER(C.c_double)]
         L.prom_ref_quantize_act_absmax.argtypes = [C.POINTER(C.c_float), C.c_int, C.c_long, C.c_float,
                                                    i8p, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+        L.prom_ref_conv_dyn.argtypes = [i8p, C.c_int, C.c_long, C.c_int, i8p, C.c_int,
+                                        C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_float,
+                                        C.POINTER(C.c_float), i8p, C.POINTER(C.c_float),
+                                        C.POINTER(C.c_float)]
         L.prom_ref_requant_from_scale.restype = C.c_int
         L.prom_ref_requant_from_scale.argtypes = [C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_int)]
         _lib = L
@@ -227,3 +231,25 @@ def quantize_act_absmax(x, eps: float = 1e-5):
     lib().prom_ref_quantize_act_absmax(_p(x, C.c_float), batch, C.c_long(per), C.c_float(eps),
                                        _p(q, C.c_int8), _p(gamma, C.c_float), _p(scale, C.c_float))
     return q, gamma, scale
+
+
+def conv_dyn(x, w, alpha, gamma_x, rows_per_sample: int, eps: float = 1e-5):
+    """A pointwise layer in the paper's inference dataflow: ternary convolution of quantised
+    activations, dequantised by alpha[o] and the input's per-sample scale, then quantised again
+    per sample.  x: int8 [batch * rows_per_sample, cin]; w: int8 [cout, cin] ternary; alpha:
+    float32 [cout]; gamma_x: float32 [batch].  Returns (q int8 [m, cout], gamma_y, scale_y
+    float32 [batch], y float32 [m, cout])."""
+    x = _c(x, np.int8); w = _c(w, np.int8)
+    alpha = _c(alpha, np.float32); gamma_x = _c(gamma_x, np.float32)
+    m, cin = x.shape
+    cout = w.shape[0]
+    batch = gamma_x.shape[0]
+    assert m == batch * rows_per_sample and w.shape[1] == cin and alpha.shape[0] == cout
+    y = np.empty((m, cout), dtype=np.float32)
+    q = np.empty((m, cout), dtype=np.int8)
+    gy = np.empty((batch,), dtype=np.float32)
+    sy = np.empty((batch,), dtype=np.float32)
+    lib().prom_ref_conv_dyn(_p(x, C.c_int8), batch, C.c_long(rows_per_sample), cin, _p(w, C.c_int8), cout,
+                            _p(alpha, C.c_float), _p(gamma_x, C.c_float), C.c_float(eps),
+                            _p(y, C.c_float), _p(q, C.c_int8), _p(gy, C.c_float), _p(sy, C.c_float))
+    return q, gy, sy, y
