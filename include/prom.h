@@ -126,6 +126,34 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin,
                                   uint8_t *packed_dev, size_t packed_bytes,
                                   float *alpha_dev, void *cuda_stream);
 
+/* A pointwise layer in the paper's own inference dataflow: pseudocode appendix, inference
+ * branch of the quantised convolution module ("perform convolution in low bit-width, dequantise
+ * after convolution"), followed by the activation quantiser of the next module (Section 3.1,
+ * Eq. 6-7).  With b(m) = m / rows_per_sample the sample of row m,
+ *     acc[m][o] = sum_k x[m][k] * W-hat[o][k]                        exact integers
+ *     y[m][o]   = acc[m][o] * alpha[o] * (max(gamma_x[b], 1e-5) / 127)  dequantised output
+ *     gamma_y[b] = max |y| over the sample,  scale_y[b] = 127 / max(gamma_y[b], 1e-5)
+ *     q[m][o]   = clip(round(y[m][o] * scale_y[b]), -128, 127)        ties to even
+ * Every float step is one correctly rounded binary32 operation in the order written, so the
+ * outputs are reproducible bit for bit.  y itself is never written: the tensor cores run the
+ * convolution twice (first pass: maxima, second pass: codes), which costs a second read of x
+ * instead of writing and re-reading four bytes per output.
+ *   x_dev        [batch * rows_per_sample][cin] int8, device, 16-byte aligned (the activation
+ *                quantiser's output; gamma_x_dev [batch] are the maxima it reported)
+ *   w_packed_dev packed ternary weights (prom_pack_ternary / prom_quantize_ternary)
+ *   alpha_dev    [cout] float32 > 0, the weight scales (prom_quantize_ternary's alpha), times
+ *                whatever per-channel factor the caller folds in
+ *   q_dev        [batch * rows_per_sample][cout] int8, device, 16-byte aligned, not x_dev
+ *   gamma_y_dev, scale_y_dev  [batch] float32 outputs
+ * Tensor-core variant only: cin a multiple of 16, cout a multiple of 8 (of 16 above 256), else
+ * PROM_ERR_UNSUPPORTED.  Asynchronous on the stream (one memset, three launches).  Other errors
+ * as for prom_pw_conv_i8; weights outside {-1,0,+1} surface as PROM_ERR_BAD_WEIGHT in
+ * prom_last_device_status. */
+prom_status prom_pw_conv_i8_dyn(const int8_t *x_dev, int batch, int64_t rows_per_sample, int cin,
+                                const uint8_t *w_packed_dev, int cout, const float *alpha_dev,
+                                const float *gamma_x_dev, int8_t *q_dev, float *gamma_y_dev,
+                                float *scale_y_dev, void *cuda_stream);
+
 /* Per-sample absmax quantisation of float activations to int8: paper, Section 3.1
  * ("Activations", Eq. 6-7) and the activation figure of the pseudocode appendix.  For each of
  * the `batch` samples, over all `per_sample` values of the sample (any layout inside it),

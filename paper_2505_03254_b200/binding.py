@@ -28,7 +28,7 @@ EXPORTS = [
     "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
     "prom_launch_count", "prom_shutdown", "prom_status_string",
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
-    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax",
+    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -84,6 +84,9 @@ def lib():
         L.prom_pw_conv_i8_addsub_static.restype = i32
         L.prom_pw_conv_i8_addsub_static.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant),
                                                     vp, vp]
+        L.prom_pw_conv_i8_dyn.restype = i32
+        L.prom_pw_conv_i8_dyn.argtypes = [C.c_void_p, i32, i64, i32, C.c_void_p, i32, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.prom_quantize_act_absmax.restype = i32
         L.prom_quantize_act_absmax.argtypes = [C.c_void_p, i32, i64, C.c_void_p, C.c_void_p, C.c_void_p,
                                                C.c_void_p]
@@ -142,6 +145,28 @@ def launch_count() -> int:
 
 def last_device_status(stream=None) -> int:
     return int(lib().prom_last_device_status(_stream(stream)))
+
+
+def pw_conv_i8_dyn(x: torch.Tensor, batch: int, w_packed: torch.Tensor, cout: int, alpha: torch.Tensor,
+                   gamma_x: torch.Tensor, out=None, stream=None):
+    """prom_pw_conv_i8_dyn: x int8 [batch * rows_per_sample, cin], alpha float32 [cout], gamma_x
+    float32 [batch], all on the device -> (q int8 [m, cout], gamma_y, scale_y float32 [batch])."""
+    m, cin = x.shape
+    if batch and m % batch:
+        raise ValueError("rows must divide evenly into samples")
+    rows = m // batch if batch else 1
+    if out is None:
+        q = torch.empty((m, cout), dtype=torch.int8, device=x.device)
+        gy = torch.empty((batch,), dtype=torch.float32, device=x.device)
+        sy = torch.empty((batch,), dtype=torch.float32, device=x.device)
+    else:
+        q, gy, sy = out
+    _check(lib().prom_pw_conv_i8_dyn(_dev(x, torch.int8, "x"), batch, rows, cin,
+                                     _dev(w_packed, torch.uint8, "w_packed"), cout,
+                                     _dev(alpha, torch.float32, "alpha"), _dev(gamma_x, torch.float32, "gamma_x"),
+                                     q.data_ptr(), gy.data_ptr(), sy.data_ptr(), _stream(stream)),
+           "prom_pw_conv_i8_dyn")
+    return q, gy, sy
 
 
 def quantize_act_absmax(x: torch.Tensor, out=None, stream=None):

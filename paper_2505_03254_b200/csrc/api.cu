@@ -292,8 +292,10 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
 
 // Picks fold, subtile width, channel groups and occupancy.  Returns false when
 // the tensor-core variant cannot run this shape.
+// dyn: the plan serves the dynamic layer (no row folding: a folded row could straddle two
+// samples; two CTAs per SM)
 static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
-                           TcPlan &best)
+                           bool dyn, TcPlan &best)
 {
     if (m <= 0 || (cin & 7) || (cout & 7)) return false;
     int fold = 1;
@@ -303,6 +305,10 @@ static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, co
         while (fold * 2 <= 8 && fold * 2 * cin <= 128 && fold * 2 * cout <= 128 &&
                m % (fold * 2) == 0)
             fold *= 2;
+    }
+    if (dyn) {
+        if ((cin & 15) || ((cout & 15) && cout > 256)) return false;
+        fold = 1;
     }
     if (g_tune.fold > 0) fold = g_tune.fold;
     if (fold < 1 || fold > 8 || m % fold) return false;
@@ -317,6 +323,7 @@ static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, co
             if (g_tune.groups > 0 && groups != g_tune.groups) continue;
             for (int occ = 4; occ >= 1; --occ) {
                 if (g_tune.occ > 0 && occ != g_tune.occ) continue;
+                if (dyn && occ != 2) continue;
                 if (g_tune.occ == 0 && occ >= 3) continue;      // only on request for now
                 TcPlan pl;
                 if (!tc_fill_plan(m, cin, cout, map, d, fold, nt, groups, occ, g_tune.stages, pl))
@@ -332,21 +339,21 @@ static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, co
 // The search above costs tens of microseconds; its result depends only on the shape, the
 // device and the tuning override, so it is remembered.
 static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
-                          TcPlan &best)
+                          TcPlan &best, bool dyn = false)
 {
     struct Entry { bool ok; TcPlan pl; };
     static std::mutex mu;
-    static std::map<std::array<long long, 14>, Entry> cache;
+    static std::map<std::array<long long, 15>, Entry> cache;
     int dev = 0;
     cudaGetDevice(&dev);
-    const std::array<long long, 14> key = {m, cin, cout, map.stride, map.ho, map.wo, map.hin, map.win,
+    const std::array<long long, 15> key = {m, cin, cout, map.stride, map.ho, map.wo, map.hin, map.win,
                                            g_tune.fold, g_tune.nt, g_tune.groups, g_tune.occ,
-                                           g_tune.stages, dev};
+                                           g_tune.stages, dev, dyn ? 1 : 0};
     std::lock_guard<std::mutex> lk(mu);
     auto it = cache.find(key);
     if (it == cache.end()) {
         Entry e;
-        e.ok = tc_search_plan(m, cin, cout, map, d, e.pl);
+        e.ok = tc_search_plan(m, cin, cout, map, d, dyn, e.pl);
         if (cache.size() > 4096) cache.clear();
         it = cache.emplace(key, e).first;
     }
@@ -410,6 +417,14 @@ static prom_status tc_set_attr(const DeviceInfo &d)
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             d.smem_optin);
         if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 1>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            d.smem_optin);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 2>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            d.smem_optin);
+        if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(tc::tc_prep_kernel,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             d.smem_optin);
@@ -427,7 +442,7 @@ static void tc_bind(const Conv &c, TcPlan &pl, uint8_t *image)
     p.image = image;
 }
 
-static prom_status tc_launch_planned(const Conv &c, TcPlan &pl)
+static prom_status tc_launch_planned(const Conv &c, TcPlan &pl, int mode = 0)
 {
     if (!tc_make_maps(c, pl)) return PROM_ERR_CUDA;
     cudaLaunchConfig_t cfg;
@@ -443,9 +458,11 @@ static prom_status tc_launch_planned(const Conv &c, TcPlan &pl)
         cfg.attrs = attr;
         cfg.numAttrs = 1;
     }
-    cudaError_t e = pl.per_sm == 3
-                        ? cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<3>, pl.xmap, pl.ymap, pl.p)
-                        : cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2>, pl.xmap, pl.ymap, pl.p);
+    cudaError_t e;
+    if (mode == 1) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 1>, pl.xmap, pl.ymap, pl.p);
+    else if (mode == 2) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 2>, pl.xmap, pl.ymap, pl.p);
+    else if (pl.per_sm == 3) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<3>, pl.xmap, pl.ymap, pl.p);
+    else e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2>, pl.xmap, pl.ymap, pl.p);
     ++g_launches;
     return cuda_status(e);
 }
@@ -658,6 +675,17 @@ static uint8_t *static_scratch_address()
     return static_cast<uint8_t *>(p);
 }
 
+// scale_y[b] = 127 / max(gamma_y[b], eps): between the two passes of the dynamic layer
+__global__ void dyn_scale_kernel(const float *__restrict__ gamma_y, int batch, float eps,
+                                        float *__restrict__ scale_y)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < batch) {
+        const float g = gamma_y[b];
+        scale_y[b] = __fdiv_rn(127.0f, g < eps ? eps : g);
+    }
+}
+
 }  // namespace prom
 
 using namespace prom;
@@ -708,6 +736,51 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin, uint8_t
         w_dev, cout, cin, 1e-5, packed_dev, alpha_dev);
     ++g_launches;
     return cuda_status(cudaGetLastError());
+}
+
+prom_status prom_pw_conv_i8_dyn(const int8_t *x_dev, int batch, int64_t rows_per_sample, int cin,
+                                const uint8_t *w_packed_dev, int cout, const float *alpha_dev,
+                                const float *gamma_x_dev, int8_t *q_dev, float *gamma_y_dev,
+                                float *scale_y_dev, void *cuda_stream)
+{
+    if (batch < 0 || rows_per_sample < 1 || cin < 1 || cout < 1 || cin > 4096 || cout > 4096)
+        return PROM_ERR_SHAPE;
+    const long long m = (long long)batch * rows_per_sample;
+    if (rows_per_sample >= (1ll << 31) || m >= (1ll << 31)) return PROM_ERR_SHAPE;
+    if (batch == 0) return PROM_OK;
+    if (!x_dev || !w_packed_dev || !alpha_dev || !gamma_x_dev || !q_dev || !gamma_y_dev || !scale_y_dev)
+        return PROM_ERR_NULL;
+    if (!aligned16(x_dev) || !aligned16(w_packed_dev) || !aligned16(q_dev)) return PROM_ERR_ALIGN;
+    if (reinterpret_cast<const void *>(x_dev) == reinterpret_cast<const void *>(q_dev)) return PROM_ERR_ALIGN;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    TcPlan pl;
+    const RowMap plain{1, 1, 1, 1, 1};
+    if (!tc_shape_plan(m, cin, cout, plain, d, pl, true)) return PROM_ERR_UNSUPPORTED;
+    if (tc_set_attr(d) != PROM_OK) return PROM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    Conv c;
+    memset(&c, 0, sizeof(c));
+    c.x = x_dev; c.m = m; c.cin = cin; c.cout = cout; c.map = plain; c.in_rows = m;
+    c.w = w_packed_dev; c.y = q_dev; c.st = st; c.pdl = false; c.pdl_next = false;
+    c.rq.bias = nullptr; c.rq.shift = nullptr;
+    c.rq.mult = reinterpret_cast<const int32_t *>(alpha_dev);     // bit patterns of alpha
+    c.rq.act_min = -128; c.rq.act_max = 127;                      // keeps the weights at +-1
+    tc_bind(c, pl, nullptr);
+    pl.p.dyn = 1;
+    pl.p.rows_per_sample = (int)rows_per_sample;
+    pl.p.batch = batch;
+    pl.p.gamma_x = gamma_x_dev;
+    pl.p.gamma_y = gamma_y_dev;
+    pl.p.scale_y = scale_y_dev;
+    if (cudaMemsetAsync(gamma_y_dev, 0, sizeof(float) * (size_t)batch, st) != cudaSuccess)
+        return PROM_ERR_CUDA;
+    prom_status e = tc_launch_planned(c, pl, 1);
+    if (e != PROM_OK) return e;
+    dyn_scale_kernel<<<(batch + 127) / 128, 128, 0, st>>>(gamma_y_dev, batch, 1e-5f, scale_y_dev);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return PROM_ERR_CUDA;
+    return tc_launch_planned(c, pl, 2);
 }
 
 prom_status prom_quantize_act_absmax(const float *x_dev, int batch, int64_t per_sample,

@@ -77,6 +77,15 @@ struct Params {
     int8_t *y;
     int pdl;            // launched with programmatic dependent launch
     int pdl_next;       // the next kernel in the stream is launched that way
+    // The dynamic layer (kernel modes 1 and 2): `mult` then holds the bit patterns of the
+    // float per-channel factors alpha, bias and shift are not read, and rows belong to
+    // samples of rows_per_sample rows each.
+    int dyn;                    // 0: static requantisation
+    int rows_per_sample;
+    int batch;
+    const float *gamma_x;       // [batch] per-sample maximum behind the int8 input
+    float *gamma_y;             // [batch] mode 1: maxima of the dequantised output (as bit patterns)
+    const float *scale_y;       // [batch] mode 2: 127 / max(gamma_y, eps)
 };
 
 // Bounded wait on an mbarrier phase.  The clock is read only every 1024 polls (a
@@ -257,6 +266,99 @@ __device__ __forceinline__ void epi_exact_subtile(const Params &p, uint32_t tadd
         epi_exact<8>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, bar_release);
 }
 
+// ---- the dynamic layer's epilogues ---------------------------------------------------------
+// y = acc * alpha[column] * dq[sample]: the int32 accumulator becomes a float exactly (the
+// magic-number form holds below 2^22; |acc| <= 4096 * 127), then two correctly rounded products
+// in this order.
+__device__ __forceinline__ float dyn_value(uint32_t acc, int alpha_bits, float dq)
+{
+    const float f = __fadd_rn(__int_as_float((int)acc + 0x4B400000), -12582912.0f);
+    return __fmul_rn(__fmul_rn(f, __int_as_float(alpha_bits)), dq);
+}
+
+// NC accumulator columns of this thread's row, already in registers.
+// Mode 1: the largest |y| among them joins m.
+template <int NC>
+__device__ __forceinline__ float dyn_piece_max(const uint32_t (&v)[NC], const int *__restrict__ cm, float dq,
+                                               float m)
+{
+#pragma unroll
+    for (int e = 0; e < NC; e += 4) {
+        const int4 mu = *reinterpret_cast<const int4 *>(cm + e);
+        m = fmaxf(m, fabsf(dyn_value(v[e], mu.x, dq)));
+        m = fmaxf(m, fabsf(dyn_value(v[e + 1], mu.y, dq)));
+        m = fmaxf(m, fabsf(dyn_value(v[e + 2], mu.z, dq)));
+        m = fmaxf(m, fabsf(dyn_value(v[e + 3], mu.w, dq)));
+    }
+    return m;
+}
+
+// Mode 2: y quantised with the sample's scale (ties to even through the magic-number add,
+// saturating packs clip to [-128, 127]) and staged like the static epilogue's bytes.
+template <int NC>
+__device__ __forceinline__ void dyn_piece_quant(const uint32_t (&v)[NC], const int *__restrict__ cm, float dq,
+                                                float sc, uint8_t *dst, bool wide)
+{
+    uint32_t out[NC / 4];
+#pragma unroll
+    for (int e = 0; e < NC; e += 4) {
+        const int4 mu = *reinterpret_cast<const int4 *>(cm + e);
+        const int a4[4] = {mu.x, mu.y, mu.z, mu.w};
+        int r[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float y = dyn_value(v[e + j], a4[j], dq);
+            r[j] = __float_as_int(__fadd_rn(__fmul_rn(y, sc), 12582912.0f)) - 0x4B400000;
+        }
+        uint32_t w;
+        asm("{\n\t.reg .b32 t;\n\t"
+            "cvt.pack.sat.s8.s32.b32 t, %4, %3, 0;\n\t"
+            "cvt.pack.sat.s8.s32.b32 %0, %2, %1, t;\n\t}"
+            : "=r"(w)
+            : "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]));
+        out[e / 4] = w;
+    }
+    put_row<NC>(dst, out, wide);
+}
+
+// One subtile in chunks of CH, then 16 and 8 columns (nt is a multiple of 8).  QUANT false:
+// returns the largest |y| of the row; true: stages the codes and returns 0.
+template <int CH, bool QUANT>
+__device__ __forceinline__ float epi_dyn_subtile(const Params &p, uint32_t taddr, const int *cm, float dq,
+                                                 float sc, uint8_t *dst_row, uint32_t bar_release)
+{
+    const bool wide = (p.nt & 15) == 0;
+    const int tail = p.nt & (CH - 1);
+    float m = 0.0f;
+    int c = 0;
+    for (; c + CH <= p.nt; c += CH) {
+        uint32_t v[CH];
+        tmem_ld<CH>(taddr + c, v);
+        ptx::tmem_wait_ld();
+        if (tail == 0 && c + CH == p.nt) release_acc(bar_release);
+        if constexpr (QUANT) dyn_piece_quant<CH>(v, cm + c, dq, sc, dst_row + c, wide);
+        else m = dyn_piece_max<CH>(v, cm + c, dq, m);
+    }
+    if (CH > 16 && c + 16 <= p.nt) {
+        uint32_t v[16];
+        ptx::tmem_ld_x16(taddr + c, v);
+        ptx::tmem_wait_ld();
+        if (c + 16 == p.nt) release_acc(bar_release);
+        if constexpr (QUANT) dyn_piece_quant<16>(v, cm + c, dq, sc, dst_row + c, wide);
+        else m = dyn_piece_max<16>(v, cm + c, dq, m);
+        c += 16;
+    }
+    if (c + 8 <= p.nt) {
+        uint32_t v[8];
+        ptx::tmem_ld_x8(taddr + c, v);
+        ptx::tmem_wait_ld();
+        release_acc(bar_release);
+        if constexpr (QUANT) dyn_piece_quant<8>(v, cm + c, dq, sc, dst_row + c, wide);
+        else m = dyn_piece_max<8>(v, cm + c, dq, m);
+    }
+    return m;
+}
+
 // Where the parts of a CTA's shared memory are.
 struct View {
     uint8_t *smem;
@@ -355,7 +457,9 @@ __device__ __forceinline__ void build_image(const Params &p, const int g, const 
             const int nfold = (g + ls * p.groups) * p.nt + c;
             if (c < p.nt && nfold < p.nf) {
                 const int n = nfold % p.n0;
-                cb_[u] = __ldg(p.bias + n); cm_[u] = __ldg(p.mult + n); cs_[u] = __ldg(p.shift + n);
+                cm_[u] = __ldg(p.mult + n);
+                cb_[u] = p.dyn ? 0 : __ldg(p.bias + n);
+                cs_[u] = p.dyn ? 0 : (int)__ldg(p.shift + n);
             }
         }
     }
@@ -514,7 +618,9 @@ __device__ __forceinline__ void build_image(const Params &p, const int g, const 
 }
 
 // MINB: CTAs of this kernel that share an SM (2 with 96 registers a thread, 3 with 64).
-template <int MINB>
+// MODE 0: static fixed-point requantisation.  MODE 1 and 2: the two passes of the dynamic layer
+// (per-sample maxima of the dequantised output; output quantised with the per-sample scale).
+template <int MINB, int MODE = 0>
 __global__ void __launch_bounds__(kThreads, MINB)
 tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
                const Params p)
@@ -794,8 +900,40 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 const uint32_t taddr = t_lane + b * p.nt_pad;
                 const int *cms = cmult + ls * p.nt_pad;
                 const uint32_t bar_rel = bar_tempty + 8 * b;
-                if (fast) epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
-                else epi_exact_subtile<CH>(p, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
+                if constexpr (MODE == 0) {
+                    if (fast) epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
+                    else epi_exact_subtile<CH>(p, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
+                } else {
+                    // this thread's row and its sample (rows past the end borrow the last sample's
+                    // factors; they are neither counted nor stored)
+                    const int row = row0 + lane;
+                    int smp = row / p.rows_per_sample;
+                    smp = smp < p.batch ? smp : p.batch - 1;
+                    const float gx = __ldg(p.gamma_x + smp);
+                    const float dq = __fdiv_rn(gx < 1e-5f ? 1e-5f : gx, 127.0f);
+                    if constexpr (MODE == 1) {
+                        float mx = epi_dyn_subtile<CH, false>(p, taddr, cms, dq, 0.0f, nullptr, bar_rel);
+                        if (row >= m_rows || p.tm - q * 32 <= lane) mx = 0.0f;
+                        // one atomic per warp when its 32 rows share a sample, else one per row
+                        const int smp0 = __shfl_sync(0xFFFFFFFFu, smp, 0);
+                        if (__all_sync(0xFFFFFFFFu, smp == smp0)) {
+#pragma unroll
+                            for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, d));
+                            if (lane == 0 && mx > 0.0f)
+                                atomicMax(reinterpret_cast<unsigned int *>(p.gamma_y + smp0), __float_as_uint(mx));
+                        } else if (mx > 0.0f) {
+                            atomicMax(reinterpret_cast<unsigned int *>(p.gamma_y + smp), __float_as_uint(mx));
+                        }
+                        // nothing is stored in this pass
+                        ls += dls; row0 += drow; col += dcol;
+                        if (ls >= subs) { ls -= subs; row0 += drow_wrap; col -= p.nf; }
+                        b ^= btoggle;
+                        if (b < (uint32_t)kEpiGroups) tph ^= 1u;
+                        continue;
+                    } else {
+                        epi_dyn_subtile<CH, true>(p, taddr, cms, dq, __ldg(p.scale_y + smp), my_row, bar_rel);
+                    }
+                }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (whole_tile && row0 + 32 <= m_rows) {
