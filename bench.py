@@ -432,6 +432,7 @@ def run_gpu(args):
         out["single_layer"] = single_layer_configs(torch, binding, synth, bw, p_i8)
         out["quantizer"] = quantizer_timing(torch, binding, table, bw)
         out["act_quantizer"] = act_quantizer_timing(torch, binding, bw)
+        out["dynamic_layer"] = dynamic_layer_timing(torch, binding, synth, bw)
         cold_us = sum(r["us"] for r in out["layers"])
         roofline["sum_layer_cold_us"] = cold_us
         roofline["sum_layer_cold_frac"] = sum(roof_us) / cold_us
@@ -513,6 +514,31 @@ def act_quantizer_timing(torch, binding, bw):
     ms = time_region(torch, fn, 20, False) / 20
     nbytes = 5 * x.numel() + 8 * BATCH
     return {"workload": "float32 [128,112,112,32] -> int8 + per-sample gamma and scale, one launch",
+            "us": round(ms * 1e3, 2), "bytes": nbytes, "gbs": round(nbytes / ms / 1e6, 1),
+            "roof_us": round(nbytes / bw * 1e6, 2), "frac": round(nbytes / bw * 1e3 / ms, 4)}
+
+
+def dynamic_layer_timing(torch, binding, synth, bw):
+    """The widest layer of the step (1 605 632 x 16 -> 96, 128 samples) in the paper's dynamic
+    form (prom_pw_conv_i8_dyn: two tensor-core passes, per-sample scales), off the timed step.
+    Algorithmic bytes: the input read twice, the output written once, nothing else."""
+    batch, rows, k, n = BATCH, 112 * 112, 16, 96
+    m = batch * rows
+    x = synth.act_uniform_i8(synth.BASE_SEED + 40, (m, k), device="cuda")
+    lay = synth.make_layer(synth.BASE_SEED + 40, k, n, 0.5, device="cuda")
+    wp = binding.pack_ternary(lay["w"])
+    g = torch.Generator(device="cuda").manual_seed(3)
+    alpha = torch.rand((n,), generator=g, device="cuda") * 0.1 + 0.01
+    gx = torch.rand((batch,), generator=g, device="cuda") * 4 + 0.5
+    out = (torch.empty((m, n), dtype=torch.int8, device="cuda"),
+           torch.empty((batch,), dtype=torch.float32, device="cuda"),
+           torch.empty((batch,), dtype=torch.float32, device="cuda"))
+    fn = lambda: binding.pw_conv_i8_dyn(x, batch, wp, n, alpha, gx, out=out)
+    for _ in range(3):
+        fn()
+    ms = time_region(torch, fn, 20, False) / 20
+    nbytes = 2 * m * k + m * n
+    return {"workload": "1605632x16->96, 128 samples: convolution, dequantise, per-sample absmax, quantise",
             "us": round(ms * 1e3, 2), "bytes": nbytes, "gbs": round(nbytes / ms / 1e6, 1),
             "roof_us": round(nbytes / bw * 1e6, 2), "frac": round(nbytes / bw * 1e3 / ms, 4)}
 
