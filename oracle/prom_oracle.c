@@ -428,3 +428,45 @@ void prom_ref_conv_dyn(const int8_t *x, int batch, long rows_per_sample, int cin
     if (y_out) memcpy(y_out, y, sizeof(float) * (size_t)m * (size_t)cout);
     free(y);
 }
+
+/*
+ * The int8 depthwise 3x3 convolution that sits between the expand and the project
+ * convolution of a block (paper, Section 2: depthwise-separable block; Section 3.1: its
+ * weights are 8-bit, quantised per channel by absmax, Eq. 4-5).  Each channel is filtered
+ * on its own, with one pixel of zero padding and the block's stride:
+ *     acc[b][i][j][c] = sum_{di,dj in 0..2} x[b][i*s + di - 1][j*s + dj - 1][c] * w[c][di][dj]
+ * (pixels outside the image count as 0), output size ho = (h - 1) / s + 1, wo likewise,
+ * followed by the same fixed-point requantisation per channel as the pointwise layers
+ * (bias, mult, shift, clamp).  The padding and the size are the reference network's
+ * (3x3, padding 1), which the paper takes over unchanged; it prints neither.
+ * x: [batch][h][w][c] int8; w: [c][3][3] int8; y: [batch][ho][wo][c] int8;
+ * acc_out (optional): same shape as y, int32.
+ */
+void prom_ref_dw3x3(const int8_t *x, int batch, int h, int w, int c, int stride,
+                    const int8_t *wt, const int32_t *bias, const int32_t *mult,
+                    const int8_t *shift, int act_min, int act_max, int32_t *acc_out, int8_t *y)
+{
+    int ho = (h - 1) / stride + 1, wo = (w - 1) / stride + 1;
+#pragma omp parallel for schedule(static)
+    for (long bi = 0; bi < (long)batch * ho; ++bi) {
+        int b = (int)(bi / ho), i = (int)(bi % ho);
+        for (int j = 0; j < wo; ++j) {
+            for (int ch = 0; ch < c; ++ch) {
+                int32_t acc = 0;
+                for (int di = 0; di < 3; ++di) {
+                    for (int dj = 0; dj < 3; ++dj) {
+                        int ii = i * stride + di - 1, jj = j * stride + dj - 1;
+                        if (ii < 0 || ii >= h || jj < 0 || jj >= w) continue;
+                        acc += (int32_t)x[(((long)b * h + ii) * w + jj) * c + ch] *
+                               (int32_t)wt[(long)ch * 9 + di * 3 + dj];
+                    }
+                }
+                long o = (((long)b * ho + i) * wo + j) * c + ch;
+                if (acc_out) acc_out[o] = acc;
+                if (y)
+                    y[o] = (int8_t)prom_ref_requant_scalar(acc + bias[ch], mult[ch], shift[ch],
+                                                           act_min, act_max);
+            }
+        }
+    }
+}

@@ -64,6 +64,8 @@ def lib():
                                         C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_float,
                                         C.POINTER(C.c_float), i8p, C.POINTER(C.c_float),
                                         C.POINTER(C.c_float)]
+        L.prom_ref_dw3x3.argtypes = [i8p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, i8p, i32p, i32p, i8p,
+                                     C.c_int, C.c_int, i32p, i8p]
         L.prom_ref_requant_from_scale.restype = C.c_int
         L.prom_ref_requant_from_scale.argtypes = [C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_int)]
         _lib = L
@@ -253,3 +255,21 @@ def conv_dyn(x, w, alpha, gamma_x, rows_per_sample: int, eps: float = 1e-5):
                             _p(alpha, C.c_float), _p(gamma_x, C.c_float), C.c_float(eps),
                             _p(y, C.c_float), _p(q, C.c_int8), _p(gy, C.c_float), _p(sy, C.c_float))
     return q, gy, sy, y
+
+
+def dw3x3(x, w, bias, mult, shift, stride: int = 1, act_min: int = -128, act_max: int = 127,
+          want_acc: bool = False):
+    """int8 depthwise 3x3 convolution, zero padding 1, per-channel fixed-point requantisation.
+    x: int8 [batch, h, w, c]; w: int8 [c, 3, 3]; bias, mult int32 [c]; shift int8 [c].
+    Returns y int8 [batch, ho, wo, c] (and the int32 accumulators when want_acc)."""
+    x = _c(x, np.int8); w = _c(w, np.int8)
+    bias = _c(bias, np.int32); mult = _c(mult, np.int32); shift = _c(shift, np.int8)
+    b, h, wd, c = x.shape
+    assert w.shape == (c, 3, 3) and stride in (1, 2)
+    ho, wo = (h - 1) // stride + 1, (wd - 1) // stride + 1
+    y = np.empty((b, ho, wo, c), dtype=np.int8)
+    acc = np.empty((b, ho, wo, c), dtype=np.int32) if want_acc else None
+    lib().prom_ref_dw3x3(_p(x, C.c_int8), b, h, wd, c, stride, _p(w, C.c_int8), _p(bias, C.c_int32),
+                         _p(mult, C.c_int32), _p(shift, C.c_int8), act_min, act_max,
+                         _p(acc, C.c_int32) if want_acc else None, _p(y, C.c_int8))
+    return (y, acc) if want_acc else y
