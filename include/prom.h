@@ -126,6 +126,23 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin,
                                   uint8_t *packed_dev, size_t packed_bytes,
                                   float *alpha_dev, void *cuda_stream);
 
+/* The int8 depthwise 3x3 convolution between a block's expand and project convolutions
+ * (paper, Section 2: depthwise-separable blocks; Section 3.1: its weights are 8-bit, Eq. 4-5).
+ * Per channel, with one pixel of zero padding and stride 1 or 2,
+ *     acc[b][i][j][c] = sum_{di,dj in 0..2} x[b][i*s + di - 1][j*s + dj - 1][c] * w[c][di][dj]
+ * and y = requant(acc + bias[c], mult[c], shift[c]) clamped to [act_min, act_max], the
+ * requantisation of prom_pw_conv_i8.  Output size: ho = (h - 1) / stride + 1, wo likewise.
+ *   x_dev  [batch][h][w][c] int8, device, 16-byte aligned (NHWC)
+ *   w_dev  [c][3][3] int8, device (the paper quantises them per channel by absmax:
+ *          prom_quantize_act_absmax over a [c][9] float matrix, 16-byte aligned, gives exactly that)
+ *   rq     per-channel constants as for prom_pw_conv_i8 (device arrays of c entries)
+ *   y_dev  [batch][ho][wo][c] int8, device, 16-byte aligned, not x_dev
+ * c must be a multiple of 4 (PROM_ERR_UNSUPPORTED otherwise).  Asynchronous on the stream.
+ * Constants out of range surface as PROM_ERR_BAD_REQUANT in prom_last_device_status. */
+prom_status prom_dw_conv3x3_i8(const int8_t *x_dev, int batch, int h, int w, int c, int stride,
+                               const int8_t *w_dev, const prom_requant *rq, int8_t *y_dev,
+                               void *cuda_stream);
+
 /* A pointwise layer in the paper's own inference dataflow: pseudocode appendix, inference
  * branch of the quantised convolution module ("perform convolution in low bit-width, dequantise
  * after convolution"), followed by the activation quantiser of the next module (Section 3.1,

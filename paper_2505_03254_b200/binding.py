@@ -28,7 +28,7 @@ EXPORTS = [
     "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
     "prom_launch_count", "prom_shutdown", "prom_status_string",
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
-    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn",
+    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -84,6 +84,9 @@ def lib():
         L.prom_pw_conv_i8_addsub_static.restype = i32
         L.prom_pw_conv_i8_addsub_static.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant),
                                                     vp, vp]
+        L.prom_dw_conv3x3_i8.restype = i32
+        L.prom_dw_conv3x3_i8.argtypes = [C.c_void_p, i32, i32, i32, i32, i32, C.c_void_p, C.POINTER(PromRequant),
+                                         C.c_void_p, C.c_void_p]
         L.prom_pw_conv_i8_dyn.restype = i32
         L.prom_pw_conv_i8_dyn.argtypes = [C.c_void_p, i32, i64, i32, C.c_void_p, i32, C.c_void_p, C.c_void_p,
                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -145,6 +148,19 @@ def launch_count() -> int:
 
 def last_device_status(stream=None) -> int:
     return int(lib().prom_last_device_status(_stream(stream)))
+
+
+def dw_conv3x3_i8(x: torch.Tensor, w: torch.Tensor, rq: "PromRequant", stride: int = 1, y=None, stream=None):
+    """prom_dw_conv3x3_i8: x int8 [batch, h, w, c], w int8 [c, 3, 3] on the device ->
+    y int8 [batch, ho, wo, c]."""
+    b, h, wd, c = x.shape
+    ho, wo = (h - 1) // stride + 1, (wd - 1) // stride + 1
+    if y is None:
+        y = torch.empty((b, ho, wo, c), dtype=torch.int8, device=x.device)
+    _check(lib().prom_dw_conv3x3_i8(_dev(x, torch.int8, "x"), b, h, wd, c, stride, _dev(w, torch.int8, "w"),
+                                    C.byref(rq), _dev(y, torch.int8, "y"), _stream(stream)),
+           "prom_dw_conv3x3_i8")
+    return y
 
 
 def pw_conv_i8_dyn(x: torch.Tensor, batch: int, w_packed: torch.Tensor, cout: int, alpha: torch.Tensor,

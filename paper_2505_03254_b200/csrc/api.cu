@@ -21,6 +21,7 @@
 #include "smallk.cuh"
 #include "addsub.cuh"
 #include "actquant.cuh"
+#include "depthwise.cuh"
 #include "quantize.cuh"
 
 namespace prom {
@@ -734,6 +735,36 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin, uint8_t
     const int grid = cout < d.sms * 8 ? cout : d.sms * 8;
     quant::quantize_ternary_kernel<<<grid, quant::kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         w_dev, cout, cin, 1e-5, packed_dev, alpha_dev);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+prom_status prom_dw_conv3x3_i8(const int8_t *x_dev, int batch, int h, int w, int c, int stride,
+                               const int8_t *w_dev, const prom_requant *rq, int8_t *y_dev,
+                               void *cuda_stream)
+{
+    if (batch < 0 || h < 1 || w < 1 || c < 1 || c > 4096 || (stride != 1 && stride != 2)) return PROM_ERR_SHAPE;
+    if (c & 3) return PROM_ERR_UNSUPPORTED;
+    if (!rq) return PROM_ERR_NULL;
+    prom_status e = check_requant(rq);
+    if (e != PROM_OK) return e;
+    if (batch == 0) return PROM_OK;
+    if (!x_dev || !w_dev || !y_dev) return PROM_ERR_NULL;
+    if (!aligned16(x_dev) || !aligned16(y_dev)) return PROM_ERR_ALIGN;
+    if (reinterpret_cast<const void *>(x_dev) == reinterpret_cast<const void *>(y_dev)) return PROM_ERR_ALIGN;
+    const int ho = (h - 1) / stride + 1, wo = (w - 1) / stride + 1;
+    if ((long long)batch * h * w * c >= (1ll << 40)) return PROM_ERR_SHAPE;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    const long long total = (long long)batch * ho * ((wo + dw::kStrip - 1) / dw::kStrip) * (c >> 2);
+    const int grid = grid_for(total, dw::kThreads, d.sms);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (stride == 1)
+        dw::dw3x3_kernel<1><<<grid, dw::kThreads, 0, st>>>(x_dev, batch, h, w, c, ho, wo, w_dev, rq->bias,
+                                                           rq->mult, rq->shift, rq->act_min, rq->act_max, y_dev);
+    else
+        dw::dw3x3_kernel<2><<<grid, dw::kThreads, 0, st>>>(x_dev, batch, h, w, c, ho, wo, w_dev, rq->bias,
+                                                           rq->mult, rq->shift, rq->act_min, rq->act_max, y_dev);
     ++g_launches;
     return cuda_status(cudaGetLastError());
 }
