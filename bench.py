@@ -433,6 +433,7 @@ def run_gpu(args):
         out["quantizer"] = quantizer_timing(torch, binding, table, bw)
         out["act_quantizer"] = act_quantizer_timing(torch, binding, bw)
         out["dynamic_layer"] = dynamic_layer_timing(torch, binding, synth, bw)
+        out["depthwise"] = depthwise_timing(torch, binding, bw)
         cold_us = sum(r["us"] for r in out["layers"])
         roofline["sum_layer_cold_us"] = cold_us
         roofline["sum_layer_cold_frac"] = sum(roof_us) / cold_us
@@ -541,6 +542,29 @@ def dynamic_layer_timing(torch, binding, synth, bw):
     return {"workload": "1605632x16->96, 128 samples: convolution, dequantise, per-sample absmax, quantise",
             "us": round(ms * 1e3, 2), "bytes": nbytes, "gbs": round(nbytes / ms / 1e6, 1),
             "roof_us": round(nbytes / bw * 1e6, 2), "frac": round(nbytes / bw * 1e3 / ms, 4)}
+
+
+def depthwise_timing(torch, binding, bw):
+    """The int8 depthwise 3x3 convolutions of the first blocks at batch 128 (off the timed step,
+    where the depthwise layer is an identity stand-in): the two largest of the network."""
+    g = torch.Generator(device="cuda").manual_seed(4)
+    rows = []
+    for (h, c, s) in ((112, 96, 2), (56, 144, 1)):
+        x = torch.randint(-128, 128, (BATCH, h, h, c), generator=g, device="cuda", dtype=torch.int8)
+        w = torch.randint(-128, 128, (c, 3, 3), generator=g, device="cuda", dtype=torch.int8)
+        bias = torch.zeros((c,), dtype=torch.int32, device="cuda")
+        rq = binding.make_requant(bias, bias + (1 << 30), torch.full((c,), 8, dtype=torch.int8, device="cuda"))
+        ho = (h - 1) // s + 1
+        y = torch.empty((BATCH, ho, ho, c), dtype=torch.int8, device="cuda")
+        fn = lambda: binding.dw_conv3x3_i8(x, w, rq, stride=s, y=y)
+        for _ in range(3):
+            fn()
+        ms = time_region(torch, fn, 20, False) / 20
+        nbytes = x.numel() + y.numel()
+        rows.append({"shape": "[%d,%d,%d,%d] stride %d" % (BATCH, h, h, c, s), "us": round(ms * 1e3, 2),
+                     "gbs": round(nbytes / ms / 1e6, 1), "roof_us": round(nbytes / bw * 1e6, 2),
+                     "frac": round(nbytes / bw * 1e3 / ms, 4)})
+    return rows
 
 
 def single_layer_configs(torch, binding, synth, bw, p_i8):

@@ -757,7 +757,15 @@ prom_status prom_dw_conv3x3_i8(const int8_t *x_dev, int batch, int h, int w, int
     DeviceInfo d = device_info();
     if (!d.ok) return PROM_ERR_CUDA;
     const long long total = (long long)batch * ho * ((wo + dw::kStrip - 1) / dw::kStrip) * (c >> 2);
-    const int grid = grid_for(total, dw::kThreads, d.sms);
+    // a multiple of c / 4 threads, so that a thread keeps its channels: blocks in multiples of
+    // (c / 4) / gcd(c / 4, threads per block)
+    int step = c >> 2;
+    for (int a = step, b = dw::kThreads; b;) { const int r = a % b; a = b; b = r; if (!b) step = (c >> 2) / a; }
+    long long blocks = (total + dw::kThreads - 1) / dw::kThreads;
+    const long long cap = (long long)d.sms * 16;
+    if (blocks > cap) blocks = cap;
+    blocks = (blocks + step - 1) / step * step;
+    const int grid = (int)blocks;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (stride == 1)
         dw::dw3x3_kernel<1><<<grid, dw::kThreads, 0, st>>>(x_dev, batch, h, w, c, ho, wo, w_dev, rq->bias,

@@ -31,8 +31,10 @@ __device__ __forceinline__ void bytes_to_floats(uint32_t wd, float (&f)[4])
     }
 }
 
+// The launch has a multiple of c / 4 threads, so a thread keeps its four channels for all the
+// strips it works on: filters and constants are fetched once.
 template <int STRIDE>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)      // 80 registers: three blocks per SM beat no spills
 dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int ho, int wo,
              const int8_t *__restrict__ wt, const int32_t *__restrict__ bias,
              const int32_t *__restrict__ mult, const int8_t *__restrict__ shift, int lo, int hi,
@@ -40,23 +42,40 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
 {
     const int cw = c >> 2;                                // channel words per pixel
     const int strips = (wo + kStrip - 1) / kStrip;
-    const long long total = (long long)batch * ho * strips * cw;
-    for (long long idx = (long long)blockIdx.x * kThreads + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * kThreads) {
-        const int cg = (int)(idx % cw);
-        long long r = idx / cw;
-        const int sp = (int)(r % strips); r /= strips;
-        const int i = (int)(r % ho);
-        const int b = (int)(r / ho);
-        const int j0 = sp * kStrip;
-        const int ch = cg * 4;
+    const long long units = (long long)batch * ho * strips;
+    const long long tid = (long long)blockIdx.x * kThreads + threadIdx.x;
+    const long long nthreads = (long long)gridDim.x * kThreads;
+    const int ch = (int)(tid % cw) * 4;
 
-        // this thread's filters: wf[tap][channel]
-        float wf[9][4];
+    // this thread's filters wf[tap][channel] and requantisation constants
+    float wf[9][4];
+    int cb[4], cm[4], cs[4];
+    bool bad = false;
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
+    for (int k = 0; k < 4; ++k) {
 #pragma unroll
-            for (int t = 0; t < 9; ++t) wf[t][k] = (float)wt[(size_t)(ch + k) * 9 + t];
+        for (int t = 0; t < 9; ++t) wf[t][k] = (float)wt[(size_t)(ch + k) * 9 + t];
+        cb[k] = __ldg(bias + ch + k); cm[k] = __ldg(mult + ch + k); cs[k] = __ldg(shift + ch + k);
+        if (!requant_ok(cb[k], cm[k], cs[k])) { bad = true; cb[k] = 0; cm[k] = 0; cs[k] = 0; }
+    }
+    if (bad) raise_status(PROM_ERR_BAD_REQUANT);
+
+    constexpr int kCols = STRIDE * (kStrip - 1) + 3;      // input columns under a strip
+    const size_t pix = (size_t)c;                         // bytes from a pixel to the next
+    for (long long u = tid / cw; u < units; u += nthreads / cw) {
+        const int sp = (int)(u % strips);
+        const long long r = u / strips;
+        const int i = (int)(r % ho), b = (int)(r / ho);
+        const int j0 = sp * kStrip;
+        const int jin0 = j0 * STRIDE - 1;
+
+        // the three input rows under this output row (null outside the image)
+        const int8_t *rowp[3];
+#pragma unroll
+        for (int di = 0; di < 3; ++di) {
+            const int ii = i * STRIDE + di - 1;
+            rowp[di] = (ii >= 0 && ii < h) ? x + (((size_t)b * h + ii) * w) * pix + ch : nullptr;
+        }
 
         float acc[kStrip][4];
 #pragma unroll
@@ -64,52 +83,44 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
 #pragma unroll
             for (int k = 0; k < 4; ++k) acc[o][k] = 0.0f;
 
-        const int8_t *xb = x + (size_t)b * h * w * c;
-        constexpr int kCols = STRIDE * (kStrip - 1) + 3;   // input columns under the strip
-        const int jin0 = j0 * STRIDE - 1;
 #pragma unroll
         for (int cidx = 0; cidx < kCols; ++cidx) {
             const int jj = jin0 + cidx;
-            if (jj < 0 || jj >= w) continue;
+            const bool col_ok = jj >= 0 && jj < w;
 #pragma unroll
             for (int di = 0; di < 3; ++di) {
-                const int ii = i * STRIDE + di - 1;
-                if (ii < 0 || ii >= h) continue;
-                const uint32_t wd = __ldg(reinterpret_cast<const uint32_t *>(xb + ((size_t)ii * w + jj) * c + ch));
+                // a pixel outside the image reads as zeros (and converts to 0.0)
+                uint32_t wd = 0;
+                if (col_ok && rowp[di]) wd = __ldg(reinterpret_cast<const uint32_t *>(rowp[di] + (size_t)jj * pix));
                 float f[4];
                 bytes_to_floats(wd, f);
                 // output o of the strip sees this column as tap dj = cidx - o * STRIDE
 #pragma unroll
                 for (int o = 0; o < kStrip; ++o) {
-                    const int dj = cidx - o * STRIDE;
-                    if (dj < 0 || dj > 2) continue;
+                    constexpr int kS = STRIDE;
+                    const int dj = cidx - o * kS;
+                    if (dj >= 0 && dj <= 2) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) acc[o][k] = fmaf(f[k], wf[di * 3 + dj][k], acc[o][k]);
+                        for (int k = 0; k < 4; ++k) acc[o][k] = fmaf(f[k], wf[di * 3 + dj][k], acc[o][k]);
+                    }
                 }
             }
         }
 
-        int cb[4], cm[4], cs[4];
-        bool bad = false;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            cb[k] = __ldg(bias + ch + k); cm[k] = __ldg(mult + ch + k); cs[k] = __ldg(shift + ch + k);
-            if (!requant_ok(cb[k], cm[k], cs[k])) { bad = true; cb[k] = 0; cm[k] = 0; cs[k] = 0; }
-        }
-        if (bad) raise_status(PROM_ERR_BAD_REQUANT);
+        int8_t *yrow = y + (((size_t)b * ho + i) * wo + j0) * pix + ch;
 #pragma unroll
         for (int o = 0; o < kStrip; ++o) {
-            const int j = j0 + o;
-            if (j >= wo) break;
-            uint32_t out = 0;
+            if (j0 + o < wo) {
+                uint32_t out = 0;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int t = (int)acc[o][k] + cb[k];
-                const int q = lo >= 0 ? requant_floor(t, cm[k], cs[k], lo, hi)
-                                      : requant_exact(t, cm[k], cs[k], lo, hi);
-                out |= ((uint32_t)q & 0xFFu) << (8 * k);
+                for (int k = 0; k < 4; ++k) {
+                    const int t = (int)acc[o][k] + cb[k];
+                    const int q = lo >= 0 ? requant_floor(t, cm[k], cs[k], lo, hi)
+                                          : requant_exact(t, cm[k], cs[k], lo, hi);
+                    out |= ((uint32_t)q & 0xFFu) << (8 * k);
+                }
+                *reinterpret_cast<uint32_t *>(yrow + (size_t)o * pix) = out;
             }
-            *reinterpret_cast<uint32_t *>(y + (((size_t)b * ho + i) * wo + j) * c + ch) = out;
         }
     }
 }
