@@ -731,6 +731,27 @@ def run_widths(args):
     return 0 if all(r["parity_image_0"] for r in rows) else 1
 
 
+def run_aux(args):
+    """One of the legs that are off the timed step, alone (for profiling): act_quantizer,
+    dynamic_layer or depthwise."""
+    import torch
+    from paper_2505_03254_b200 import binding, build, synth
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(0)
+    build.build()
+    binding.lib()
+    bw = peaks()["hbm_gbs"] * 1e9
+    if args.aux == "act_quantizer":
+        out = act_quantizer_timing(torch, binding, bw)
+    elif args.aux == "dynamic_layer":
+        out = dynamic_layer_timing(torch, binding, synth, bw)
+    else:
+        out = depthwise_timing(torch, binding, bw)
+    print(json.dumps({"aux": args.aux, "result": out, "device_status": binding.last_device_status()}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -743,6 +764,8 @@ def main():
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
     ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
+    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise"],
+                    help="run one of the legs that are off the timed step, alone")
     ap.add_argument("--widths", default=None, help="comma-separated width multipliers: time the sequence at each")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")
     args = ap.parse_args()
@@ -750,6 +773,8 @@ def main():
         return run_reference(args)
     if args.widths:
         return run_widths(args)
+    if args.aux:
+        return run_aux(args)
     if args.single:
         return run_single(args)
     if args.sweep:

@@ -5,12 +5,11 @@
 // pointwise layers.  NHWC, so a pixel's channels are contiguous.
 //
 // A thread owns 4 channels (one 32-bit word per pixel) and a strip of kStrip output pixels of
-// one output row.  It walks over the input columns of the strip once: the 3 x 4 bytes of a
-// column become floats (exactly: byte inserted into the mantissa of 2^23, one subtraction) and
-// feed the up to three outputs whose window contains the column with fused multiply-adds in
-// binary32, exact because |acc| <= 9 * 128 * 128 < 2^24.  The 36 weights of the thread's
-// channels stay in registers as floats.  Threads of a warp take consecutive channel words, so
-// loads and stores of a pixel are contiguous.
+// one output row.  It loads the 3 x (columns under the strip) words once; for every output the
+// nine tap words are transposed with byte permutes into one word per channel holding four taps,
+// and each channel's sum is three dp4a instructions against the channel's nine weights kept as
+// three packed words: no byte is ever unpacked or converted, and the int32 sums are exact.
+// Threads of a warp take consecutive channel words, so loads and stores of a pixel are contiguous.
 #pragma once
 
 #include "common.cuh"
@@ -20,15 +19,14 @@ namespace prom { namespace dw {
 constexpr int kThreads = 256;
 constexpr int kStrip = 4;
 
-// four signed bytes of a word -> four floats
-__device__ __forceinline__ void bytes_to_floats(uint32_t wd, float (&f)[4])
+// 4 x 4 byte transpose: words a, b, c, d hold one tap each (byte k = channel k); o[k] gets the
+// four taps of channel k.
+__device__ __forceinline__ void transpose4(uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t (&o)[4])
 {
-    const uint32_t u = wd ^ 0x80808080u;                  // signed -> offset binary
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const uint32_t bits = __byte_perm(u, 0x4B000000u, 0x7650 + k);   // 2^23 + byte k
-        f[k] = __uint_as_float(bits) - 8388736.0f;                       // - (2^23 + 128)
-    }
+    const uint32_t t0 = __byte_perm(a, b, 0x5140), t1 = __byte_perm(a, b, 0x7362);
+    const uint32_t t2 = __byte_perm(c, d, 0x5140), t3 = __byte_perm(c, d, 0x7362);
+    o[0] = __byte_perm(t0, t2, 0x5410); o[1] = __byte_perm(t0, t2, 0x7632);
+    o[2] = __byte_perm(t1, t3, 0x5410); o[3] = __byte_perm(t1, t3, 0x7632);
 }
 
 // The launch has a multiple of c / 4 threads, so a thread keeps its four channels for all the
@@ -47,14 +45,17 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
     const long long nthreads = (long long)gridDim.x * kThreads;
     const int ch = (int)(tid % cw) * 4;
 
-    // this thread's filters wf[tap][channel] and requantisation constants
-    float wf[9][4];
+    // this thread's filters, wk[group][channel]: taps 0-3, taps 4-7, tap 8 (low byte), and its
+    // requantisation constants
+    uint32_t wk[3][4];
     int cb[4], cm[4], cs[4];
     bool bad = false;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-#pragma unroll
-        for (int t = 0; t < 9; ++t) wf[t][k] = (float)wt[(size_t)(ch + k) * 9 + t];
+        const uint8_t *wp = reinterpret_cast<const uint8_t *>(wt) + (size_t)(ch + k) * 9;
+        wk[0][k] = (uint32_t)wp[0] | ((uint32_t)wp[1] << 8) | ((uint32_t)wp[2] << 16) | ((uint32_t)wp[3] << 24);
+        wk[1][k] = (uint32_t)wp[4] | ((uint32_t)wp[5] << 8) | ((uint32_t)wp[6] << 16) | ((uint32_t)wp[7] << 24);
+        wk[2][k] = (uint32_t)wp[8];
         cb[k] = __ldg(bias + ch + k); cm[k] = __ldg(mult + ch + k); cs[k] = __ldg(shift + ch + k);
         if (!requant_ok(cb[k], cm[k], cs[k])) { bad = true; cb[k] = 0; cm[k] = 0; cs[k] = 0; }
     }
@@ -77,33 +78,33 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
             rowp[di] = (ii >= 0 && ii < h) ? x + (((size_t)b * h + ii) * w) * pix + ch : nullptr;
         }
 
-        float acc[kStrip][4];
-#pragma unroll
-        for (int o = 0; o < kStrip; ++o)
-#pragma unroll
-            for (int k = 0; k < 4; ++k) acc[o][k] = 0.0f;
-
+        // the words under the strip: xin[row][column], zeros outside the image
+        uint32_t xin[3][kCols];
 #pragma unroll
         for (int cidx = 0; cidx < kCols; ++cidx) {
             const int jj = jin0 + cidx;
             const bool col_ok = jj >= 0 && jj < w;
+            const unsigned off = (unsigned)(jj < 0 ? 0 : jj) * (unsigned)c;
 #pragma unroll
-            for (int di = 0; di < 3; ++di) {
-                // a pixel outside the image reads as zeros (and converts to 0.0)
-                uint32_t wd = 0;
-                if (col_ok && rowp[di]) wd = __ldg(reinterpret_cast<const uint32_t *>(rowp[di] + (size_t)jj * pix));
-                float f[4];
-                bytes_to_floats(wd, f);
-                // output o of the strip sees this column as tap dj = cidx - o * STRIDE
+            for (int di = 0; di < 3; ++di)
+                xin[di][cidx] = (col_ok && rowp[di]) ? __ldg(reinterpret_cast<const uint32_t *>(rowp[di] + off)) : 0u;
+        }
+
+        int acc[kStrip][4];
 #pragma unroll
-                for (int o = 0; o < kStrip; ++o) {
-                    constexpr int kS = STRIDE;
-                    const int dj = cidx - o * kS;
-                    if (dj >= 0 && dj <= 2) {
+        for (int o = 0; o < kStrip; ++o) {
+            const int c0 = o * STRIDE;                    // first column of this output's window
+            uint32_t g0[4], g1[4];
+            // taps (0,0) (0,1) (0,2) (1,0) and (1,1) (1,2) (2,0) (2,1); tap (2,2) on its own
+            transpose4(xin[0][c0], xin[0][c0 + 1], xin[0][c0 + 2], xin[1][c0], g0);
+            transpose4(xin[1][c0 + 1], xin[1][c0 + 2], xin[2][c0], xin[2][c0 + 1], g1);
+            const uint32_t last = xin[2][c0 + 2];
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) acc[o][k] = fmaf(f[k], wf[di * 3 + dj][k], acc[o][k]);
-                    }
-                }
+            for (int k = 0; k < 4; ++k) {
+                int a = __dp4a((int)g0[k], (int)wk[0][k], 0);
+                a = __dp4a((int)g1[k], (int)wk[1][k], a);
+                a = __dp4a((int)__byte_perm(last, 0u, 0x4440 + k), (int)wk[2][k], a);
+                acc[o][k] = a;
             }
         }
 
@@ -114,7 +115,7 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
                 uint32_t out = 0;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const int t = (int)acc[o][k] + cb[k];
+                    const int t = acc[o][k] + cb[k];
                     const int q = lo >= 0 ? requant_floor(t, cm[k], cs[k], lo, hi)
                                           : requant_exact(t, cm[k], cs[k], lo, hi);
                     out |= ((uint32_t)q & 0xFFu) << (8 * k);
