@@ -63,10 +63,12 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
 
     constexpr int kCols = STRIDE * (kStrip - 1) + 3;      // input columns under a strip
     const size_t pix = (size_t)c;                         // bytes from a pixel to the next
-    for (long long u = tid / cw; u < units; u += nthreads / cw) {
-        const int sp = (int)(u % strips);
-        const long long r = u / strips;
-        const int i = (int)(r % ho), b = (int)(r / ho);
+    // 32-bit unit indices (the host keeps batch * ho * strips below 2^31)
+    const unsigned ustep = (unsigned)(nthreads / cw);
+    for (unsigned u = (unsigned)(tid / cw); u < (unsigned)units; u += ustep) {
+        const unsigned r = u / (unsigned)strips;
+        const int sp = (int)(u - r * (unsigned)strips);
+        const int b = (int)(r / (unsigned)ho), i = (int)(r - (unsigned)b * (unsigned)ho);
         const int j0 = sp * kStrip;
         const int jin0 = j0 * STRIDE - 1;
 
@@ -112,14 +114,20 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
 #pragma unroll
         for (int o = 0; o < kStrip; ++o) {
             if (j0 + o < wo) {
-                uint32_t out = 0;
+                int q[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const int t = acc[o][k] + cb[k];
-                    const int q = lo >= 0 ? requant_floor(t, cm[k], cs[k], lo, hi)
-                                          : requant_exact(t, cm[k], cs[k], lo, hi);
-                    out |= ((uint32_t)q & 0xFFu) << (8 * k);
+                    q[k] = lo >= 0 ? requant_floor(t, cm[k], cs[k], lo, hi)
+                                   : requant_exact(t, cm[k], cs[k], lo, hi);
                 }
+                // already within [-128, 127]: the saturating packs only gather the low bytes
+                uint32_t out;
+                asm("{\n\t.reg .b32 t;\n\t"
+                    "cvt.pack.sat.s8.s32.b32 t, %4, %3, 0;\n\t"
+                    "cvt.pack.sat.s8.s32.b32 %0, %2, %1, t;\n\t}"
+                    : "=r"(out)
+                    : "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3]));
                 *reinterpret_cast<uint32_t *>(yrow + (size_t)o * pix) = out;
             }
         }
