@@ -434,6 +434,7 @@ def run_gpu(args):
         out["act_quantizer"] = act_quantizer_timing(torch, binding, bw)
         out["dynamic_layer"] = dynamic_layer_timing(torch, binding, synth, bw)
         out["depthwise"] = depthwise_timing(torch, binding, bw)
+        out["body_with_depthwise"] = body_with_depthwise_timing(torch, binding, synth, bw)
         cold_us = sum(r["us"] for r in out["layers"])
         roofline["sum_layer_cold_us"] = cold_us
         roofline["sum_layer_cold_frac"] = sum(roof_us) / cold_us
@@ -565,6 +566,45 @@ def depthwise_timing(torch, binding, bw):
                      "gbs": round(nbytes / ms / 1e6, 1), "roof_us": round(nbytes / bw * 1e6, 2),
                      "frac": round(nbytes / bw * 1e3 / ms, 4)})
     return rows
+
+
+def body_with_depthwise_timing(torch, binding, synth, bw):
+    """The 34 pointwise layers with a real int8 depthwise 3x3 in front of every project
+    convolution (17 of them) in place of the identity stand-in: the body of MobileNetV2 without
+    its residual adds, batch 128, CUDA graph.  Algorithmic bytes: the pointwise layers' plus one
+    byte in and one byte out per depthwise value."""
+    seed = synth.BASE_SEED + 3
+    table, _, dev = build_network(seed, synth, binding, "cuda")
+    g = torch.Generator(device="cuda").manual_seed(5)
+    nbytes = 0
+    for l, d in zip(table, dev):
+        m = BATCH * l.h * l.w
+        nbytes += layer_bytes(m, l.cin, l.cout)
+        if l.name.endswith("project"):
+            c = l.cin
+            d["dw_w"] = torch.randint(-20, 21, (c, 3, 3), generator=g, device="cuda", dtype=torch.int8)
+            d["dw_bias"] = torch.zeros((c,), dtype=torch.int32, device="cuda")
+            d["dw_mult"] = torch.full((c,), 1 << 30, dtype=torch.int32, device="cuda")
+            d["dw_shift"] = torch.full((c,), 6, dtype=torch.int8, device="cuda")
+            nbytes += m * c * l.in_stride * l.in_stride + m * c
+    seq = binding.LayerSeq(dev)
+    x0 = synth.act_post_relu6(seed, (BATCH, 112, 112, 32), device="cuda")
+    ws = torch.empty((seq.workspace_bytes(BATCH, 112, 112),), dtype=torch.uint8, device="cuda")
+    y = torch.empty((BATCH, 7, 7, 1280), dtype=torch.int8, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
+    for _ in range(3):
+        graph.replay()
+    ms = time_region(torch, graph.replay, 50, False) / 50
+    return {"workload": "34 pointwise + 17 depthwise 3x3 layers, chained, batch 128",
+            "ms_per_step": round(ms, 4), "images_per_s": round(BATCH / ms * 1e3, 1), "bytes": nbytes,
+            "roof_us": round(nbytes / bw * 1e6, 1), "frac": round(nbytes / bw * 1e3 / ms, 4),
+            "device_status": binding.last_device_status()}
 
 
 def single_layer_configs(torch, binding, synth, bw, p_i8):
@@ -746,6 +786,8 @@ def run_aux(args):
         out = act_quantizer_timing(torch, binding, bw)
     elif args.aux == "dynamic_layer":
         out = dynamic_layer_timing(torch, binding, synth, bw)
+    elif args.aux == "body":
+        out = body_with_depthwise_timing(torch, binding, synth, bw)
     else:
         out = depthwise_timing(torch, binding, bw)
     print(json.dumps({"aux": args.aux, "result": out, "device_status": binding.last_device_status()}))
@@ -764,7 +806,7 @@ def main():
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
     ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
-    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise"],
+    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body"],
                     help="run one of the legs that are off the timed step, alone")
     ap.add_argument("--widths", default=None, help="comma-separated width multipliers: time the sequence at each")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")

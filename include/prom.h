@@ -86,15 +86,21 @@ typedef struct {
 } prom_requant;
 
 /* One layer of a sequence.  in_stride (1 or 2) is the spatial subsampling
- * applied to this layer's input: the depthwise convolution that sits between
- * an expand and a project convolution (Section 2) is modelled as the identity
- * on values plus its stride, so output pixel (i, j) reads input pixel
- * (in_stride*i, in_stride*j). */
+ * applied to this layer's input.  With dw_w == NULL the depthwise convolution
+ * that sits between an expand and a project convolution (Section 2) is
+ * modelled as the identity on values plus its stride: output pixel (i, j)
+ * reads input pixel (in_stride*i, in_stride*j).  With dw_w set, the int8
+ * depthwise 3x3 convolution of prom_dw_conv3x3_i8 (weights dw_w [cin][3][3],
+ * constants dw_rq, stride in_stride) runs on the layer's input first and the
+ * pointwise convolution reads its output; the input's height and width must
+ * then be multiples of in_stride. */
 typedef struct {
     int cin, cout;
     int in_stride;
     const uint8_t *w_packed;   /* device, prom_packed_bytes(cout, cin) bytes */
     prom_requant rq;
+    const int8_t *dw_w;        /* device, or NULL: no depthwise convolution in front */
+    prom_requant dw_rq;        /* read only when dw_w is set */
 } prom_layer;
 
 /* Bytes of the 2-bit form of a [cout][cin] ternary matrix: cout*ceil(cin/4).

@@ -40,7 +40,8 @@ class PromRequant(C.Structure):
 
 class PromLayer(C.Structure):
     _fields_ = [("cin", C.c_int), ("cout", C.c_int), ("in_stride", C.c_int),
-                ("w_packed", C.c_void_p), ("rq", PromRequant)]
+                ("w_packed", C.c_void_p), ("rq", PromRequant),
+                ("dw_w", C.c_void_p), ("dw_rq", PromRequant)]
 
 
 class PromError(RuntimeError):
@@ -324,6 +325,12 @@ class LayerSeq:
             self.array[i] = PromLayer(int(l["cin"]), int(l["cout"]), int(l["in_stride"]),
                                       _dev(l["w_packed"], torch.uint8, "w_packed"),
                                       make_requant(l["bias"], l["mult"], l["shift"], act_min, act_max))
+            if l.get("dw_w") is not None:
+                # a real depthwise 3x3 in front: int8 [cin, 3, 3] weights and their constants
+                for k in ("dw_w", "dw_bias", "dw_mult", "dw_shift"):
+                    self._keep.append(l[k])
+                self.array[i].dw_w = _dev(l["dw_w"], torch.int8, "dw_w")
+                self.array[i].dw_rq = make_requant(l["dw_bias"], l["dw_mult"], l["dw_shift"], act_min, act_max)
         self.cout_last = int(layers[-1]["cout"])
         self.cin0 = int(layers[0]["cin"])
         self.total_stride = 1

@@ -530,6 +530,10 @@ static bool seq_shapes(const prom_layer *layers, int n, int batch, int h0, int w
         mp.stride = l.in_stride; mp.hin = h; mp.win = w;
         h /= l.in_stride; w /= l.in_stride;
         mp.ho = h; mp.wo = w;
+        if (l.dw_w) {                 // the depthwise convolution applies the stride itself
+            if (l.cin & 3) return false;
+            mp.stride = 1; mp.hin = h; mp.win = w;
+        }
         s.map.push_back(mp);
         s.m.push_back((long long)batch * h * w);
         s.h.push_back(h); s.w.push_back(w);
@@ -537,14 +541,26 @@ static bool seq_shapes(const prom_layer *layers, int n, int batch, int h0, int w
     return true;
 }
 
-static void seq_regions(const prom_layer *layers, int n, const SeqShape &s, size_t &a, size_t &b)
+// Workspace regions: a and b take the outputs of even and odd layers in turn; b also ends with
+// room for the largest depthwise output (the input of the pointwise convolution behind it).
+static void seq_regions(const prom_layer *layers, int n, const SeqShape &s, size_t &a, size_t &b,
+                        size_t *dw_off = nullptr)
 {
     a = b = 0;
-    for (int i = 0; i + 1 < n; ++i) {
-        size_t bytes = round256((size_t)s.m[i] * layers[i].cout);
-        if (i & 1) { if (bytes > b) b = bytes; }
-        else { if (bytes > a) a = bytes; }
+    size_t c = 0;
+    for (int i = 0; i < n; ++i) {
+        if (i + 1 < n) {
+            size_t bytes = round256((size_t)s.m[i] * layers[i].cout);
+            if (i & 1) { if (bytes > b) b = bytes; }
+            else { if (bytes > a) a = bytes; }
+        }
+        if (layers[i].dw_w) {
+            size_t bytes = round256((size_t)s.m[i] * layers[i].cin);
+            if (bytes > c) c = bytes;
+        }
     }
+    if (dw_off) *dw_off = a + b;
+    b += c;
 }
 
 // Bytes of prepared-operand images a sequence wants in its workspace (0 for layers the
@@ -564,23 +580,31 @@ static size_t seq_image_bytes(const prom_layer *layers, int n, const SeqShape &s
     return total;
 }
 
+extern "C" prom_status prom_dw_conv3x3_i8(const int8_t *, int, int, int, int, int, const int8_t *,
+                                          const prom_requant *, int8_t *, void *);
+
 static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, int batch, int h0,
                            int w0, void *ws, size_t ws_bytes, int8_t *y_out, prom_variant variant,
                            cudaStream_t st)
 {
     SeqShape s;
     if (!seq_shapes(layers, n, batch, h0, w0, s)) return PROM_ERR_SHAPE;
-    size_t ra, rb;
-    seq_regions(layers, n, s, ra, rb);
+    size_t ra, rb, dw_off;
+    seq_regions(layers, n, s, ra, rb, &dw_off);
     if (ra + rb > 0) {
         if (!ws) return PROM_ERR_NULL;
         if (!aligned16(ws)) return PROM_ERR_ALIGN;
         if (ws_bytes < ra + rb) return PROM_ERR_WORKSPACE;
     }
     int8_t *reg[2] = {static_cast<int8_t *>(ws), static_cast<int8_t *>(ws) + ra};
+    int8_t *dw_buf = static_cast<int8_t *>(ws) + dw_off;      // depthwise outputs
     // validate everything before the first launch
     for (int i = 0; i < n; ++i) {
         if (!layers[i].w_packed) return PROM_ERR_NULL;
+        if (layers[i].dw_w) {
+            prom_status de = check_requant(&layers[i].dw_rq);
+            if (de != PROM_OK) return de;
+        }
         prom_status e = check_requant(&layers[i].rq);
         if (e != PROM_OK) return e;
         if (!aligned16(layers[i].w_packed)) return PROM_ERR_ALIGN;
@@ -603,8 +627,9 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
     long long in_rows = (long long)batch * h0 * w0;
     for (int i = 0; i < n; ++i) {
         Conv &c = conv[i];
-        c.x = cur; c.m = s.m[i]; c.cin = layers[i].cin; c.cout = layers[i].cout;
-        c.map = s.map[i]; c.in_rows = in_rows;
+        // behind a depthwise convolution the pointwise layer reads that convolution's output
+        c.x = layers[i].dw_w ? dw_buf : cur; c.m = s.m[i]; c.cin = layers[i].cin; c.cout = layers[i].cout;
+        c.map = s.map[i]; c.in_rows = layers[i].dw_w ? s.m[i] : in_rows;
         c.w = layers[i].w_packed; c.rq = layers[i].rq;
         c.y = (i == n - 1) ? y_out : reg[i & 1];
         c.st = st;
@@ -646,6 +671,13 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
     }
 
     for (int i = 0; i < n; ++i) {
+        if (layers[i].dw_w && s.m[i] > 0) {
+            const int stride = layers[i].in_stride;
+            const int8_t *src = i == 0 ? x0 : conv[i - 1].y;
+            prom_status de = prom_dw_conv3x3_i8(src, batch, s.h[i] * stride, s.w[i] * stride, layers[i].cin,
+                                                stride, layers[i].dw_w, &layers[i].dw_rq, dw_buf, st);
+            if (de != PROM_OK) return de;
+        }
         prom_status e = is_tc[i] ? tc_launch_planned(conv[i], plan[i]) : run_conv(conv[i], variant);
         if (e != PROM_OK) return e;
     }

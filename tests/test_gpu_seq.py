@@ -90,6 +90,49 @@ def test_width_multiplier_layers_on_the_tensor_cores(oracle, width):
             assert first_mismatch(y.cpu().numpy(), want) is None, (l.cin, l.cout, variant)
 
 
+@pytest.mark.parametrize("batch,hw", [(2, 32), (1, 64)])
+def test_sequence_with_real_depthwise_convolutions(oracle, batch, hw):
+    """The body of the network with the int8 depthwise 3x3 in front of every project
+    convolution (stride in the depthwise layer) instead of the identity stand-in, against the
+    oracle's depthwise and pointwise functions applied layer by layer."""
+    table = synth.mobilenetv2_pointwise_layers(h0=hw, w0=hw)
+    rng = np.random.default_rng(35)
+    host, dev = [], []
+    for i, l in enumerate(table):
+        d = synth.make_layer(35, l.cin, l.cout, 0.5, index=i + 1)
+        hl = dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride, w=d["w"].numpy(), bias=d["bias"].numpy(),
+                  mult=d["mult"].numpy(), shift=d["shift"].numpy())
+        dl = dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride, w_packed=binding.pack_ternary(d["w"].cuda()),
+                  bias=d["bias"].cuda(), mult=d["mult"].cuda(), shift=d["shift"].cuda())
+        if l.name.endswith("project"):
+            hl["dw_w"] = rng.integers(-20, 21, size=(l.cin, 3, 3)).astype(np.int8)
+            hl["dw_bias"] = rng.integers(-64, 65, size=l.cin).astype(np.int32)
+            hl["dw_mult"] = rng.integers(1 << 30, (1 << 31) - 1, size=l.cin).astype(np.int32)
+            hl["dw_shift"] = rng.integers(5, 8, size=l.cin).astype(np.int8)
+            for k in ("dw_w", "dw_bias", "dw_mult", "dw_shift"):
+                dl[k] = torch.from_numpy(hl[k]).cuda()
+        host.append(hl); dev.append(dl)
+    seq = binding.LayerSeq(dev)
+    x0 = synth.act_post_relu6(35, (batch, hw, hw, 32))
+    ws = torch.empty((seq.workspace_bytes(batch, hw, hw),), dtype=torch.uint8, device="cuda")
+    y = binding.pw_layer_seq(seq, x0.cuda(), ws)
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == binding.PROM_OK
+    cur = x0.numpy()
+    for hl in host:
+        if "dw_w" in hl:
+            cur = oracle.dw3x3(cur, hl["dw_w"], hl["dw_bias"], hl["dw_mult"], hl["dw_shift"],
+                               stride=hl["in_stride"], act_min=0, act_max=127)
+        elif hl["in_stride"] != 1:
+            cur = oracle.subsample(cur, hl["in_stride"])
+        b, h, w, c = cur.shape
+        out = oracle.conv_mul(cur.reshape(-1, c), hl["w"], hl["bias"], hl["mult"], hl["shift"])
+        cur = out.reshape(b, h, w, hl["cout"])
+    assert y.shape == cur.shape
+    assert first_mismatch(y.cpu().numpy().reshape(-1, 1280), cur.reshape(-1, 1280)) is None
+    assert (cur != 0).mean() > 0.05          # the chain has not collapsed to zeros
+
+
 def test_sequence_host_entry_point(oracle):
     table = synth.mobilenetv2_pointwise_layers(h0=32, w0=32)[:9]
     host, seq = build_sequence(32, table)
