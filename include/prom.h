@@ -325,6 +325,10 @@ uint64_t prom_launch_count(void);
  * 1, or returns 0 if TC cannot run it.  Without a CUDA device it plans for a
  * B200's nominal limits (148 SMs, 227 KB of shared memory per CTA). */
 void prom_debug_tc_plan(int fold, int nt, int groups, int occ, int stages);
+/* The same override for one shape only (m rows, cin, cout, input stride of the layer); it takes
+ * precedence over prom_debug_tc_plan for that shape.  All five values 0 removes it. */
+void prom_debug_tc_plan_shape(int64_t m, int cin, int cout, int stride, int fold, int nt, int groups,
+                              int occ, int stages);
 int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
 
 /* Frees the library's internal caches (all devices).  Optional. */

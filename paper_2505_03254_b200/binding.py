@@ -28,7 +28,7 @@ EXPORTS = [
     "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
     "prom_launch_count", "prom_shutdown", "prom_status_string",
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
-    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8",
+    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8", "prom_debug_tc_plan_shape",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -94,6 +94,8 @@ def lib():
         L.prom_quantize_act_absmax.restype = i32
         L.prom_quantize_act_absmax.argtypes = [C.c_void_p, i32, i64, C.c_void_p, C.c_void_p, C.c_void_p,
                                                C.c_void_p]
+        L.prom_debug_tc_plan_shape.restype = None
+        L.prom_debug_tc_plan_shape.argtypes = [i64, i32, i32, i32, i32, i32, i32, i32, i32]
         L.prom_debug_tc_plan.restype = None
         L.prom_debug_tc_plan.argtypes = [i32, i32, i32, i32, i32]
         L.prom_debug_tc_plan_query.restype = i32
@@ -210,6 +212,12 @@ def quantize_act_absmax(x: torch.Tensor, out=None, stream=None):
 def debug_tc_plan(fold: int = 0, nt: int = 0, groups: int = 0, occ: int = 0, stages: int = 0) -> None:
     """prom_debug_tc_plan: force parts of the tensor-core launch plan (0 = automatic)."""
     lib().prom_debug_tc_plan(fold, nt, groups, occ, stages)
+
+
+def debug_tc_plan_shape(m: int, cin: int, cout: int, stride: int = 1, fold: int = 0, nt: int = 0,
+                        groups: int = 0, occ: int = 0, stages: int = 0) -> None:
+    """prom_debug_tc_plan_shape: force parts of the plan of one shape (all 0 removes the override)."""
+    lib().prom_debug_tc_plan_shape(m, cin, cout, stride, fold, nt, groups, occ, stages)
 
 
 def debug_tc_plan_query(m: int, cin: int, cout: int):
