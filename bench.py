@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio on B200 (4.5 : 2.25)
 FLUSH_BYTES = 512 << 20       # > 2x the 126 MB L2
-NCU_TRAFFIC_PER_LAUNCH = 15.30e6
+NCU_TRAFFIC_PER_LAUNCH = 15.46e6
 MULHI_LANES_PER_CLK_SM = 31.6   # mul.hi.s32 issue rate measured on B200 (independent chains, all SMs)
 
 

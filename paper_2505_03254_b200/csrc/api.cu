@@ -304,11 +304,14 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
 
 // Picks fold, subtile width, channel groups and occupancy.  Returns false when
 // the tensor-core variant cannot run this shape.
-// dyn: the plan serves the dynamic layer (no row folding: a folded row could straddle two
-// samples; two CTAs per SM)
+// use: kPlanSingle (one call: the kernel builds its operands itself), kPlanDynamic (the dynamic
+// layer: no row folding, a folded row could straddle two samples; two CTAs per SM) or
+// kPlanPrepared (a layer of a sequence, whose operands tc_prep_kernel builds once)
+enum { kPlanSingle = 0, kPlanDynamic = 1, kPlanPrepared = 2 };
 static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
-                           bool dyn, TcPlan &best)
+                           int use, TcPlan &best)
 {
+    const bool dyn = use == kPlanDynamic;
     if (m <= 0 || (cin & 7) || (cout & 7)) return false;
     const TcTune tn = tune_for(m, cin, cout, map.stride);
     int fold = 1;
@@ -319,8 +322,9 @@ static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, co
                m % (fold * 2) == 0)
             fold *= 2;
         // rows of fewer than 32 bytes make poor TMA boxes (measured on the 16 -> 96 layer: 3 us
-        // of 58): fold once more whatever the width
-        if (cin * fold < 32 && fold * 2 <= 8 && m % (fold * 2) == 0) fold *= 2;
+        // of 58): fold once more whatever the width, where the larger block-diagonal weights
+        // are expanded once per sequence and not by every CTA
+        if (use == kPlanPrepared && cin * fold < 32 && fold * 2 <= 8 && m % (fold * 2) == 0) fold *= 2;
     }
     if (dyn) {
         if ((cin & 15) || ((cout & 15) && cout > 256)) return false;
@@ -355,7 +359,7 @@ static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, co
 // The search above costs tens of microseconds; its result depends only on the shape, the
 // device and the tuning override, so it is remembered.
 static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
-                          TcPlan &best, bool dyn = false)
+                          TcPlan &best, int use = kPlanSingle)
 {
     struct Entry { bool ok; TcPlan pl; };
     static std::mutex mu;
@@ -364,12 +368,12 @@ static bool tc_shape_plan(long long m, int cin, int cout, const RowMap &map, con
     cudaGetDevice(&dev);
     const TcTune tn = tune_for(m, cin, cout, map.stride);
     const std::array<long long, 15> key = {m, cin, cout, map.stride, map.ho, map.wo, map.hin, map.win,
-                                           tn.fold, tn.nt, tn.groups, tn.occ, tn.stages, dev, dyn ? 1 : 0};
+                                           tn.fold, tn.nt, tn.groups, tn.occ, tn.stages, dev, use};
     std::lock_guard<std::mutex> lk(mu);
     auto it = cache.find(key);
     if (it == cache.end()) {
         Entry e;
-        e.ok = tc_search_plan(m, cin, cout, map, d, dyn, e.pl);
+        e.ok = tc_search_plan(m, cin, cout, map, d, use, e.pl);
         if (cache.size() > 4096) cache.clear();
         it = cache.emplace(key, e).first;
     }
@@ -587,7 +591,7 @@ static size_t seq_image_bytes(const prom_layer *layers, int n, const SeqShape &s
     for (int i = 0; i < n; ++i) {
         TcPlan pl;
         size_t bytes = 0;
-        if (tc_shape_plan(s.m[i], layers[i].cin, layers[i].cout, s.map[i], d, pl))
+        if (tc_shape_plan(s.m[i], layers[i].cin, layers[i].cout, s.map[i], d, pl, kPlanPrepared))
             bytes = round256((size_t)pl.p.groups * pl.p.image_stride);
         if (offsets) offsets->push_back(bytes ? total : (size_t)-1);
         total += bytes;
@@ -650,7 +654,7 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
         c.st = st;
         c.pdl = i > 0;
         c.pdl_next = i + 1 < n;
-        if (want_tc && c.m > 0 && tc_shape_plan(c.m, c.cin, c.cout, c.map, d, plan[i])) {
+        if (want_tc && c.m > 0 && tc_shape_plan(c.m, c.cin, c.cout, c.map, d, plan[i], kPlanPrepared)) {
             is_tc[i] = 1;
             tc_bind(c, plan[i], img_base && img_off[i] != (size_t)-1 ? img_base + img_off[i] : nullptr);
         } else if (variant == PROM_VARIANT_TC && c.m > 0) {
@@ -843,7 +847,7 @@ prom_status prom_pw_conv_i8_dyn(const int8_t *x_dev, int batch, int64_t rows_per
     if (!d.ok) return PROM_ERR_CUDA;
     TcPlan pl;
     const RowMap plain{1, 1, 1, 1, 1};
-    if (!tc_shape_plan(m, cin, cout, plain, d, pl, true)) return PROM_ERR_UNSUPPORTED;
+    if (!tc_shape_plan(m, cin, cout, plain, d, pl, kPlanDynamic)) return PROM_ERR_UNSUPPORTED;
     if (tc_set_attr(d) != PROM_OK) return PROM_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Conv c;
