@@ -210,3 +210,35 @@ def test_largest_channel_counts(oracle):
             ref = got
         else:
             assert np.array_equal(got, ref)
+
+
+def test_seeded_shape_fuzz(oracle):
+    """Sixty seeded random shapes (rows 1..5000, channel counts multiples of 8 up to 640, both
+    clamps, a shift span that forces either epilogue) through AUTO and, where it accepts the
+    shape, the tensor-core variant: the planner's corner cases rather than the network's shapes."""
+    rng = np.random.default_rng(4242)
+    for case in range(60):
+        m = int(rng.integers(1, 5001))
+        cin = 8 * int(rng.integers(1, 81))
+        cout = 8 * int(rng.integers(1, 81))
+        x = synth.act_uniform_i8(900 + case, (m, cin)) if case % 2 else synth.act_uniform_0_127(900 + case, (m, cin))
+        lay = synth.make_layer(900 + case, cin, cout, float(rng.choice([0.3, 0.5, 0.9])))
+        shift = lay["shift"].numpy().copy()
+        if case % 3 == 0:
+            shift[: max(1, cout // 4)] = 2            # a shift span above 4: the exact epilogue
+        lo, hi = (0, 127) if case % 4 else (-128, 127)
+        want = oracle.conv_mul(x.numpy(), lay["w"].numpy(), lay["bias"].numpy(), lay["mult"].numpy(), shift,
+                               act_min=lo, act_max=hi)
+        wp = binding.pack_ternary(lay["w"].cuda())
+        rq = binding.make_requant(lay["bias"].cuda(), lay["mult"].cuda(), torch.from_numpy(shift).cuda(),
+                                  act_min=lo, act_max=hi)
+        for variant in ("auto", "tc"):
+            try:
+                y = binding.pw_conv_i8(x.cuda(), wp, cout, rq, variant=variant)
+            except binding.PromError as e:
+                assert variant == "tc" and e.code == binding.PROM_ERR_UNSUPPORTED, (case, m, cin, cout, variant, e)
+                continue
+            torch.cuda.synchronize()
+            assert binding.last_device_status() == binding.PROM_OK, (case, m, cin, cout, variant)
+            bad = np.argwhere(y.cpu().numpy() != want)
+            assert len(bad) == 0, (case, m, cin, cout, variant, lo, hi, bad[:3].tolist())
