@@ -310,3 +310,53 @@ def test_sequence_twice_and_in_a_cuda_graph(oracle):
         torch.cuda.synchronize()
         assert np.array_equal(y.cpu().numpy(), want)
     assert binding.last_device_status() == binding.PROM_OK
+
+
+def test_seeded_random_stacks(oracle):
+    """Twelve seeded random stacks of 2-6 layers: random channel counts (multiples of 8),
+    strides, image sizes, and a depthwise 3x3 in front of some layers, against the oracle's
+    functions applied layer by layer."""
+    rng = np.random.default_rng(777)
+    for case in range(12):
+        n = int(rng.integers(2, 7))
+        batch = int(rng.integers(1, 4))
+        h = int(rng.choice([8, 12, 16, 24])); w = int(rng.choice([8, 12, 16, 20]))
+        chans = [8 * int(rng.integers(1, 41)) for _ in range(n + 1)]
+        host, dev = [], []
+        hh, ww = h, w
+        for i in range(n):
+            stride = 2 if (hh % 2 == 0 and ww % 2 == 0 and hh >= 4 and ww >= 4 and rng.random() < 0.35) else 1
+            hh //= stride; ww //= stride
+            d = synth.make_layer(500 + case, chans[i], chans[i + 1], 0.5, index=i + 1)
+            hl = dict(cin=chans[i], cout=chans[i + 1], in_stride=stride, w=d["w"].numpy(), bias=d["bias"].numpy(),
+                      mult=d["mult"].numpy(), shift=d["shift"].numpy())
+            dl = dict(cin=chans[i], cout=chans[i + 1], in_stride=stride, w_packed=binding.pack_ternary(d["w"].cuda()),
+                      bias=d["bias"].cuda(), mult=d["mult"].cuda(), shift=d["shift"].cuda())
+            if rng.random() < 0.4:
+                c = chans[i]
+                hl["dw_w"] = rng.integers(-30, 31, size=(c, 3, 3)).astype(np.int8)
+                hl["dw_bias"] = rng.integers(-64, 65, size=c).astype(np.int32)
+                hl["dw_mult"] = rng.integers(1 << 30, (1 << 31) - 1, size=c).astype(np.int32)
+                hl["dw_shift"] = rng.integers(5, 8, size=c).astype(np.int8)
+                for k in ("dw_w", "dw_bias", "dw_mult", "dw_shift"):
+                    dl[k] = torch.from_numpy(hl[k]).cuda()
+            host.append(hl); dev.append(dl)
+        seq = binding.LayerSeq(dev)
+        x0 = synth.act_post_relu6(500 + case, (batch, h, w, chans[0]))
+        ws = torch.empty((max(seq.workspace_bytes(batch, h, w), 16),), dtype=torch.uint8, device="cuda")
+        y = binding.pw_layer_seq(seq, x0.cuda(), ws)
+        torch.cuda.synchronize()
+        assert binding.last_device_status() == binding.PROM_OK, case
+        cur = x0.numpy()
+        for hl in host:
+            if "dw_w" in hl:
+                cur = oracle.dw3x3(cur, hl["dw_w"], hl["dw_bias"], hl["dw_mult"], hl["dw_shift"],
+                                   stride=hl["in_stride"], act_min=0, act_max=127)
+            elif hl["in_stride"] != 1:
+                cur = oracle.subsample(cur, hl["in_stride"])
+            b, ch_h, ch_w, c = cur.shape
+            cur = oracle.conv_mul(cur.reshape(-1, c), hl["w"], hl["bias"], hl["mult"], hl["shift"]).reshape(
+                b, ch_h, ch_w, hl["cout"])
+        got = y.cpu().numpy()
+        assert got.shape == cur.shape, (case, got.shape, cur.shape)
+        assert np.array_equal(got, cur), (case, [(l["cin"], l["cout"], l["in_stride"], "dw_w" in l) for l in host])
