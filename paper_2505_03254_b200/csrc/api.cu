@@ -305,7 +305,7 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
 // Picks fold, subtile width, channel groups and occupancy.  Returns false when
 // the tensor-core variant cannot run this shape.
 // use: kPlanSingle (one call: the kernel builds its operands itself), kPlanDynamic (the dynamic
-// layer: no row folding, a folded row could straddle two samples; two CTAs per SM) or
+// layer: no row folding, a folded row could straddle two samples) or
 // kPlanPrepared (a layer of a sequence, whose operands tc_prep_kernel builds once)
 enum { kPlanSingle = 0, kPlanDynamic = 1, kPlanPrepared = 2 };
 static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
@@ -343,7 +343,7 @@ static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, co
             if (tn.groups > 0 && groups != tn.groups) continue;
             for (int occ = 4; occ >= 1; --occ) {
                 if (tn.occ > 0 && occ != tn.occ) continue;
-                if (dyn && occ != 2) continue;
+                if (dyn && occ > 2) continue;
                 if (tn.occ == 0 && occ >= 3) continue;      // only on request for now
                 TcPlan pl;
                 if (!tc_fill_plan(m, cin, cout, map, d, fold, nt, groups, occ, tn.stages, pl))

@@ -81,3 +81,11 @@ def test_refusals_and_degenerate_inputs(oracle):
     _run(oracle, x, w, alpha, gx, 100)
     # twice in a row on the same buffers
     _run(oracle, x, w, alpha, gx, 100)
+
+
+def test_seeded_shape_fuzz(oracle):
+    rng = np.random.default_rng(98)
+    for case in range(16):
+        batch = int(rng.integers(1, 9)); rows = int(rng.integers(1, 700))
+        cin = 16 * int(rng.integers(1, 25)); cout = 8 * int(rng.integers(1, 33))
+        _run(oracle, *_case(200 + case, batch, rows, cin, cout), rows)

@@ -58,3 +58,13 @@ def test_refusals():
     with pytest.raises(binding.PromError) as e:
         binding.dw_conv3x3_i8(x, w, rq)
     assert e.value.code == binding.PROM_ERR_UNSUPPORTED
+
+
+def test_seeded_shape_fuzz(oracle):
+    rng = np.random.default_rng(99)
+    for case in range(24):
+        b = int(rng.integers(1, 4)); h = int(rng.integers(1, 40)); w = int(rng.integers(1, 40))
+        c = 4 * int(rng.integers(1, 80))
+        stride = int(rng.choice([1, 2]))
+        lo, hi = (0, 127) if case % 2 else (-128, 127)
+        _run(oracle, *_case(100 + case, b, h, w, c), stride, lo, hi)
