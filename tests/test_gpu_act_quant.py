@@ -76,3 +76,20 @@ def test_repeated_calls_and_empty_batch(oracle):
     e = torch.empty((0, 16), dtype=torch.float32, device="cuda")
     q, g, s = binding.quantize_act_absmax(e)
     assert q.shape == (0, 16) and g.numel() == 0
+
+
+def test_seeded_shape_fuzz(oracle):
+    """Random batch sizes and sample sizes across all three routes (multiples of 16 small and
+    large, and sizes that are not)."""
+    rng = np.random.default_rng(97)
+    for case in range(20):
+        batch = int(rng.integers(1, 40))
+        kind = case % 3
+        if kind == 0:
+            per = 16 * int(rng.integers(1, 4000))
+        elif kind == 1:
+            per = int(rng.integers(1, 50000))
+        else:
+            per = 16 * int(rng.integers(30000, 60000))          # beyond a cluster's shared memory
+            batch = min(batch, 4)
+        _check(oracle, _input(300 + case, (batch, per)))
