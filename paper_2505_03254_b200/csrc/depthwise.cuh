@@ -60,6 +60,10 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
         if (!requant_ok(cb[k], cm[k], cs[k])) { bad = true; cb[k] = 0; cm[k] = 0; cs[k] = 0; }
     }
     if (bad) raise_status(PROM_ERR_BAD_REQUANT);
+    const bool relu127 = lo == 0 && hi == 127;
+    int cb4[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) cb4[k] = cb[k] * 4;
 
     constexpr int kCols = STRIDE * (kStrip - 1) + 3;      // input columns under a strip
     const size_t pix = (size_t)c;                         // bytes from a pixel to the next
@@ -114,20 +118,38 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
 #pragma unroll
         for (int o = 0; o < kStrip; ++o) {
             if (j0 + o < wo) {
-                int q[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int t = acc[o][k] + cb[k];
-                    q[k] = lo >= 0 ? requant_floor(t, cm[k], cs[k], lo, hi)
-                                   : requant_exact(t, cm[k], cs[k], lo, hi);
-                }
-                // already within [-128, 127]: the saturating packs only gather the low bytes
                 uint32_t out;
-                asm("{\n\t.reg .b32 t;\n\t"
-                    "cvt.pack.sat.s8.s32.b32 t, %4, %3, 0;\n\t"
-                    "cvt.pack.sat.s8.s32.b32 %0, %2, %1, t;\n\t}"
-                    : "=r"(out)
-                    : "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3]));
+                if (relu127) {
+                    // clamp [0, 127]: negative values clamp to 0 under either rounding, so the
+                    // nested floors ((hi32((4 t) * mult) >> shift) + 1) >> 1 apply; the value is
+                    // kept at twice its scale through a saturating pack to [0, 255] and halved
+                    // with a mask, which is the clamp at 127
+                    int q2[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        q2[k] = (__mulhi(acc[o][k] * 4 + cb4[k], cm[k]) >> cs[k]) + 1;
+                    uint32_t wv;
+                    asm("{\n\t.reg .b32 t;\n\t"
+                        "cvt.pack.sat.u8.s32.b32 t, %4, %3, 0;\n\t"
+                        "cvt.pack.sat.u8.s32.b32 %0, %2, %1, t;\n\t}"
+                        : "=r"(wv)
+                        : "r"(q2[0]), "r"(q2[1]), "r"(q2[2]), "r"(q2[3]));
+                    out = (wv >> 1) & 0x7F7F7F7Fu;
+                } else {
+                    int q[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int t = acc[o][k] + cb[k];
+                        q[k] = lo >= 0 ? requant_floor(t, cm[k], cs[k], lo, hi)
+                                       : requant_exact(t, cm[k], cs[k], lo, hi);
+                    }
+                    // already within [-128, 127]: the saturating packs only gather the low bytes
+                    asm("{\n\t.reg .b32 t;\n\t"
+                        "cvt.pack.sat.s8.s32.b32 t, %4, %3, 0;\n\t"
+                        "cvt.pack.sat.s8.s32.b32 %0, %2, %1, t;\n\t}"
+                        : "=r"(out)
+                        : "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3]));
+                }
                 *reinterpret_cast<uint32_t *>(yrow + (size_t)o * pix) = out;
             }
         }
