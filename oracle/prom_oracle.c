@@ -218,6 +218,24 @@ void prom_ref_subsample(const int8_t *in, int batch, int h, int w, int c,
                        (size_t)c);
 }
 
+/*
+ * The skip connection of an inverted-residual block (Section 2): when a
+ * block keeps the shape of its input, the input is added to the output of
+ * the project convolution.  Both tensors are int8 on one scale here (the
+ * paper adds in floating point after dequantising), so the sum is the
+ * integer sum clamped to the int8 range.
+ */
+void prom_ref_residual_add(const int8_t *y_layer, const int8_t *block_in, long n,
+                           int8_t *out)
+{
+    for (long i = 0; i < n; ++i) {
+        int s = (int)y_layer[i] + (int)block_in[i];
+        if (s < -128) s = -128;
+        if (s > 127) s = 127;
+        out[i] = (int8_t)s;
+    }
+}
+
 /* ---- the layer sequence -------------------------------------------------- */
 /*
  * Runs n pointwise layers back to back: the output of layer i is the input

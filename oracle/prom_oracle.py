@@ -51,6 +51,7 @@ def lib():
         L.prom_ref_conv_mul.argtypes = conv
         L.prom_ref_conv_addsub.argtypes = conv
         L.prom_ref_subsample.argtypes = [i8p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, i8p]
+        L.prom_ref_residual_add.argtypes = [i8p, i8p, C.c_long, i8p]
         L.prom_ref_layer_seq.restype = C.c_int
         L.prom_ref_layer_seq.argtypes = [
             C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int),
@@ -164,6 +165,15 @@ def subsample(x, stride: int) -> np.ndarray:
     b, h, w, c = x.shape
     out = np.empty((b, h // stride, w // stride, c), dtype=np.int8)
     lib().prom_ref_subsample(_p(x, C.c_int8), b, h, w, c, stride, _p(out, C.c_int8))
+    return out
+
+
+def residual_add(y_layer, block_in) -> np.ndarray:
+    """Skip connection (Section 2): clamp(y_layer + block_in, -128, 127), int8 arrays of one shape."""
+    a, b = _c(y_layer, np.int8), _c(block_in, np.int8)
+    assert a.shape == b.shape
+    out = np.empty_like(a)
+    lib().prom_ref_residual_add(_p(a, C.c_int8), _p(b, C.c_int8), a.size, _p(out, C.c_int8))
     return out
 
 
