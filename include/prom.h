@@ -93,7 +93,14 @@ typedef struct {
  * depthwise 3x3 convolution of prom_dw_conv3x3_i8 (weights dw_w [cin][3][3],
  * constants dw_rq, stride in_stride) runs on the layer's input first and the
  * pointwise convolution reads its output; the input's height and width must
- * then be multiples of in_stride. */
+ * then be multiples of in_stride.  With add_block_input nonzero the input of
+ * the previous layer (in an inverted-residual block, Section 2: the block's
+ * input, when this layer is the project convolution and the previous one the
+ * expand convolution) is added to this layer's output as in
+ * prom_pw_conv_i8_res; both layers must then have in_stride 1 and this
+ * layer's cout must equal the previous layer's cin (PROM_ERR_SHAPE
+ * otherwise), and the variants SMALLK and ADDSUB refuse the sequence
+ * (PROM_ERR_UNSUPPORTED). */
 typedef struct {
     int cin, cout;
     int in_stride;
@@ -101,6 +108,7 @@ typedef struct {
     prom_requant rq;
     const int8_t *dw_w;        /* device, or NULL: no depthwise convolution in front */
     prom_requant dw_rq;        /* read only when dw_w is set */
+    int add_block_input;       /* nonzero: add the previous layer's input to the output */
 } prom_layer;
 
 /* Bytes of the 2-bit form of a [cout][cin] ternary matrix: cout*ceil(cin/4).
@@ -221,6 +229,25 @@ prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin,
                             const uint8_t *w_packed_dev, int cout,
                             const prom_requant *rq, int8_t *y_dev,
                             prom_variant variant, void *cuda_stream);
+
+/* The project convolution of an inverted-residual block with the block's
+ * skip connection (Section 2): the layer of prom_pw_conv_i8, then
+ *   y[r][o] = clamp(y[r][o] + res[r][o], -128, 127),
+ * both terms on the output's scale (the requantisation constants are chosen
+ * so; the paper adds in floating point after dequantising).  The kernel adds
+ * in its epilogue: the sum costs one more read of m*cout bytes and no pass of
+ * its own.
+ *   res_dev  [m][cout] int8, 16-byte aligned base; it may be y_dev itself
+ *            (the sum is then formed in place) but must not overlap y_dev
+ *            in any other way, nor x_dev at all
+ * Everything else as in prom_pw_conv_i8.  Variants: AUTO, TC and NAIVE; SMALLK
+ * and ADDSUB return PROM_ERR_UNSUPPORTED, and AUTO falls back on NAIVE where
+ * TC does not apply. */
+prom_status prom_pw_conv_i8_res(const int8_t *x_dev, int64_t m, int cin,
+                                const uint8_t *w_packed_dev, int cout,
+                                const prom_requant *rq, const int8_t *res_dev,
+                                int8_t *y_dev, prom_variant variant,
+                                void *cuda_stream);
 
 /* Test/debug: the raw accumulators acc[m][cout] (int32) of the same layer,
  * computed by the plain one-thread-per-output kernel. */

@@ -28,7 +28,7 @@ EXPORTS = [
     "prom_layer_seq_host_workspace_bytes", "prom_pw_layer_seq_host", "prom_last_device_status",
     "prom_launch_count", "prom_shutdown", "prom_status_string",
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
-    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8", "prom_debug_tc_plan_shape",
+    "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8", "prom_debug_tc_plan_shape", "prom_pw_conv_i8_res",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -41,7 +41,7 @@ class PromRequant(C.Structure):
 class PromLayer(C.Structure):
     _fields_ = [("cin", C.c_int), ("cout", C.c_int), ("in_stride", C.c_int),
                 ("w_packed", C.c_void_p), ("rq", PromRequant),
-                ("dw_w", C.c_void_p), ("dw_rq", PromRequant)]
+                ("dw_w", C.c_void_p), ("dw_rq", PromRequant), ("add_block_input", C.c_int)]
 
 
 class PromError(RuntimeError):
@@ -67,6 +67,8 @@ def lib():
         L.prom_pack_ternary.argtypes = [vp, i32, i32, vp, sz, vp]
         L.prom_pw_conv_i8.restype = i32
         L.prom_pw_conv_i8.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant), vp, i32, vp]
+        L.prom_pw_conv_i8_res.restype = i32
+        L.prom_pw_conv_i8_res.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant), vp, vp, i32, vp]
         L.prom_pw_conv_i8_acc32.restype = i32
         L.prom_pw_conv_i8_acc32.argtypes = [vp, i64, i32, vp, i32, vp, vp]
         L.prom_pw_conv_i8_host.restype = i32
@@ -282,6 +284,24 @@ def pw_conv_i8(x: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequa
     return y
 
 
+def pw_conv_i8_res(x: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequant,
+                   res: torch.Tensor, y: Optional[torch.Tensor] = None, variant="auto",
+                   stream=None) -> torch.Tensor:
+    """prom_pw_conv_i8_res: the layer plus the int8 tensor `res` ([m, cout]) with saturation;
+    pass y=res to form the sum in place."""
+    m, cin = x.shape
+    if tuple(res.shape) != (m, cout):
+        raise ValueError("res must be [m, cout]")
+    if y is None:
+        y = torch.empty((m, cout), dtype=torch.int8, device=x.device)
+    _check(lib().prom_pw_conv_i8_res(_dev(x, torch.int8, "x"), m, cin,
+                                     _dev(w_packed, torch.uint8, "w_packed"), cout, C.byref(rq),
+                                     _dev(res, torch.int8, "res"), _dev(y, torch.int8, "y"),
+                                     _variant(variant), _stream(stream)),
+           "prom_pw_conv_i8_res")
+    return y
+
+
 def pw_conv_i8_addsub_static(x: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequant,
                              y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
     """prom_pw_conv_i8_addsub_static: the add/sub variant on the library's built-in
@@ -332,7 +352,10 @@ class LayerSeq:
                 self._keep.append(l[k])
             self.array[i] = PromLayer(int(l["cin"]), int(l["cout"]), int(l["in_stride"]),
                                       _dev(l["w_packed"], torch.uint8, "w_packed"),
-                                      make_requant(l["bias"], l["mult"], l["shift"], act_min, act_max))
+                                      make_requant(l["bias"], l["mult"], l["shift"],
+                                                   int(l.get("act_min", act_min)),
+                                                   int(l.get("act_max", act_max))))
+            self.array[i].add_block_input = 1 if l.get("add_block_input") else 0
             if l.get("dw_w") is not None:
                 # a real depthwise 3x3 in front: int8 [cin, 3, 3] weights and their constants
                 for k in ("dw_w", "dw_bias", "dw_mult", "dw_shift"):

@@ -68,6 +68,7 @@ struct Conv {
     cudaStream_t st;
     bool pdl;           // chain to the previous kernel with programmatic dependent launch
     bool pdl_next;      // the next kernel of the sequence chains to this one
+    const int8_t *res = nullptr;   // added to the output with int8 saturation (may be y)
 };
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -119,7 +120,8 @@ static prom_status launch_naive(const Conv &c, int32_t *acc_out)
     int grid = grid_for(c.m * c.cout, threads, d.sms);
     naive_conv_kernel<<<grid, threads, 0, c.st>>>(c.x, c.m, c.cin, c.map, c.w, c.cout, c.rq.bias,
                                                   c.rq.mult, c.rq.shift, c.rq.act_min,
-                                                  c.rq.act_max, acc_out ? nullptr : c.y, acc_out);
+                                                  c.rq.act_max, acc_out ? nullptr : c.y, acc_out,
+                                                  acc_out ? nullptr : c.res);
     ++g_launches;
     return cuda_status(cudaGetLastError());
 }
@@ -445,6 +447,10 @@ static prom_status tc_set_attr(const DeviceInfo &d)
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             d.smem_optin);
         if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 3>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            d.smem_optin);
+        if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(tc::tc_prep_kernel,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             d.smem_optin);
@@ -460,6 +466,7 @@ static void tc_bind(const Conv &c, TcPlan &pl, uint8_t *image)
     p.act_min = c.rq.act_min; p.act_max = c.rq.act_max; p.y = c.y; p.pdl = c.pdl ? 1 : 0;
     p.pdl_next = c.pdl_next ? 1 : 0;
     p.image = image;
+    p.res = c.res;
 }
 
 static prom_status tc_launch_planned(const Conv &c, TcPlan &pl, int mode = 0)
@@ -481,6 +488,7 @@ static prom_status tc_launch_planned(const Conv &c, TcPlan &pl, int mode = 0)
     cudaError_t e;
     if (mode == 1) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 1>, pl.xmap, pl.ymap, pl.p);
     else if (mode == 2) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 2>, pl.xmap, pl.ymap, pl.p);
+    else if (c.res) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 3>, pl.xmap, pl.ymap, pl.p);
     else if (pl.per_sm == 3) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<3>, pl.xmap, pl.ymap, pl.p);
     else e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2>, pl.xmap, pl.ymap, pl.p);
     ++g_launches;
@@ -510,6 +518,8 @@ static bool tc_supported(const Conv &c)
 static prom_status run_conv(const Conv &c, prom_variant v)
 {
     if (c.m == 0) return PROM_OK;
+    // the residual is fused into the tensor-core and the naive kernels only
+    if (c.res && (v == PROM_VARIANT_SMALLK || v == PROM_VARIANT_ADDSUB)) return PROM_ERR_UNSUPPORTED;
     switch (v) {
     case PROM_VARIANT_NAIVE: return launch_naive(c, nullptr);
     case PROM_VARIANT_TC: return launch_tc(c);
@@ -519,7 +529,7 @@ static prom_status run_conv(const Conv &c, prom_variant v)
                                                     c.st, g_launches);
     case PROM_VARIANT_AUTO:
         if (tc_supported(c)) return launch_tc(c);
-        if (smallk::supported(c.cin, c.cout))
+        if (!c.res && smallk::supported(c.cin, c.cout))
             return smallk::launch(c.x, c.m, c.cin, c.map, c.w, c.cout, c.rq, c.y, c.st, g_launches);
         return launch_naive(c, nullptr);
     default: return PROM_ERR_UNSUPPORTED;
@@ -545,6 +555,10 @@ static bool seq_shapes(const prom_layer *layers, int n, int batch, int h0, int w
         if (i > 0 && l.cin != layers[i - 1].cout) return false;
         if (l.in_stride != 1 && l.in_stride != 2) return false;
         if (h % l.in_stride || w % l.in_stride) return false;
+        // the block's input (the previous layer's input) has this layer's output shape
+        if (l.add_block_input &&
+            (i < 1 || l.in_stride != 1 || layers[i - 1].in_stride != 1 || l.cout != layers[i - 1].cin))
+            return false;
         RowMap mp;
         mp.stride = l.in_stride; mp.hin = h; mp.win = w;
         h /= l.in_stride; w /= l.in_stride;
@@ -627,6 +641,9 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
         prom_status e = check_requant(&layers[i].rq);
         if (e != PROM_OK) return e;
         if (!aligned16(layers[i].w_packed)) return PROM_ERR_ALIGN;
+        if (layers[i].add_block_input &&
+            (variant == PROM_VARIANT_SMALLK || variant == PROM_VARIANT_ADDSUB))
+            return PROM_ERR_UNSUPPORTED;
     }
     DeviceInfo d = device_info();
     if (!d.ok) return PROM_ERR_CUDA;
@@ -654,6 +671,9 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
         c.st = st;
         c.pdl = i > 0;
         c.pdl_next = i + 1 < n;
+        // The block's input is the output of layer i-2, which sits where this layer's output
+        // goes: the sum is formed in place.
+        if (layers[i].add_block_input) c.res = i == 1 ? x0 : conv[i - 2].y;
         if (want_tc && c.m > 0 && tc_shape_plan(c.m, c.cin, c.cout, c.map, d, plan[i], kPlanPrepared)) {
             is_tc[i] = 1;
             tc_bind(c, plan[i], img_base && img_off[i] != (size_t)-1 ? img_base + img_off[i] : nullptr);
@@ -1043,6 +1063,28 @@ prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin, const uint8
     c.st = static_cast<cudaStream_t>(cuda_stream);
     c.pdl = false;
     c.pdl_next = false;
+    return run_conv(c, variant);
+}
+
+prom_status prom_pw_conv_i8_res(const int8_t *x_dev, int64_t m, int cin, const uint8_t *w_packed_dev,
+                                int cout, const prom_requant *rq, const int8_t *res_dev,
+                                int8_t *y_dev, prom_variant variant, void *cuda_stream)
+{
+    if (m == 0 && cin >= 1 && cin <= 4096 && cout >= 1 && cout <= 4096 && w_packed_dev && rq)
+        return check_requant(rq);
+    prom_status s = check_conv(x_dev, m, cin, w_packed_dev, cout, rq, y_dev);
+    if (s != PROM_OK) return s;
+    if (!res_dev) return PROM_ERR_NULL;
+    if (!aligned16(res_dev)) return PROM_ERR_ALIGN;
+    Conv c;
+    c.x = x_dev; c.m = m; c.cin = cin; c.cout = cout;
+    c.map = RowMap{1, 1, 1, 1, 1};
+    c.in_rows = m;
+    c.w = w_packed_dev; c.rq = *rq; c.y = y_dev;
+    c.st = static_cast<cudaStream_t>(cuda_stream);
+    c.pdl = false;
+    c.pdl_next = false;
+    c.res = res_dev;
     return run_conv(c, variant);
 }
 

@@ -32,13 +32,14 @@ __global__ void pack_ternary_kernel(const int8_t *__restrict__ w, int cout, int 
 }
 
 // One thread per output element; the definition written out.  Either y
-// (requantised int8) or acc_out (raw int32) is produced.
+// (requantised int8, plus res[i] with int8 saturation when res is set; res may be y)
+// or acc_out (raw int32) is produced.
 __global__ void naive_conv_kernel(const int8_t *__restrict__ x, long long m, int cin, RowMap map,
                                   const uint8_t *__restrict__ w_packed, int cout,
                                   const int32_t *__restrict__ bias,
                                   const int32_t *__restrict__ mult,
                                   const int8_t *__restrict__ shift, int act_min, int act_max,
-                                  int8_t *__restrict__ y, int32_t *__restrict__ acc_out)
+                                  int8_t *y, int32_t *__restrict__ acc_out, const int8_t *res)
 {
     int rowb = (cin + 3) >> 2;
     long long total = m * cout;
@@ -59,7 +60,12 @@ __global__ void naive_conv_kernel(const int8_t *__restrict__ x, long long m, int
         if (y) {
             int b = bias[o], mu = mult[o], sh = shift[o];
             if (!requant_ok(b, mu, sh)) { raise_status(PROM_ERR_BAD_REQUANT); continue; }
-            y[i] = (int8_t)requant_exact(acc + b, mu, sh, act_min, act_max);
+            int q = requant_exact(acc + b, mu, sh, act_min, act_max);
+            if (res) {
+                q += res[i];
+                q = q < -128 ? -128 : (q > 127 ? 127 : q);
+            }
+            y[i] = (int8_t)q;
         }
     }
 }

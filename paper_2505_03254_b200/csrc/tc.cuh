@@ -86,6 +86,9 @@ struct Params {
     const float *gamma_x;       // [batch] per-sample maximum behind the int8 input
     float *gamma_y;             // [batch] mode 1: maxima of the dequantised output (as bit patterns)
     const float *scale_y;       // [batch] mode 2: 127 / max(gamma_y, eps)
+    // Kernel mode 3: an int8 tensor of Y's shape added to the requantised output with
+    // saturation.  It may be Y itself: a warp reads the bytes of a slab before it stores there.
+    const int8_t *res;
 };
 
 // Bounded wait on an mbarrier phase.  The clock is read only every 1024 polls (a
@@ -620,6 +623,7 @@ __device__ __forceinline__ void build_image(const Params &p, const int g, const 
 // MINB: CTAs of this kernel that share an SM (2 with 96 registers a thread, 3 with 64).
 // MODE 0: static fixed-point requantisation.  MODE 1 and 2: the two passes of the dynamic layer
 // (per-sample maxima of the dequantised output; output quantised with the per-sample scale).
+// MODE 3: mode 0 plus a residual tensor added to the output with int8 saturation.
 template <int MINB, int MODE = 0>
 __global__ void __launch_bounds__(kThreads, MINB)
 tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap ymap,
@@ -858,6 +862,10 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             // scalar instructions issued among many busy warps, tens of cycles each: positions,
             // addresses and phases advance by additions, and a full slab takes the short path.
             const int q = warp & 3;                     // TMEM lane quarter of this warp
+            if constexpr (MODE == 3) {
+                // the residual was written two kernels back: complete once the previous one is
+                if (p.pdl) ptx::grid_dep_wait();
+            }
             // Unit u goes to group u % 2 and accumulator u % nbuf; nbuf is even, so a group meets
             // each of its accumulators in cyclic order and never waits on a barrier that is more
             // than one phase away.
@@ -900,9 +908,28 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 const uint32_t taddr = t_lane + b * p.nt_pad;
                 const int *cms = cmult + ls * p.nt_pad;
                 const uint32_t bar_rel = bar_tempty + 8 * b;
-                if constexpr (MODE == 0) {
+                if constexpr (MODE == 0 || MODE == 3) {
                     if (fast) epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
                     else epi_exact_subtile<CH>(p, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
+                    if constexpr (MODE == 3) {
+                        // The residual: the bytes that sit where this slab goes in Y, read past
+                        // L1 in 8-byte granules across the warp and added to the slab.
+                        __syncwarp();
+                        int rows_valid = p.tm - q * 32;
+                        if (m_rows - row0 < rows_valid) rows_valid = m_rows - row0;
+                        if (rows_valid > 32) rows_valid = 32;
+                        const int g8 = p.nt >> 3;
+                        const int8_t *rp = p.res + (long long)row0 * p.nf + col;
+                        for (int i = lane; i < rows_valid * g8; i += 32) {
+                            const int r = i / g8, c = (i - r * g8) * 8;
+                            const uint2 rv = __ldcg(reinterpret_cast<const uint2 *>(rp + (long long)r * p.nf + c));
+                            uint2 *sp = reinterpret_cast<uint2 *>(slab + r * p.nt + c);
+                            uint2 sv = *sp;
+                            sv.x = __vaddss4(sv.x, rv.x);
+                            sv.y = __vaddss4(sv.y, rv.y);
+                            *sp = sv;
+                        }
+                    }
                 } else {
                     // this thread's row and its sample (rows past the end borrow the last sample's
                     // factors; they are neither counted nor stored)

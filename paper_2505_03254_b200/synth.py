@@ -188,6 +188,14 @@ def mobilenetv2_pointwise_layers(stem_channels: int = 32, h0: int = 112, w0: int
     return layers
 
 
+def has_skip_connection(layers: List[LayerShape], i: int) -> bool:
+    """Whether layer i of `mobilenetv2_pointwise_layers` closes a block that keeps its input's
+    shape (stride 1, equal channel counts): the block's input is then added to its output."""
+    return (i > 0 and layers[i].name.endswith("project") and layers[i - 1].name.endswith("expand")
+            and layers[i].in_stride == 1 and layers[i - 1].in_stride == 1
+            and layers[i].cout == layers[i - 1].cin)
+
+
 def layer_seed(seed: int, index: int) -> int:
     """Seed offset of layer `index` in a sequence (streams 1000*index + s)."""
     return 1000 * index
