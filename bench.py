@@ -435,6 +435,7 @@ def run_gpu(args):
         out["dynamic_layer"] = dynamic_layer_timing(torch, binding, synth, bw)
         out["depthwise"] = depthwise_timing(torch, binding, bw)
         out["body_with_depthwise"] = body_with_depthwise_timing(torch, binding, synth, bw)
+        out["body_with_skip_connections"] = body_with_depthwise_timing(torch, binding, synth, bw, skips=True)
         cold_us = sum(r["us"] for r in out["layers"])
         roofline["sum_layer_cold_us"] = cold_us
         roofline["sum_layer_cold_frac"] = sum(roof_us) / cold_us
@@ -568,11 +569,13 @@ def depthwise_timing(torch, binding, bw):
     return rows
 
 
-def body_with_depthwise_timing(torch, binding, synth, bw):
+def body_with_depthwise_timing(torch, binding, synth, bw, skips=False):
     """The 34 pointwise layers with a real int8 depthwise 3x3 in front of every project
-    convolution (17 of them) in place of the identity stand-in: the body of MobileNetV2 without
-    its residual adds, batch 128, CUDA graph.  Algorithmic bytes: the pointwise layers' plus one
-    byte in and one byte out per depthwise value."""
+    convolution (17 of them) in place of the identity stand-in: the body of MobileNetV2, batch
+    128, CUDA graph.  With `skips` the project layers are linear (clamp [-128, 127]) and the ten
+    blocks that keep their input's shape add it to their output in the project layer's epilogue.
+    Algorithmic bytes: the pointwise layers' plus one byte in and one byte out per depthwise
+    value, plus one byte per output of a block with a skip connection."""
     seed = synth.BASE_SEED + 3
     table, _, dev = build_network(seed, synth, binding, "cuda")
     g = torch.Generator(device="cuda").manual_seed(5)
@@ -587,6 +590,15 @@ def body_with_depthwise_timing(torch, binding, synth, bw):
             d["dw_mult"] = torch.full((c,), 1 << 30, dtype=torch.int32, device="cuda")
             d["dw_shift"] = torch.full((c,), 6, dtype=torch.int8, device="cuda")
             nbytes += m * c * l.in_stride * l.in_stride + m * c
+            if skips:
+                d["act_min"] = -128
+    n_skips = 0
+    if skips:
+        for i, (l, d) in enumerate(zip(table, dev)):
+            if synth.has_skip_connection(table, i):
+                d["add_block_input"] = True
+                nbytes += BATCH * l.h * l.w * l.cout
+                n_skips += 1
     seq = binding.LayerSeq(dev)
     x0 = synth.act_post_relu6(seed, (BATCH, 112, 112, 32), device="cuda")
     ws = torch.empty((seq.workspace_bytes(BATCH, 112, 112),), dtype=torch.uint8, device="cuda")
@@ -601,7 +613,8 @@ def body_with_depthwise_timing(torch, binding, synth, bw):
     for _ in range(3):
         graph.replay()
     ms = time_region(torch, graph.replay, 50, False) / 50
-    return {"workload": "34 pointwise + 17 depthwise 3x3 layers, chained, batch 128",
+    return {"workload": "34 pointwise + 17 depthwise 3x3 layers, chained, batch 128"
+                        + (f", linear project layers, {n_skips} skip connections" if skips else ""),
             "ms_per_step": round(ms, 4), "images_per_s": round(BATCH / ms * 1e3, 1), "bytes": nbytes,
             "roof_us": round(nbytes / bw * 1e6, 1), "frac": round(nbytes / bw * 1e3 / ms, 4),
             "device_status": binding.last_device_status()}
@@ -787,7 +800,8 @@ def run_aux(args):
     elif args.aux == "dynamic_layer":
         out = dynamic_layer_timing(torch, binding, synth, bw)
     elif args.aux == "body":
-        out = body_with_depthwise_timing(torch, binding, synth, bw)
+        out = {"plain": body_with_depthwise_timing(torch, binding, synth, bw),
+               "skips": body_with_depthwise_timing(torch, binding, synth, bw, skips=True)}
     else:
         out = depthwise_timing(torch, binding, bw)
     print(json.dumps({"aux": args.aux, "result": out, "device_status": binding.last_device_status()}))

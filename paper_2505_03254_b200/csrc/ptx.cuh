@@ -225,4 +225,12 @@ __device__ __forceinline__ uint32_t pack_sat_u8(int a, int b, uint32_t c)
     return d;
 }
 
+// (c << 16) | (sat_s8(a) << 8) | sat_s8(b)
+__device__ __forceinline__ uint32_t pack_sat_s8(int a, int b, uint32_t c)
+{
+    uint32_t d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 }}  // namespace prom::ptx

@@ -192,9 +192,17 @@ __device__ __forceinline__ void epi_exact(uint32_t taddr, const int *__restrict_
     put_row<NC>(dst, out, wide);
 }
 
+// One output of the fast epilogue for the full int8 range: the rounding term loses one unit
+// when the product is negative (ties go away from zero), and the shift drops the extra bit.
+__device__ __forceinline__ int fast_signed(int v, int mu, long long r64, int shmax)
+{
+    return (int)(((long long)v * mu + (r64 + (long long)(v >> 31))) >> 32) >> (shmax + 1);
+}
+
 // NC accumulator columns of this thread's row, already in registers: the high word of a
 // 64-bit multiply-add (rounding term in the addend), one shift, saturating pack, halve.
-template <int NC>
+// SIGNED: the clamp is [-128, 127] instead of [0, 127].
+template <int NC, bool SIGNED = false>
 __device__ __forceinline__ void fast_piece(const uint32_t (&v)[NC], const int *__restrict__ cm,
                                            long long r64, int shmax, uint8_t *dst, bool wide)
 {
@@ -202,6 +210,14 @@ __device__ __forceinline__ void fast_piece(const uint32_t (&v)[NC], const int *_
 #pragma unroll
     for (int c = 0; c < NC; c += 4) {
         const int4 mu = *reinterpret_cast<const int4 *>(cm + c);
+        if constexpr (SIGNED) {
+            const int q0 = fast_signed((int)v[c], mu.x, r64, shmax);
+            const int q1 = fast_signed((int)v[c + 1], mu.y, r64, shmax);
+            const int q2 = fast_signed((int)v[c + 2], mu.z, r64, shmax);
+            const int q3 = fast_signed((int)v[c + 3], mu.w, r64, shmax);
+            out[c / 4] = ptx::pack_sat_s8(q1, q0, ptx::pack_sat_s8(q3, q2, 0u));
+            continue;
+        }
         const int q0 = (int)(((long long)(int)v[c] * mu.x + r64) >> 32) >> shmax;
         const int q1 = (int)(((long long)(int)v[c + 1] * mu.y + r64) >> 32) >> shmax;
         const int q2 = (int)(((long long)(int)v[c + 2] * mu.z + r64) >> 32) >> shmax;
@@ -215,7 +231,7 @@ __device__ __forceinline__ void fast_piece(const uint32_t (&v)[NC], const int *_
 
 // The fast epilogue over one subtile, in chunks of CH (32 or 16), then 16 and 8 columns.  The
 // accumulator goes back to the MMA thread as soon as its last columns are in registers.
-template <int CH>
+template <int CH, bool SIGNED = false>
 __device__ __forceinline__ void epi_fast_subtile(const Params &p, uint32_t taddr, const int *cm,
                                                  int shmax, uint8_t *dst_row, uint32_t bar_release)
 {
@@ -228,14 +244,14 @@ __device__ __forceinline__ void epi_fast_subtile(const Params &p, uint32_t taddr
         tmem_ld<CH>(taddr + c, v);
         ptx::tmem_wait_ld();
         if (tail == 0 && c + CH == p.nt) release_acc(bar_release);
-        fast_piece<CH>(v, cm + c, r64, shmax, dst_row + c, wide);
+        fast_piece<CH, SIGNED>(v, cm + c, r64, shmax, dst_row + c, wide);
     }
     if (CH > 16 && c + 16 <= p.nt) {
         uint32_t v[16];
         ptx::tmem_ld_x16(taddr + c, v);
         ptx::tmem_wait_ld();
         if (c + 16 == p.nt) release_acc(bar_release);
-        fast_piece<16>(v, cm + c, r64, shmax, dst_row + c, wide);
+        fast_piece<16, SIGNED>(v, cm + c, r64, shmax, dst_row + c, wide);
         c += 16;
     }
     if (c + 8 <= p.nt) {
@@ -243,7 +259,7 @@ __device__ __forceinline__ void epi_fast_subtile(const Params &p, uint32_t taddr
         ptx::tmem_ld_x8(taddr + c, v);
         ptx::tmem_wait_ld();
         release_acc(bar_release);
-        fast_piece<8>(v, cm + c, r64, shmax, dst_row + c, wide);
+        fast_piece<8, SIGNED>(v, cm + c, r64, shmax, dst_row + c, wide);
     }
 }
 
@@ -523,8 +539,8 @@ __device__ __forceinline__ void build_image(const Params &p, const int g, const 
     __syncthreads();
     const int shmax = flags[2];
     const bool bad_consts = flags[3] != 0;
-    const bool fast = flags[4] == 0 && p.act_min == 0 && p.act_max == 127 && shmax - flags[1] <= 4 &&
-                      shmax <= 24;
+    const bool fast = !p.dyn && flags[4] == 0 && (p.act_min == 0 || p.act_min == -128) && p.act_max == 127 &&
+                      shmax - flags[1] <= 4 && shmax <= 24;
 
     // bias digits of the resident channels (fast path): row n of a 32-byte-swizzled block
     if (fast)
@@ -909,7 +925,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 const int *cms = cmult + ls * p.nt_pad;
                 const uint32_t bar_rel = bar_tempty + 8 * b;
                 if constexpr (MODE == 0 || MODE == 3) {
-                    if (fast) epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
+                    if (fast && p.act_min == 0) epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
+                    else if (fast) epi_fast_subtile<CH, true>(p, taddr, cms, shmax, my_row, bar_rel);
                     else epi_exact_subtile<CH>(p, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
                     if constexpr (MODE == 3) {
                         // The residual: the bytes that sit where this slab goes in Y, read past

@@ -110,6 +110,32 @@ def test_ties_on_device(oracle, variant):
         assert first_mismatch(got, oracle_y(oracle, x, lay, lo, hi)) is None
 
 
+@pytest.mark.parametrize("variant", ["tc", "naive"])
+def test_small_negative_ties_with_the_full_int8_clamp(oracle, variant):
+    """One-hot weight rows (an output is +-1 times one input value, plus a small bias) with
+    mult = 2^30 and shifts 0..4: outputs inside [-128, 127] that sit on ties of either sign,
+    which round away from zero."""
+    m, cin, cout = 512, 32, 32
+    x = synth.act_uniform_i8(19, (m, cin))
+    lay = synth.make_layer(19, cin, cout, 0.5)
+    w = torch.zeros((cout, cin), dtype=torch.int8)
+    for o in range(cout):
+        w[o, (5 * o) % cin] = 1 if o % 3 else -1
+    lay["w"] = w
+    lay["bias"] = (torch.arange(cout, dtype=torch.int32) % 5) - 2
+    lay["mult"] = torch.full((cout,), 1 << 30, dtype=torch.int32)
+    lay["shift"] = (torch.arange(cout) % 5).to(torch.int8)
+    xd, wp, consts = to_device(x, lay)
+    want = oracle_y(oracle, x, lay, -128, 127)
+    t = (x.numpy().astype(np.int64) @ w.numpy().T.astype(np.int64)) + lay["bias"].numpy()
+    sh = lay["shift"].numpy().astype(np.int64) + 1
+    ties = (t % (1 << sh)) == (1 << (sh - 1))
+    assert (ties & (t < 0)).sum() > 100 and (ties & (t > 0)).sum() > 100
+    assert np.array_equal(want[ties], (np.sign(t) * ((np.abs(t) + (1 << (sh - 1))) >> sh))[ties])
+    got = run_variant(xd, wp, consts, cout, variant, -128, 127)
+    assert first_mismatch(got, want) is None
+
+
 def test_extreme_values(oracle):
     """All activations -128 against all +1 / all -1 weights at Cin = 960."""
     m, cin, cout = 130, 960, 16
