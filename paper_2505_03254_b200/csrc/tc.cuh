@@ -911,6 +911,35 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             uint32_t b = (uint32_t)grp, tph = 0;
             uint32_t st = (uint32_t)grp % (uint32_t)p.stages;    // stage of this group's unit (epi_frees)
             while (row0 < row_end && ok) {
+                // The residual (mode 3): the bytes that sit where this slab goes in Y, in 8-byte
+                // granules across the warp.  The first kResHeld granules of a lane are requested
+                // before the wait for the accumulator, so that their latency hides behind it.
+                constexpr int kResHeld = 4;
+                uint2 res_held[kResHeld];
+                int res_total = 0, res_g8 = 1;
+                const int8_t *res_p = nullptr;
+                if constexpr (MODE == 3) {
+                    int rows_valid = p.tm - q * 32;
+                    if (m_rows - row0 < rows_valid) rows_valid = m_rows - row0;
+                    if (rows_valid > 32) rows_valid = 32;
+                    res_g8 = p.nt >> 3;
+                    res_total = rows_valid * res_g8;
+                    res_p = p.res + (long long)row0 * p.nf + col;
+#pragma unroll
+                    for (int j = 0; j < kResHeld; ++j) {
+                        const int i = lane + 32 * j;
+                        res_held[j] = make_uint2(0u, 0u);
+                        if (i < res_total) {
+                            const int r = i / res_g8, c = (i - r * res_g8) * 8;
+                            res_held[j] = __ldcg(reinterpret_cast<const uint2 *>(res_p + (long long)r * p.nf + c));
+                        }
+                    }
+                    // the rest is asked into L2
+                    for (int i = lane + 32 * kResHeld; i < res_total; i += 32) {
+                        const int r = i / res_g8, c = (i - r * res_g8) * 8;
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(res_p + (long long)r * p.nf + c));
+                    }
+                }
                 if (!wait_bar<true>(bar_tfull + 8 * b, tph, flags)) { ok = false; break; }
                 if (epi_frees) {
                     if (q == 0 && lane == 0) ptx::mbar_arrive(bar_empty + 8 * st);
@@ -929,22 +958,21 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                     else if (fast) epi_fast_subtile<CH, true>(p, taddr, cms, shmax, my_row, bar_rel);
                     else epi_exact_subtile<CH>(p, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
                     if constexpr (MODE == 3) {
-                        // The residual: the bytes that sit where this slab goes in Y, read past
-                        // L1 in 8-byte granules across the warp and added to the slab.
                         __syncwarp();
-                        int rows_valid = p.tm - q * 32;
-                        if (m_rows - row0 < rows_valid) rows_valid = m_rows - row0;
-                        if (rows_valid > 32) rows_valid = 32;
-                        const int g8 = p.nt >> 3;
-                        const int8_t *rp = p.res + (long long)row0 * p.nf + col;
-                        for (int i = lane; i < rows_valid * g8; i += 32) {
-                            const int r = i / g8, c = (i - r * g8) * 8;
-                            const uint2 rv = __ldcg(reinterpret_cast<const uint2 *>(rp + (long long)r * p.nf + c));
+                        auto add_to_slab = [&](int i, uint2 rv) {
+                            const int r = i / res_g8, c = (i - r * res_g8) * 8;
                             uint2 *sp = reinterpret_cast<uint2 *>(slab + r * p.nt + c);
                             uint2 sv = *sp;
                             sv.x = __vaddss4(sv.x, rv.x);
                             sv.y = __vaddss4(sv.y, rv.y);
                             *sp = sv;
+                        };
+#pragma unroll
+                        for (int j = 0; j < kResHeld; ++j)
+                            if (lane + 32 * j < res_total) add_to_slab(lane + 32 * j, res_held[j]);
+                        for (int i = lane + 32 * kResHeld; i < res_total; i += 32) {
+                            const int r = i / res_g8, c = (i - r * res_g8) * 8;
+                            add_to_slab(i, __ldcg(reinterpret_cast<const uint2 *>(res_p + (long long)r * p.nf + c)));
                         }
                     }
                 } else {
