@@ -447,6 +447,10 @@ static prom_status tc_set_attr(const DeviceInfo &d)
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             d.smem_optin);
         if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 4>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            d.smem_optin);
+        if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 3>,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             d.smem_optin);
@@ -489,6 +493,8 @@ static prom_status tc_launch_planned(const Conv &c, TcPlan &pl, int mode = 0)
     if (mode == 1) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 1>, pl.xmap, pl.ymap, pl.p);
     else if (mode == 2) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 2>, pl.xmap, pl.ymap, pl.p);
     else if (c.res) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 3>, pl.xmap, pl.ymap, pl.p);
+    else if (pl.p.act_min == -128 && pl.p.act_max == 127)
+        e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2, 4>, pl.xmap, pl.ymap, pl.p);
     else if (pl.per_sm == 3) e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<3>, pl.xmap, pl.ymap, pl.p);
     else e = cudaLaunchKernelEx(&cfg, tc::tc_conv_kernel<2>, pl.xmap, pl.ymap, pl.p);
     ++g_launches;
