@@ -833,8 +833,10 @@ prom_status prom_dw_conv3x3_i8(const int8_t *x_dev, int batch, int h, int w, int
     if ((long long)batch * h * w * c >= (1ll << 40)) return PROM_ERR_SHAPE;
     DeviceInfo d = device_info();
     if (!d.ok) return PROM_ERR_CUDA;
-    if ((long long)batch * ho * ((wo + dw::kStrip - 1) / dw::kStrip) >= (1ll << 31)) return PROM_ERR_SHAPE;
-    const long long total = (long long)batch * ho * ((wo + dw::kStrip - 1) / dw::kStrip) * (c >> 2);
+    const int rows = dw::rows_per_unit(stride);
+    const long long units = (long long)batch * ((ho + rows - 1) / rows) * ((wo + dw::kStrip - 1) / dw::kStrip);
+    if (units >= (1ll << 31)) return PROM_ERR_SHAPE;
+    const long long total = units * (c >> 2);
     // a multiple of c / 4 threads, so that a thread keeps its channels: blocks in multiples of
     // (c / 4) / gcd(c / 4, threads per block)
     int step = c >> 2;
