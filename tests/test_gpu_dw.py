@@ -50,6 +50,27 @@ def test_signed_clamp_and_extreme_values(oracle):
     _run(oracle, *_case(33, 1, 6, 6, 32, extreme=True), 1, 0, 127)
 
 
+@pytest.mark.parametrize("stride", [1, 2])
+@pytest.mark.parametrize("lo", [0, -128])
+def test_small_and_mixed_shifts_and_large_biases(oracle, stride, lo):
+    """Shifts 0..3 (below 2 the requantiser keeps two more bits of the product), mixed within a
+    thread's four channels, small weights so that outputs stay inside the clamp, and biases up to
+    the limit of 2^28 with shifts that bring them back into range."""
+    rng = np.random.default_rng(36)
+    b, h, w, c = 2, 11, 9, 48
+    x = rng.integers(-128, 128, size=(b, h, w, c)).astype(np.int8)
+    wt = rng.integers(-2, 3, size=(c, 3, 3)).astype(np.int8)
+    bias = rng.integers(-300, 301, size=c).astype(np.int32)
+    mult = rng.integers(1 << 28, (1 << 31) - 1, size=c).astype(np.int32)
+    shift = (np.arange(c) % 4).astype(np.int8)
+    _run(oracle, x, wt, bias, mult, shift, stride, lo, 127)
+    shift[:] = rng.integers(0, 2, size=c)
+    _run(oracle, x, wt, bias, mult, shift, stride, lo, 127)
+    bias = (rng.integers(-(1 << 28), (1 << 28) + 1, size=c)).astype(np.int32)
+    shift[:] = rng.integers(20, 24, size=c)
+    _run(oracle, x, wt, bias, mult, shift, stride, lo, 127)
+
+
 def test_refusals():
     x = torch.zeros((1, 4, 4, 6), dtype=torch.int8, device="cuda")
     w = torch.zeros((6, 3, 3), dtype=torch.int8, device="cuda")
