@@ -916,7 +916,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 // The residual (mode 3): the bytes that sit where this slab goes in Y, in 8-byte
                 // granules across the warp.  The first kResHeld granules of a lane are requested
                 // before the wait for the accumulator, so that their latency hides behind it.
-                constexpr int kResHeld = 4;
+                constexpr int kResHeld = 6;
                 uint2 res_held[kResHeld];
                 int res_total = 0, res_g8 = 1;
                 const int8_t *res_p = nullptr;
