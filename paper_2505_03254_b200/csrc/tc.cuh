@@ -265,24 +265,49 @@ __device__ __forceinline__ void epi_fast_subtile(const Params &p, uint32_t taddr
 
 // The exact epilogue over one subtile, in chunks of CH (32 or 16), then 16 and 8 columns.
 template <int CH>
-__device__ __forceinline__ void epi_exact_subtile(const Params &p, uint32_t taddr, const int *cm,
-                                                  const int2 *cbs, uint8_t *dst_row,
-                                                  uint32_t bar_release)
+__device__ __noinline__ void epi_exact_subtile(int nt, int act_min, int act_max, uint32_t taddr,
+                                               const int *cm, const int2 *cbs, uint8_t *dst_row,
+                                               uint32_t bar_release)
 {
-    const bool wide = (p.nt & 15) == 0;
-    const int tail = p.nt & (CH - 1);    // columns after the last full chunk
+    const bool wide = (nt & 15) == 0;
+    const int tail = nt & (CH - 1);    // columns after the last full chunk
     int c = 0;
-    for (; c + CH <= p.nt; c += CH) {
-        const uint32_t rel = (tail == 0 && c + CH == p.nt) ? bar_release : 0u;
-        epi_exact<CH>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, rel);
+    for (; c + CH <= nt; c += CH) {
+        const uint32_t rel = (tail == 0 && c + CH == nt) ? bar_release : 0u;
+        epi_exact<CH>(taddr + c, cm + c, cbs + c, act_min, act_max, dst_row + c, wide, rel);
     }
-    if (CH > 16 && c + 16 <= p.nt) {
-        const uint32_t rel = (c + 16 == p.nt) ? bar_release : 0u;
-        epi_exact<16>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, rel);
+    if (CH > 16 && c + 16 <= nt) {
+        const uint32_t rel = (c + 16 == nt) ? bar_release : 0u;
+        epi_exact<16>(taddr + c, cm + c, cbs + c, act_min, act_max, dst_row + c, wide, rel);
         c += 16;
     }
-    if (c + 8 <= p.nt)
-        epi_exact<8>(taddr + c, cm + c, cbs + c, p.act_min, p.act_max, dst_row + c, wide, bar_release);
+    if (c + 8 <= nt)
+        epi_exact<8>(taddr + c, cm + c, cbs + c, act_min, act_max, dst_row + c, wide, bar_release);
+}
+
+// Stores the first rows_valid rows of a warp's 32 x nt staging slab (a short tile or the end of
+// the matrix); yp points at the slab's first row in Y.  Out of line: it runs at most once per CTA.
+__device__ __noinline__ void store_partial_slab(int8_t *yp, const uint8_t *slab, int rows_valid, int nf,
+                                                int nt, int col, bool store_2d, int lane)
+{
+    const uint32_t slab_addr = ptx::smem_u32(slab);
+    if (!store_2d) {
+        // one subtile spans the row: the slab is one contiguous range of Y
+        if (lane == 0 && rows_valid > 0) {
+            const uint32_t bytes = (uint32_t)(rows_valid * nf);
+            const uint32_t whole = bytes & ~15u;      // bulk copies move 16-byte granules
+            if (whole) {
+                ptx::bulk_store(yp, slab_addr, whole);
+                ptx::bulk_commit();
+            }
+            if (bytes & 15u)                          // odd last row of an 8-multiple width
+                *reinterpret_cast<uint2 *>(yp + whole) = *reinterpret_cast<const uint2 *>(slab + whole);
+        }
+    } else if (lane < rows_valid) {
+        // the slab leaves row by row
+        ptx::bulk_store(yp + (long long)lane * nf + col, slab_addr + (uint32_t)(lane * nt), (uint32_t)nt);
+        ptx::bulk_commit();
+    }
 }
 
 // ---- the dynamic layer's epilogues ---------------------------------------------------------
@@ -960,7 +985,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                     const bool full_range = MODE == 4 || (MODE == 3 && p.act_min < 0);
                     if (fast && !full_range) epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
                     else if (fast) epi_fast_subtile<CH, true>(p, taddr, cms, shmax, my_row, bar_rel);
-                    else epi_exact_subtile<CH>(p, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
+                    else epi_exact_subtile<CH>(p.nt, p.act_min, p.act_max, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
                     if constexpr (MODE == 3) {
                         __syncwarp();
                         auto add_to_slab = [&](int i, uint2 rv) {
@@ -1024,26 +1049,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                     int rows_valid = p.tm - q * 32;
                     if (m_rows - row0 < rows_valid) rows_valid = m_rows - row0;
                     if (rows_valid > 32) rows_valid = 32;
-                    int8_t *yp = p.y + (long long)row0 * p.nf;
-                    if (!store_2d) {
-                        // one subtile spans the row: the slab is one contiguous range of Y
-                        if (lane == 0 && rows_valid > 0) {
-                            const uint32_t bytes = (uint32_t)(rows_valid * p.nf);
-                            const uint32_t whole = bytes & ~15u;      // bulk copies move 16-byte granules
-                            if (whole) {
-                                ptx::bulk_store(yp, slab_addr, whole);
-                                ptx::bulk_commit();
-                            }
-                            if (bytes & 15u)                          // odd last row of an 8-multiple width
-                                *reinterpret_cast<uint2 *>(yp + whole) =
-                                    *reinterpret_cast<const uint2 *>(slab + whole);
-                        }
-                    } else if (lane < rows_valid) {
-                        // the slab leaves row by row
-                        ptx::bulk_store(yp + (long long)lane * p.nf + col,
-                                        slab_addr + (uint32_t)(lane * p.nt), (uint32_t)p.nt);
-                        ptx::bulk_commit();
-                    }
+                    store_partial_slab(p.y + (long long)row0 * p.nf, slab, rows_valid, p.nf, p.nt, col,
+                                       store_2d, lane);
                 }
                 // this group's next unit and accumulator
                 ls += dls; row0 += drow; col += dcol;
