@@ -94,6 +94,23 @@ struct Params {
 // Bounded wait on an mbarrier phase.  The clock is read only every 1024 polls (a
 // poll that finds the phase incomplete already suspends the thread for a while), so
 // that a wait which ends within microseconds never pays for a timer read.
+constexpr unsigned long long kWaitGiveUp = ~0ull;
+
+// The rare part of a wait, out of line: returns the time the wait began (set on the first call),
+// or kWaitGiveUp when another thread has given up or this wait has run past its limit.
+__device__ __noinline__ unsigned long long wait_check(unsigned long long t0, volatile int *abort_flag)
+{
+    if (*abort_flag) return kWaitGiveUp;
+    const unsigned long long now = ptx::globaltimer();
+    if (t0 == 0) return now;
+    if (now - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        raise_status(PROM_ERR_TIMEOUT);
+        return kWaitGiveUp;
+    }
+    return t0;
+}
+
 template <bool BACKOFF = false>
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
@@ -102,14 +119,8 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
         if (ptx::mbar_try_wait(bar, parity)) return true;
         if constexpr (BACKOFF) __nanosleep(20);      // whole warps wait here: poll gently
         if ((i & 1023u) == 0) {
-            if (*abort_flag) return false;
-            const unsigned long long now = ptx::globaltimer();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                raise_status(PROM_ERR_TIMEOUT);
-                return false;
-            }
+            t0 = wait_check(t0, abort_flag);
+            if (t0 == kWaitGiveUp) return false;
         }
     }
 }
