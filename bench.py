@@ -34,7 +34,7 @@ FALLBACK_BF16_TFLOPS = 1590.0
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio on B200 (4.5 : 2.25)
 FLUSH_BYTES = 512 << 20       # > 2x the 126 MB L2
 NCU_TRAFFIC_PER_LAUNCH = 15.46e6
-MULHI_LANES_PER_CLK_SM = 31.6   # mul.hi.s32 issue rate measured on B200 (independent chains, all SMs)
+NOMINAL_I8_TOPS = 4500.0      # data-sheet dense int8 figure of the part, for context
 
 
 # --------------------------------------------------------------------------- helpers
@@ -126,6 +126,58 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def i8_peak_probe(torch, binding, iters=8192, reps=5, sustained_s=0.0):
+    """Measured tensor-pipe rate on tcgen05.mma.kind::i8 (128x256x32, operands fixed in shared
+    memory, one CTA per SM): the best of `reps` launches (burst) and, when asked, launches back to
+    back for `sustained_s` seconds."""
+    cycles = torch.zeros((4096,), dtype=torch.int64, device="cuda")
+    grid = binding.debug_i8_mma_rate(256, cycles)
+    torch.cuda.synchronize()
+    ops_per_launch = grid * iters * 4 * 2 * 128 * 256 * 32
+    stream = torch.cuda.current_stream()
+    best = None
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        binding.debug_i8_mma_rate(iters, cycles)
+        e1.record(stream)
+        e1.synchronize()
+        ms = e0.elapsed_time(e1)
+        best = ms if best is None or ms < best else best
+    cyc = int(cycles[:grid].max().item())
+    out = {"shape": "128x256x32 kind::i8, cta_group::1, one issuing thread per SM", "ctas": grid,
+           "iters": iters, "tops_burst": ops_per_launch / best / 1e9,
+           "macs_per_clk_per_sm": iters * 4 * 128 * 256 * 32 / cyc,
+           "sm_mhz_from_cycles": cyc / best / 1e3}
+    if sustained_s > 0:
+        n = max(1, int(sustained_s * 1e3 / best))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            binding.debug_i8_mma_rate(iters, cycles)
+        e1.record(stream)
+        e1.synchronize()
+        ms = e0.elapsed_time(e1)
+        out["tops_sustained"] = ops_per_launch * n / ms / 1e9
+        out["sustained_s"] = ms / 1e3
+    return out
+
+
+def alu_rate_probe(torch, binding, iters=2000):
+    """Measured issue rates (lanes per clock per SM) of the requantiser's 32-bit high multiply and,
+    beside it, of mad.lo.s32 and fma.rn.f32: 8 independent chains per thread, 1024 threads per SM."""
+    cycles = torch.zeros((4096,), dtype=torch.int64, device="cuda")
+    sink = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    out = {}
+    for op, name in ((0, "mul_hi_s32"), (1, "mad_lo_s32"), (2, "fma_f32")):
+        binding.debug_alu_rate(op, 100, sink, cycles)
+        grid = binding.debug_alu_rate(op, iters, sink, cycles)
+        torch.cuda.synchronize()
+        cyc = int(cycles[:grid].max().item())
+        out[name] = round(1024 * 64 * iters / cyc, 2)
+    return out
+
+
 def build_network(seed, synth, binding=None, device=None, width=1.0):
     """Layer table plus per-layer weights/constants: host arrays for the oracle,
     and (when a binding is given) packed device tensors for the library."""
@@ -210,6 +262,47 @@ def whole_job_value(images_per_rank_per_step, steps, world, ms):
     return world * images_per_rank_per_step * steps / (ms * 1e-3)
 
 
+def spawn_ranks(args, argv):
+    """`--gpus N` without a launcher's environment: start N ranks of this script itself, one
+    process per GPU (LOCAL_RANK picks the device), rendezvous on 127.0.0.1.  Rank 0 prints the
+    JSON line; the exit code is the worst of the ranks'."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(args.gpus):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(args.gpus),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env))
+    rc = 0
+    for pr in procs:
+        rc = max(rc, abs(pr.wait()))
+    return rc
+
+
+def run_stub(args):
+    """The multi-rank bookkeeping of the GPU arm with the step replaced by a fixed per-rank time
+    and `gloo` in place of NCCL: what a machine without GPUs can run of `--gpus N`."""
+    import torch.distributed as dist
+    rank, _, world = rank_info()
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+        dist.barrier()
+    ms = max_over_ranks(10.0 + 5.0 * rank, device="cpu")
+    if rank == 0:
+        print(json.dumps({"impl": "stub", "metric": METRIC, "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "ms_per_step": ms / args.steps,
+                          "value": whole_job_value(BATCH, args.steps, world, ms), "scaling": "weak"}),
+              flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
 # --------------------------------------------------------------------------- GPU arm
 def time_region(torch, fn, steps, dist_on):
     """Times `steps` calls of fn with CUDA events on the current stream, bracketed
@@ -267,7 +360,10 @@ def run_gpu(args):
         dist.barrier()
     binding.lib()
     pk = peaks()
-    p_i8 = INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12
+    # the tensor roof is measured here, on this GPU, before anything is timed against it
+    i8 = i8_peak_probe(torch, binding, sustained_s=0.25)
+    alu = alu_rate_probe(torch, binding)
+    p_i8 = i8["tops_burst"] * 1e12
     bw = pk["hbm_gbs"] * 1e9
 
     seed = synth.BASE_SEED + 3
@@ -395,13 +491,29 @@ def run_gpu(args):
                 "step_roofline_us": sum(roof_us),
                 "step_roofline_frac": sum(roof_us) / (ms_per_step * 1e3)}
 
-    # second roof of the requantising epilogue: one 32-bit high multiply per output, an
-    # instruction the SM retires at 31.6 lanes per clock (measured), i.e. a quarter of the fp32 rate
+    # second roof of the requantising epilogue: one 32-bit high multiply per output, at the rate
+    # the probe above measured on this GPU (lanes per clock per SM) and the sampled SM clock
     step_outputs = sum(m * l.cout for m, l in zip(ms_layers, table))
-    alu_peak = 148 * MULHI_LANES_PER_CLK_SM * 1.965e9
+    sms = torch.cuda.get_device_properties(local).multi_processor_count
+    clk = (sampler.summary()["sm_mhz"] or 1965) * 1e6
+    alu_peak = sms * alu["mul_hi_s32"] * clk
     roofline["epilogue_alu"] = {"bound": "alu", "achieved": step_outputs / (ms_per_step * 1e-3),
                                 "peak": alu_peak, "unit": "outputs/s",
-                                "frac": step_outputs / (ms_per_step * 1e-3) / alu_peak}
+                                "frac": step_outputs / (ms_per_step * 1e-3) / alu_peak,
+                                "lanes_per_clk_per_sm": alu}
+    # the tensor roof behind the compute-bound layers' figures: measured, with the two other
+    # candidates beside it
+    roofline["tensor_peak"] = {"used_tops": p_i8 / 1e12, "source": "measured here (tcgen05.mma.kind::i8 issue loop)",
+                               "probe": i8, "two_x_measured_bf16_tops": INT8_OVER_BF16 * pk["bf16_tflops"],
+                               "nominal_tops": NOMINAL_I8_TOPS,
+                               "step_roofline_us_at_2x_bf16": sum(
+                                   max(layer_bytes(m, l.cin, l.cout) / bw,
+                                       layer_ops(m, l.cin, l.cout) / (INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12)) * 1e6
+                                   for m, l in zip(ms_layers, table)),
+                               "step_roofline_us_at_nominal": sum(
+                                   max(layer_bytes(m, l.cin, l.cout) / bw,
+                                       layer_ops(m, l.cin, l.cout) / (NOMINAL_I8_TOPS * 1e12)) * 1e6
+                                   for m, l in zip(ms_layers, table))}
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -653,25 +765,52 @@ def single_layer_configs(torch, binding, synth, bw, p_i8):
 
 
 # --------------------------------------------------------------------------- sweep
+def sweep_rows(m, torch, tile=128, edge=512, one_in=64):
+    """Rows the oracle checks at a sweep point: all of them up to 16384 rows, else the first and
+    last `edge`, both rows at every tile boundary, and every `one_in`-th of the rest (staggered)."""
+    if m <= 16384:
+        return torch.arange(m, dtype=torch.int64)
+    keep = torch.zeros(m, dtype=torch.bool)
+    keep[:edge] = True
+    keep[m - edge:] = True
+    b = torch.arange(tile, m, tile, dtype=torch.int64)
+    keep[b] = True
+    keep[b - 1] = True
+    keep[torch.arange(37, m, one_in + 1, dtype=torch.int64)] = True
+    return torch.nonzero(keep).flatten()
+
+
 def run_sweep(args):
-    """Shape and sparsity sweep of single layers: the tensor-core (or, where it
-    does not apply, small-K) variant and the add/sub variant on every point."""
+    """Shape and sparsity sweep of single layers: the tensor-core variant (or what AUTO picks
+    where it refuses the shape, labelled) and the add/sub variant on every point, each timed with
+    a cold L2 and checked: the whole output against the plain one-thread-per-output kernel, and
+    sampled rows against the CPU oracle."""
     import torch
     from paper_2505_03254_b200 import binding, build, synth
     torch.cuda.set_device(0)
     build.build()
     binding.lib()
+    oracle = None
+    if not args.no_cpu:
+        from oracle import prom_oracle as oracle
+        oracle.build()
     pk = peaks()
-    bw, p_i8 = pk["hbm_gbs"] * 1e9, INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12
+    i8 = i8_peak_probe(torch, binding)
+    bw, p_i8 = pk["hbm_gbs"] * 1e9, i8["tops_burst"] * 1e12
     flush = torch.empty((FLUSH_BYTES,), dtype=torch.uint8, device="cuda")
     ms_list = synth.CONFIG5_M if not args.sweep_small else synth.CONFIG5_M[:2]
-    n = 0
+    n = bad = 0
     with open(args.sweep, "w") as f:
+        f.write(json.dumps({"int8_peak_probe": i8, "hbm_gbs": pk["hbm_gbs"], "peak_source": pk["source"]}) + "\n")
         for m in ms_list:
+            rows = sweep_rows(m, torch)
+            rows_d = rows.cuda()
             for cin in synth.CONFIG5_CIN:
                 x = synth.act_uniform_i8(synth.BASE_SEED + 5, (m, cin), device="cuda")
+                x_rows = x[rows_d].cpu().numpy() if oracle is not None else None
                 for cout in synth.CONFIG5_COUT:
                     y = torch.empty((m, cout), dtype=torch.int8, device="cuda")
+                    y_ref = torch.empty((m, cout), dtype=torch.int8, device="cuda")
                     for z in synth.CONFIG5_ZERO:
                         lay = synth.make_layer(synth.BASE_SEED + 5, cin, cout, z, device="cuda")
                         wp = binding.pack_ternary(lay["w"])
@@ -679,6 +818,13 @@ def run_sweep(args):
                         b, o = layer_bytes(m, cin, cout), layer_ops(m, cin, cout)
                         roof = max(b / bw, o / p_i8) * 1e6
                         nnz = int((lay["w"] != 0).sum().item())
+                        binding.pw_conv_i8(x, wp, cout, rq, y=y_ref, variant="naive")
+                        want, naive_ok = None, True
+                        if oracle is not None:
+                            want = torch.from_numpy(oracle.conv_mul(
+                                x_rows, lay["w"].cpu().numpy(), lay["bias"].cpu().numpy(),
+                                lay["mult"].cpu().numpy(), lay["shift"].cpu().numpy())).cuda()
+                            naive_ok = bool(torch.equal(y_ref[rows_d], want))
                         for variant in ("tc", "addsub"):
                             used = variant
                             try:
@@ -690,19 +836,29 @@ def run_sweep(args):
                                 fn()
                             iters = 5 if variant == "addsub" else 10
                             med, mn = cold_time_us(torch, fn, flush, iters=iters, warm=1)
+                            same_as_naive = bool(torch.equal(y, y_ref))
                             rec = {"m": m, "k": cin, "n": cout, "zero_frac": z, "variant": variant,
                                    "ran_as": used, "us": round(med, 2),
                                    "gops": round(o / med / 1e3, 1), "gbs": round(b / med / 1e3, 1),
                                    "roof_us": round(roof, 2), "frac": round(roof / med, 4),
-                                   "adds": m * nnz}
+                                   "bound": "tensor" if o / p_i8 > b / bw else "hbm",
+                                   "adds": m * nnz, "parity_vs_naive_whole": same_as_naive}
+                            ok = same_as_naive
+                            if want is not None:
+                                rec["parity_vs_oracle_rows"] = bool(torch.equal(y[rows_d], want)) and naive_ok
+                                rec["oracle_rows"] = int(rows.numel())
+                                ok = ok and rec["parity_vs_oracle_rows"]
+                            rec["parity"] = ok
+                            bad += 0 if ok else 1
                             f.write(json.dumps(rec) + "\n")
                             f.flush()
                             n += 1
-                    del y
+                    del y, y_ref
                 del x
     st = binding.last_device_status()
-    print(json.dumps({"sweep_points": n, "device_status": st, "file": args.sweep}), flush=True)
-    return 0 if st == binding.PROM_OK else 1
+    print(json.dumps({"sweep_points": n, "parity_failures": bad, "device_status": st, "file": args.sweep}),
+          flush=True)
+    return 0 if st == binding.PROM_OK and bad == 0 else 1
 
 
 def run_single(args):
@@ -717,7 +873,7 @@ def run_single(args):
     variant = parts[3] if len(parts) > 3 else "auto"
     z = float(parts[4]) if len(parts) > 4 else 0.5
     pk = peaks()
-    bw, p_i8 = pk["hbm_gbs"] * 1e9, INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12
+    bw, p_i8 = pk["hbm_gbs"] * 1e9, i8_peak_probe(torch, binding)["tops_burst"] * 1e12
     seed = synth.BASE_SEED + 2
     x = synth.act_post_relu6(seed, (m, cin), device="cuda")
     lay = synth.make_layer(seed, cin, cout, z, device="cuda")
@@ -750,7 +906,7 @@ def run_widths(args):
     prom_oracle.build()
     binding.lib()
     pk = peaks()
-    p_i8 = INT8_OVER_BF16 * pk["bf16_tflops"] * 1e12
+    p_i8 = i8_peak_probe(torch, binding)["tops_burst"] * 1e12
     bw = pk["hbm_gbs"] * 1e9
     seed = synth.BASE_SEED + 3
     rows = []
@@ -795,7 +951,19 @@ def run_aux(args):
     build.build()
     binding.lib()
     bw = peaks()["hbm_gbs"] * 1e9
-    if args.aux == "act_quantizer":
+    if args.aux == "i8_peak":
+        sampler = ClockSampler(0)
+        sampler.start()
+        out = i8_peak_probe(torch, binding, sustained_s=2.0)
+        sampler.stop()
+        pk = peaks()
+        out["clocks"] = sampler.summary()
+        out["two_x_measured_bf16_tops"] = INT8_OVER_BF16 * pk["bf16_tflops"]
+        out["two_x_measured_bf16_sustained_tops"] = INT8_OVER_BF16 * pk["bf16_tflops_sustained"]
+        out["nominal_tops"] = NOMINAL_I8_TOPS
+    elif args.aux == "alu_rate":
+        out = alu_rate_probe(torch, binding)
+    elif args.aux == "act_quantizer":
         out = act_quantizer_timing(torch, binding, bw)
     elif args.aux == "dynamic_layer":
         out = dynamic_layer_timing(torch, binding, synth, bw)
@@ -813,20 +981,25 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "stub"])
     ap.add_argument("--variant", default="auto", choices=["auto", "tc", "naive"])
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of a CUDA graph")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
     ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
-    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body"],
+    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate"],
                     help="run one of the legs that are off the timed step, alone")
     ap.add_argument("--widths", default=None, help="comma-separated width multipliers: time the sequence at each")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    plain_leg = not (args.widths or args.aux or args.single or args.sweep)
+    if args.gpus > 1 and plain_leg and "RANK" not in os.environ and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args, sys.argv[1:])
+    if args.impl == "stub":
+        return run_stub(args)
     if args.widths:
         return run_widths(args)
     if args.aux:

@@ -19,7 +19,7 @@
  *     Y[m][o] = min(act_max, max(act_min, q))
  *
  * The paper applies the per-channel weight scale and the activation scale in
- * floating point (Figure 12: "dequantize after convolution"); this library
+ * floating point, after the integer convolution (Figure 12, inference branch); this library
  * takes them, with BatchNorm and the next layer's activation scale folded in,
  * as the fixed-point pair (mult, shift): one rounding of the exact product,
  * ties away from zero.  Integer sums and this rounding are exact, so there is
@@ -119,8 +119,8 @@ typedef struct {
 size_t prom_packed_bytes(int cout, int cin);
 
 /* Packs device int8 ternary weights w_dev[cout][cin] into packed_dev.
- * "Weights can be quantized and fixed in advance" (Figure 12): this runs once
- * per layer, off the hot path.  Synchronises `cuda_stream`.  Returns
+ * Weights are quantised once, ahead of inference (Figure 12, inference
+ * branch): this runs once per layer, off the hot path.  Synchronises `cuda_stream`.  Returns
  * PROM_ERR_BAD_WEIGHT (packed_dev contents then unspecified) if any value is
  * outside {-1,0,+1}; PROM_ERR_WORKSPACE if packed_bytes is too small. */
 prom_status prom_pack_ternary(const int8_t *w_dev, int cout, int cin,
@@ -158,8 +158,8 @@ prom_status prom_dw_conv3x3_i8(const int8_t *x_dev, int batch, int h, int w, int
                                void *cuda_stream);
 
 /* A pointwise layer in the paper's own inference dataflow: pseudocode appendix, inference
- * branch of the quantised convolution module ("perform convolution in low bit-width, dequantise
- * after convolution"), followed by the activation quantiser of the next module (Section 3.1,
+ * branch of the quantised convolution module (integer convolution first, the scales applied to
+ * its result), followed by the activation quantiser of the next module (Section 3.1,
  * Eq. 6-7).  With b(m) = m / rows_per_sample the sample of row m,
  *     acc[m][o] = sum_k x[m][k] * W-hat[o][k]                        exact integers
  *     y[m][o]   = acc[m][o] * alpha[o] * (max(gamma_x[b], 1e-5) / 127)  dequantised output
@@ -338,25 +338,6 @@ prom_status prom_last_device_status(void *cuda_stream);
 /* Number of kernels this library has launched since it was loaded (all
  * streams, this process); used by the benchmark to count launches. */
 uint64_t prom_launch_count(void);
-
-/* Tuning aid for the TC variant: forces the row fold (1, 2, 4, 8), the subtile
- * width, the number of output-channel groups, the way CTAs share an SM (1: one
- * CTA with all of tensor memory; 2: two CTAs of the kernel per SM; 3: one
- * half-sized CTA per SM; 4: three CTAs per SM, on a build of the kernel with 64
- * registers a thread) and the depth of the activation ring of later calls;
- * 0 leaves a choice to the library.  A forced combination that does not fit
- * makes TC report PROM_ERR_UNSUPPORTED.  Results never depend on the plan.  Not
- * thread-safe.  prom_debug_tc_plan_query writes the plan the library would
- * use for a plain [m][cin] x [cout] layer ({fold, nt, groups, grid, stages,
- * accumulators, shared bytes, chunk bytes, estimate in 1/100 us}) and returns
- * 1, or returns 0 if TC cannot run it.  Without a CUDA device it plans for a
- * B200's nominal limits (148 SMs, 227 KB of shared memory per CTA). */
-void prom_debug_tc_plan(int fold, int nt, int groups, int occ, int stages);
-/* The same override for one shape only (m rows, cin, cout, input stride of the layer); it takes
- * precedence over prom_debug_tc_plan for that shape.  All five values 0 removes it. */
-void prom_debug_tc_plan_shape(int64_t m, int cin, int cout, int stride, int fold, int nt, int groups,
-                              int occ, int stages);
-int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
 
 /* Frees the library's internal caches (all devices).  Optional. */
 void prom_shutdown(void);

@@ -1,0 +1,77 @@
+/*
+ * prom_debug.h -- tuning, measurement and test aids of the ternary
+ * pointwise-convolution library.  Nothing here is needed to run the path of
+ * prom.h; results of that path never depend on anything set here.  The paper
+ * has no counterpart for any of these.
+ */
+#ifndef PROM_DEBUG_H_
+#define PROM_DEBUG_H_
+
+#include "prom.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Tuning aid for the TC variant: forces the row fold (1, 2, 4, 8), the subtile
+ * width, the number of output-channel groups, the way CTAs share an SM (1: one
+ * CTA with all of tensor memory; 2: two CTAs of the kernel per SM; 3: one
+ * half-sized CTA per SM; 4: three CTAs per SM, on a build of the kernel with 64
+ * registers a thread) and the depth of the activation ring of later calls;
+ * 0 leaves a choice to the library.  A forced combination that does not fit
+ * makes TC report PROM_ERR_UNSUPPORTED.  The override is process-wide (one
+ * lock guards it; a call that plans while another thread changes it sees the
+ * old or the new override, never a mixture).  prom_debug_tc_plan_query writes
+ * the plan the library would use for a plain [m][cin] x [cout] layer ({fold,
+ * nt, groups, grid, stages, accumulators, shared bytes, chunk bytes, estimate
+ * in 1/100 us}) and returns 1, or returns 0 if TC cannot run it.  Without a
+ * CUDA device it plans for a B200's nominal limits (148 SMs, 227 KB of shared
+ * memory per CTA). */
+void prom_debug_tc_plan(int fold, int nt, int groups, int occ, int stages);
+/* The same override for one shape only (m rows, cin, cout, input stride of the
+ * layer); it takes precedence over prom_debug_tc_plan for that shape.  All five
+ * values 0 removes it. */
+void prom_debug_tc_plan_shape(int64_t m, int cin, int cout, int stride, int fold, int nt,
+                              int groups, int occ, int stages);
+int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
+
+/* Which parts of a layer sequence run depth-first in one launch (see
+ * prom_pw_layer_seq): 0 = none (one launch per layer), 1 = the library's
+ * choice (default).  Process-wide. */
+void prom_debug_seq_chain(int mode);
+
+/* Failure-detection check: launches one warp that waits, with the library's
+ * bounded mbarrier wait and a limit of limit_ns nanoseconds (1000 ..
+ * 100 000 000), on a barrier phase nothing ever completes.  The wait gives up
+ * by itself and the kernel returns normally; afterwards
+ * prom_last_device_status reports PROM_ERR_TIMEOUT.  gave_up_dev (device int,
+ * may be NULL) receives 1.  Nothing traps, faults or waits without a limit. */
+prom_status prom_debug_wait_timeout(uint64_t limit_ns, int *gave_up_dev, void *cuda_stream);
+
+/* Rate probes for the roofline figures.  Both launch one grid over all SMs and
+ * write, per CTA, the SM clock cycles of its measured loop into cycles_dev
+ * (device, cycles_len >= the grid size, which *grid_out receives); the host
+ * times the launch itself with events.
+ *   i8_mma_rate: one CTA per SM, one thread issuing iters x 4
+ *     tcgen05.mma.kind::i8 instructions of shape 128 x 256 x 32 on fixed
+ *     shared-memory operands into two alternating accumulators, one commit and
+ *     a bounded wait at the end: 2 * 128 * 256 * 32 * 4 * iters operations per CTA.
+ *     1 <= iters <= 2^20.
+ *   alu_rate: op 0 = mul.hi.s32 (the requantiser's multiply), 1 = mad.lo.s32,
+ *     2 = fma.rn.f32; two CTAs of 512 threads per SM, 8 independent chains per
+ *     thread, 64 * iters instructions per thread.  sink_dev: one device int.
+ * Asynchronous on the stream. */
+prom_status prom_debug_i8_mma_rate(int iters, long long *cycles_dev, int cycles_len, int *grid_out,
+                                   void *cuda_stream);
+prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cycles_dev,
+                                int cycles_len, int *grid_out, void *cuda_stream);
+
+/* Bookkeeping check, no CUDA call: returns 1 the first time (device, key) is
+ * asked about on the table used for per-device kernel attributes, 0
+ * afterwards (the table behind this entry is a separate instance). */
+int prom_debug_once_per_device(int device, int key);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PROM_DEBUG_H_ */

@@ -29,6 +29,8 @@ EXPORTS = [
     "prom_launch_count", "prom_shutdown", "prom_status_string",
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
     "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8", "prom_debug_tc_plan_shape", "prom_pw_conv_i8_res",
+    "prom_debug_seq_chain", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
+    "prom_debug_once_per_device",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -102,6 +104,16 @@ def lib():
         L.prom_debug_tc_plan.argtypes = [i32, i32, i32, i32, i32]
         L.prom_debug_tc_plan_query.restype = i32
         L.prom_debug_tc_plan_query.argtypes = [i64, i32, i32, C.POINTER(C.c_int)]
+        L.prom_debug_seq_chain.restype = None
+        L.prom_debug_seq_chain.argtypes = [i32]
+        L.prom_debug_wait_timeout.restype = i32
+        L.prom_debug_wait_timeout.argtypes = [C.c_uint64, vp, vp]
+        L.prom_debug_i8_mma_rate.restype = i32
+        L.prom_debug_i8_mma_rate.argtypes = [i32, vp, i32, C.POINTER(C.c_int), vp]
+        L.prom_debug_alu_rate.restype = i32
+        L.prom_debug_alu_rate.argtypes = [i32, i32, vp, vp, i32, C.POINTER(C.c_int), vp]
+        L.prom_debug_once_per_device.restype = i32
+        L.prom_debug_once_per_device.argtypes = [i32, i32]
         L.prom_quantize_ternary.restype = i32
         L.prom_quantize_ternary.argtypes = [vp, i32, i32, vp, sz, vp, vp]
         L.prom_requant_from_scale.restype = i32
@@ -229,6 +241,43 @@ def debug_tc_plan_query(m: int, cin: int, cout: int):
         return None
     keys = ("fold", "nt", "groups", "grid", "stages", "nbuf", "smem", "cw", "est_us_x100")
     return dict(zip(keys, list(out)))
+
+
+def debug_seq_chain(mode: int = 1) -> None:
+    """prom_debug_seq_chain: 0 = one launch per layer, 1 = the library's choice of depth-first parts."""
+    lib().prom_debug_seq_chain(int(mode))
+
+
+def debug_wait_timeout(limit_ns: int = 5000, stream=None) -> int:
+    """prom_debug_wait_timeout: a bounded wait that is left to run out; returns 1 when the
+    wait gave up (read back after a synchronise)."""
+    flag = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    _check(lib().prom_debug_wait_timeout(int(limit_ns), flag.data_ptr(), _stream(stream)),
+           "prom_debug_wait_timeout")
+    torch.cuda.synchronize()
+    return int(flag.item())
+
+
+def debug_i8_mma_rate(iters: int, cycles: torch.Tensor, stream=None) -> int:
+    """prom_debug_i8_mma_rate: launches the tensor-pipe probe; cycles is an int64 CUDA tensor
+    that receives per-CTA SM clocks.  Returns the grid size."""
+    grid = C.c_int(0)
+    _check(lib().prom_debug_i8_mma_rate(int(iters), _dev(cycles, torch.int64, "cycles"), cycles.numel(),
+                                        C.byref(grid), _stream(stream)), "prom_debug_i8_mma_rate")
+    return int(grid.value)
+
+
+def debug_alu_rate(op: int, iters: int, sink: torch.Tensor, cycles: torch.Tensor, stream=None) -> int:
+    """prom_debug_alu_rate: op 0 mul.hi.s32, 1 mad.lo.s32, 2 fma.rn.f32.  Returns the grid size."""
+    grid = C.c_int(0)
+    _check(lib().prom_debug_alu_rate(int(op), int(iters), _dev(sink, torch.int32, "sink"),
+                                     _dev(cycles, torch.int64, "cycles"), cycles.numel(), C.byref(grid),
+                                     _stream(stream)), "prom_debug_alu_rate")
+    return int(grid.value)
+
+
+def debug_once_per_device(device: int, key: int) -> bool:
+    return bool(lib().prom_debug_once_per_device(int(device), int(key)))
 
 
 def shutdown() -> None:

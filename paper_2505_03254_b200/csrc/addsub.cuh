@@ -21,6 +21,7 @@
 #include <unordered_map>
 
 #include "common.cuh"
+#include "hostutil.cuh"
 
 namespace prom { namespace addsub {
 
@@ -175,7 +176,7 @@ addsub_conv_kernel(const int8_t *__restrict__ x, long long m, int cin, RowMap ma
                 long long row = row0 + lane * 4 + j;
                 if (row >= m) continue;
                 int8_t *yp = y + row * cout + o4;
-                if (four) {
+                if (four && okc[0] && okc[1] && okc[2] && okc[3]) {
                     uint32_t wv = ((uint32_t)q[0][j] & 0xFFu) | (((uint32_t)q[1][j] & 0xFFu) << 8) |
                                   (((uint32_t)q[2][j] & 0xFFu) << 16) |
                                   (((uint32_t)q[3][j] & 0xFFu) << 24);
@@ -250,14 +251,7 @@ static inline prom_status launch_on(const int8_t *x, long long m, int cin, const
     ++launches;
     if (cudaGetLastError() != cudaSuccess) return PROM_ERR_CUDA;
     size_t smem = conv_smem(cin);
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(addsub_conv_kernel,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)conv_smem(kMaxCin));
-    });
-    if (attr_err != cudaSuccess) return PROM_ERR_CUDA;
+    if (raise_smem_limit(addsub_conv_kernel, (int)conv_smem(kMaxCin)) != cudaSuccess) return PROM_ERR_CUDA;
     long long tiles = (m + kRows - 1) / kRows;
     int occ = smem > 100 * 1024 ? 1 : 2;
     long long cap = (long long)sms * occ;

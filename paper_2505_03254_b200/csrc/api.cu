@@ -14,8 +14,10 @@
 #include <vector>
 
 #include "prom.h"
+#include "prom_debug.h"
 
 #include "common.cuh"
+#include "hostutil.cuh"
 #include "simple.cuh"
 #include "tc.cuh"
 #include "smallk.cuh"
@@ -23,6 +25,7 @@
 #include "actquant.cuh"
 #include "depthwise.cuh"
 #include "quantize.cuh"
+#include "peak.cuh"
 
 namespace prom {
 
@@ -170,6 +173,9 @@ static TcTune tune_for(long long m, int cin, int cout, int stride)
     auto it = g_shape_tune.find({m, cin, cout, stride});
     return it == g_shape_tune.end() ? g_tune : it->second;
 }
+
+// Depth-first execution of parts of a sequence (0 = off), set by prom_debug_seq_chain.
+static std::atomic<int> g_seq_chain{1};
 
 static int round_up(int v, int a) { return (v + a - 1) / a * a; }
 
@@ -429,37 +435,15 @@ static bool tc_make_maps(const Conv &c, TcPlan &pl)
 
 static prom_status tc_set_attr(const DeviceInfo &d)
 {
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [&] {
-        attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<3>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            d.smem_optin);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 1>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            d.smem_optin);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 2>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            d.smem_optin);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 4>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            d.smem_optin);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(tc::tc_conv_kernel<2, 3>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            d.smem_optin);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(tc::tc_prep_kernel,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            d.smem_optin);
-    });
-    return attr_err == cudaSuccess ? PROM_OK : PROM_ERR_CUDA;
+    // once per device: the limit is an attribute of the (function, device) pair
+    cudaError_t e = raise_smem_limit(tc::tc_conv_kernel<2>, d.smem_optin);
+    if (e == cudaSuccess) e = raise_smem_limit(tc::tc_conv_kernel<3>, d.smem_optin);
+    if (e == cudaSuccess) e = raise_smem_limit(tc::tc_conv_kernel<2, 1>, d.smem_optin);
+    if (e == cudaSuccess) e = raise_smem_limit(tc::tc_conv_kernel<2, 2>, d.smem_optin);
+    if (e == cudaSuccess) e = raise_smem_limit(tc::tc_conv_kernel<2, 4>, d.smem_optin);
+    if (e == cudaSuccess) e = raise_smem_limit(tc::tc_conv_kernel<2, 3>, d.smem_optin);
+    if (e == cudaSuccess) e = raise_smem_limit(tc::tc_prep_kernel, d.smem_optin);
+    return e == cudaSuccess ? PROM_OK : PROM_ERR_CUDA;
 }
 
 // Fills in the pointers of a planned layer (image: prepared operands, or null).
@@ -925,12 +909,7 @@ prom_status prom_quantize_act_absmax(const float *x_dev, int batch, int64_t per_
         }
     }
     if (cluster) {
-        static std::once_flag once;
-        static cudaError_t attr_err = cudaSuccess;
-        std::call_once(once, [&] {
-            attr_err = cudaFuncSetAttribute(actq::act_quant_cluster_kernel,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, d.smem_optin - 4096);
-        });
+        const cudaError_t attr_err = raise_smem_limit(actq::act_quant_cluster_kernel, d.smem_optin - 4096);
         if (attr_err != cudaSuccess) return cuda_status(attr_err);
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof(cfg));
@@ -1200,6 +1179,9 @@ prom_status prom_pw_conv_i8_addsub_static(const int8_t *x_dev, int64_t m, int ci
                                           const prom_requant *rq, int8_t *y_dev,
                                           void *cuda_stream)
 {
+    // an empty matrix has no rows to read or write: its pointers may be anything
+    if (m == 0 && cin >= 1 && cin <= 4096 && cout >= 1 && cout <= 4096 && w_packed_dev && rq)
+        return check_requant(rq);
     prom_status s = check_conv(x_dev, m, cin, w_packed_dev, cout, rq, y_dev);
     if (s != PROM_OK) return s;
     if (cin > addsub::kMaxCin) return PROM_ERR_UNSUPPORTED;
@@ -1240,7 +1222,59 @@ void prom_debug_tc_plan_shape(int64_t m, int cin, int cout, int stride, int fold
 
 void prom_debug_tc_plan(int fold, int nt, int groups, int occ, int stages)
 {
+    std::lock_guard<std::mutex> lk(g_shape_tune_mu);
     g_tune = TcTune{fold, nt, groups, occ, stages};
+}
+
+prom_status prom_debug_wait_timeout(uint64_t limit_ns, int *gave_up_dev, void *cuda_stream)
+{
+    if (limit_ns < 1000 || limit_ns > 100000000ull) return PROM_ERR_SHAPE;
+    tc::wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        (unsigned long long)limit_ns, gave_up_dev);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+prom_status prom_debug_i8_mma_rate(int iters, long long *cycles_dev, int cycles_len, int *grid_out,
+                                   void *cuda_stream)
+{
+    if (!cycles_dev || !grid_out) return PROM_ERR_NULL;
+    if (iters < 1 || iters > (1 << 20)) return PROM_ERR_SHAPE;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    if (cycles_len < d.sms) return PROM_ERR_WORKSPACE;
+    if (raise_smem_limit(peak::i8_mma_rate_kernel, peak::kMmaSmem) != cudaSuccess) return PROM_ERR_CUDA;
+    *grid_out = d.sms;
+    peak::i8_mma_rate_kernel<<<d.sms, peak::kMmaThreads, peak::kMmaSmem,
+                               static_cast<cudaStream_t>(cuda_stream)>>>(iters, cycles_dev);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cycles_dev,
+                                int cycles_len, int *grid_out, void *cuda_stream)
+{
+    if (!sink_dev || !cycles_dev || !grid_out) return PROM_ERR_NULL;
+    if (op < 0 || op > 2 || iters < 1 || iters > (1 << 24)) return PROM_ERR_SHAPE;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    const int grid = 2 * d.sms;
+    if (cycles_len < grid) return PROM_ERR_WORKSPACE;
+    *grid_out = grid;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (op == 0) peak::alu_rate_kernel<0><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
+    else if (op == 1) peak::alu_rate_kernel<1><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
+    else peak::alu_rate_kernel<2><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode ? 1 : 0); }
+
+int prom_debug_once_per_device(int device, int key)
+{
+    static OncePerDevice table;
+    return table.first(device, reinterpret_cast<const void *>((intptr_t)key)) ? 1 : 0;
 }
 
 int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9)

@@ -98,12 +98,13 @@ constexpr unsigned long long kWaitGiveUp = ~0ull;
 
 // The rare part of a wait, out of line: returns the time the wait began (set on the first call),
 // or kWaitGiveUp when another thread has given up or this wait has run past its limit.
-__device__ __noinline__ unsigned long long wait_check(unsigned long long t0, volatile int *abort_flag)
+__device__ __noinline__ unsigned long long wait_check(unsigned long long t0, volatile int *abort_flag,
+                                                      unsigned long long limit_ns)
 {
     if (*abort_flag) return kWaitGiveUp;
     const unsigned long long now = ptx::globaltimer();
     if (t0 == 0) return now;
-    if (now - t0 > kWaitLimitNs) {
+    if (now - t0 > limit_ns) {
         *abort_flag = 1;
         raise_status(PROM_ERR_TIMEOUT);
         return kWaitGiveUp;
@@ -112,14 +113,15 @@ __device__ __noinline__ unsigned long long wait_check(unsigned long long t0, vol
 }
 
 template <bool BACKOFF = false>
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                         unsigned long long limit_ns = kWaitLimitNs)
 {
     unsigned long long t0 = 0;
     for (uint32_t i = 1;; ++i) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
         if constexpr (BACKOFF) __nanosleep(20);      // whole warps wait here: poll gently
         if ((i & 1023u) == 0) {
-            t0 = wait_check(t0, abort_flag);
+            t0 = wait_check(t0, abort_flag, limit_ns);
             if (t0 == kWaitGiveUp) return false;
         }
     }
@@ -756,7 +758,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         } else {
             build_aconst(aconst_smem, (int)threadIdx.x - 32, kThreads - 32);
             ptx::named_sync(1, kThreads);
-            wait_bar<true>(bar_wload, 0u, flags);
+            // an image that never lands stops the whole CTA (the header is then never read)
+            if (!wait_bar<true>(bar_wload, 0u, flags)) flags[0] = 1;
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before_sync();
             ptx::named_sync(2, kThreads - 32);
@@ -771,10 +774,11 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
         ptx::tc_fence_after_sync();
     }
     const bool solo = split && warp == 0;        // has not seen the image or tensor memory
+    const bool no_image = !solo && split && flags[0] != 0;
     const uint32_t tmem_base = solo ? 0u : *tmem_slot;
-    const int shmax = solo ? 0 : vw.hdr[0];
-    const bool fast = solo ? false : vw.hdr[1] != 0;
-    const bool bad_consts = solo ? false : vw.hdr[2] != 0;
+    const int shmax = solo || no_image ? 0 : vw.hdr[0];
+    const bool fast = solo || no_image ? false : vw.hdr[1] != 0;
+    const bool bad_consts = solo ? false : (no_image || vw.hdr[2] != 0);
     if (bad_consts && threadIdx.x == 32) flags[0] = 1;      // stops the producer too
 
     // instruction descriptor: s8 x s8 -> s32, both K-major, M = 128, N = nt_pad
@@ -1075,6 +1079,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     }
 
     // ---- teardown -------------------------------------------------------------------------
+    // A CTA whose roles were skipped has not waited for the previous kernel yet; it must, or
+    // this grid could end (and release the next one) while that kernel is still running.
+    if (p.pdl && bad_consts && threadIdx.x == 0) ptx::grid_dep_wait();
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -1083,6 +1090,25 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     }
 }
 
+
+// Test aid: one warp waits, with the library's bounded wait and a limit of `limit_ns`, on an
+// mbarrier phase that nothing will ever complete.  The wait gives up by itself, records
+// PROM_ERR_TIMEOUT in the device status word and the kernel returns normally.
+__global__ void __launch_bounds__(32, 1) wait_timeout_probe_kernel(unsigned long long limit_ns, int *gave_up)
+{
+    __shared__ uint64_t bar;
+    __shared__ int flag;
+    if (threadIdx.x == 0) {
+        flag = 0;
+        ptx::mbar_init(ptx::smem_u32(&bar), 1);
+        ptx::mbar_init_fence();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        const bool done = wait_bar(ptx::smem_u32(&bar), 0u, &flag, limit_ns);
+        if (gave_up) *gave_up = done ? 0 : 1;
+    }
+}
 
 // Prepared operands for a whole layer sequence in one launch: CTA b builds the image of
 // (layer, channel group) = the b-th entry of the table and writes it to that layer's

@@ -18,9 +18,13 @@ def lib():
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "prom.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(prom_[a-z0-9_]+)\s*\(", text)))
+    import glob
+    names = set()
+    for path in glob.glob(os.path.join(ROOT, "include", "*.h")):
+        text = open(path).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(prom_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_every_declared_symbol_is_exported(lib):
@@ -102,3 +106,15 @@ def test_requant_from_scale_matches_the_oracle(lib, oracle):
         assert e.value.code == binding.PROM_ERR_BAD_REQUANT
         with pytest.raises(ValueError):
             oracle.requant_from_scale(bad)
+
+
+def test_attributes_are_recorded_per_device(lib):
+    """The table behind the per-device kernel attributes (a kernel's shared-memory limit
+    belongs to the device that was current when it was raised): each (device, kernel) pair is
+    new exactly once, whatever the order of the calls."""
+    assert binding.debug_once_per_device(0, 11)
+    assert not binding.debug_once_per_device(0, 11)
+    assert binding.debug_once_per_device(1, 11)          # the same kernel on a second device
+    assert binding.debug_once_per_device(0, 12)          # another kernel on the first
+    assert not binding.debug_once_per_device(1, 11)
+    assert not binding.debug_once_per_device(0, 12)

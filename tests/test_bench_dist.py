@@ -69,3 +69,19 @@ def test_reference_arm_prints_on_rank_0_only():
     assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["value"] > 0
     assert rec["cpu_baseline"]["kind"] == "oracle" and rec["cpu_baseline"]["cores"] >= 1
     assert rec["e2e"]["h2d_bytes_per_step"] == 0 and rec["unit"] == "images/s"
+
+
+def test_gpus_flag_alone_starts_that_many_ranks():
+    """`bench.py --gpus 2` called plainly (no launcher environment) starts two ranks itself; here
+    with the step stubbed out and `gloo`, which is what runs without GPUs.  One JSON line comes
+    back, from rank 0, for two ranks, with the slowest rank's time and both ranks' images."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "stub", "--gpus", "2",
+                        "--steps", "4"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr
+    lines = [l for l in r.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1, r.stdout
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2 and rec["impl"] == "stub"
+    assert abs(rec["ms_per_step"] - 15.0 / 4) < 1e-9
+    assert abs(rec["value"] - 2 * 128 * 4 / 15e-3) < 1e-6
