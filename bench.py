@@ -732,6 +732,46 @@ def body_with_depthwise_timing(torch, binding, synth, bw, skips=False):
             "device_status": binding.last_device_status()}
 
 
+def depth_first_timing(torch, binding, synth):
+    """The three runs of late layers of the network (28x28, 14x14 and 7x7 feature maps) and the
+    whole step, each as a CUDA graph, with one launch per layer and with the depth-first launches
+    of prom_debug_seq_chain(1); outputs compared."""
+    table = synth.mobilenetv2_pointwise_layers()
+    seed = synth.BASE_SEED + 3
+    rows = []
+    for lo, hi in ((6, 12), (12, 26), (26, 34), (0, 34)):
+        res = {}
+        outs = []
+        for mode in (0, 1):
+            binding.debug_seq_chain(mode)
+            dev = []
+            for i, l in enumerate(table[lo:hi]):
+                d = synth.make_layer(seed, l.cin, l.cout, 0.5, index=lo + i + 1, device="cuda")
+                dev.append(dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride, w_packed=binding.pack_ternary(d["w"]),
+                                bias=d["bias"], mult=d["mult"], shift=d["shift"]))
+            seq = binding.LayerSeq(dev)
+            l0, ll = table[lo], table[hi - 1]
+            hin, win = l0.h * l0.in_stride, l0.w * l0.in_stride
+            x0 = synth.act_post_relu6(seed, (BATCH, hin, win, l0.cin), device="cuda")
+            ws = torch.empty((max(16, seq.workspace_bytes(BATCH, hin, win)),), dtype=torch.uint8, device="cuda")
+            y = torch.empty((BATCH, ll.h, ll.w, ll.cout), dtype=torch.int8, device="cuda")
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
+            for _ in range(5):
+                g.replay()
+            res[mode] = time_region(torch, g.replay, 200, False) / 200 * 1e3
+            outs.append(y.clone())
+        binding.debug_seq_chain(0)
+        rows.append({"layers": f"{lo + 1}..{hi}", "us_one_launch_per_layer": round(res[0], 1),
+                     "us_depth_first": round(res[1], 1), "same_output": bool(torch.equal(outs[0], outs[1]))})
+    return rows
+
+
 def single_layer_configs(torch, binding, synth, bw, p_i8):
     """Configs 1, 2 and 4 as single layers (cold L2), every variant that runs them."""
     flush = torch.empty((FLUSH_BYTES,), dtype=torch.uint8, device="cuda")
@@ -963,6 +1003,8 @@ def run_aux(args):
         out["nominal_tops"] = NOMINAL_I8_TOPS
     elif args.aux == "alu_rate":
         out = alu_rate_probe(torch, binding)
+    elif args.aux == "depth_first":
+        out = depth_first_timing(torch, binding, synth)
     elif args.aux == "act_quantizer":
         out = act_quantizer_timing(torch, binding, bw)
     elif args.aux == "dynamic_layer":
@@ -988,7 +1030,7 @@ def main():
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
     ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
-    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate"],
+    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate", "depth_first"],
                     help="run one of the legs that are off the timed step, alone")
     ap.add_argument("--widths", default=None, help="comma-separated width multipliers: time the sequence at each")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")

@@ -35,10 +35,30 @@ void prom_debug_tc_plan_shape(int64_t m, int cin, int cout, int stride, int fold
                               int groups, int occ, int stages);
 int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
 
-/* Which parts of a layer sequence run depth-first in one launch (see
- * prom_pw_layer_seq): 0 = none (one launch per layer), 1 = the library's
- * choice (default).  Process-wide. */
+/* Depth-first launches inside prom_pw_layer_seq: 0 = none, one launch per layer
+ * (default); 1 = every run of consecutive layers that qualifies (same number
+ * of rows in all of them, only the first may subsample its input; channel
+ * counts that are multiples of 16 with cin >= 32; clamp [0, 127]; no depthwise
+ * convolution, no skip connection; at most 8 tiles of 128 rows per SM) is
+ * executed by one launch in which a CTA takes its tiles of rows through all
+ * the layers of the run.  Every layer's output is still written to the
+ * workspace (each to a buffer of its own) and read back from there by the next
+ * layer.  Results do not depend on the mode; the workspace size does
+ * (prom_layer_seq_workspace_bytes follows the mode; a workspace that is too
+ * small for the depth-first buffers falls back to one launch per layer).
+ * Process-wide. */
 void prom_debug_seq_chain(int mode);
+
+/* Where layer `layer`'s output ([rows][cout] int8) sits in the workspace of a
+ * prom_pw_layer_seq call whose workspace has prom_layer_seq_workspace_bytes
+ * bytes, with AUTO or TC as the variant: the byte offset from the workspace's
+ * start, or -1 for the last layer (its output is y_out_dev) or a bad argument.
+ * *chained (may be NULL) receives 1 when the layer runs inside a depth-first
+ * launch.  A layer's output stays intact until the layer two further on has
+ * run (ping-pong regions) or, inside a depth-first launch, until the next
+ * call. */
+int64_t prom_debug_layer_seq_output_offset(const prom_layer *layers, int n, int batch, int h0,
+                                           int w0, int layer, int *chained);
 
 /* Failure-detection check: launches one warp that waits, with the library's
  * bounded mbarrier wait and a limit of limit_ns nanoseconds (1000 ..

@@ -30,7 +30,7 @@ EXPORTS = [
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
     "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8", "prom_debug_tc_plan_shape", "prom_pw_conv_i8_res",
     "prom_debug_seq_chain", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
-    "prom_debug_once_per_device",
+    "prom_debug_once_per_device", "prom_debug_layer_seq_output_offset",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -106,6 +106,9 @@ def lib():
         L.prom_debug_tc_plan_query.argtypes = [i64, i32, i32, C.POINTER(C.c_int)]
         L.prom_debug_seq_chain.restype = None
         L.prom_debug_seq_chain.argtypes = [i32]
+        L.prom_debug_layer_seq_output_offset.restype = i64
+        L.prom_debug_layer_seq_output_offset.argtypes = [C.POINTER(PromLayer), i32, i32, i32, i32, i32,
+                                                         C.POINTER(C.c_int)]
         L.prom_debug_wait_timeout.restype = i32
         L.prom_debug_wait_timeout.argtypes = [C.c_uint64, vp, vp]
         L.prom_debug_i8_mma_rate.restype = i32
@@ -243,9 +246,18 @@ def debug_tc_plan_query(m: int, cin: int, cout: int):
     return dict(zip(keys, list(out)))
 
 
-def debug_seq_chain(mode: int = 1) -> None:
-    """prom_debug_seq_chain: 0 = one launch per layer, 1 = the library's choice of depth-first parts."""
+def debug_seq_chain(mode: int = 0) -> None:
+    """prom_debug_seq_chain: 0 = one launch per layer (default), 1 = depth-first launches for
+    every run of layers that qualifies."""
     lib().prom_debug_seq_chain(int(mode))
+
+
+def debug_layer_seq_output_offset(seq: "LayerSeq", batch: int, h0: int, w0: int, layer: int):
+    """prom_debug_layer_seq_output_offset: (byte offset of the layer's output in the workspace or
+    -1, whether the layer runs inside a depth-first launch)."""
+    chained = C.c_int(0)
+    off = lib().prom_debug_layer_seq_output_offset(seq.array, seq.n, batch, h0, w0, layer, C.byref(chained))
+    return int(off), bool(chained.value)
 
 
 def debug_wait_timeout(limit_ns: int = 5000, stream=None) -> int:

@@ -20,6 +20,7 @@
 #include "hostutil.cuh"
 #include "simple.cuh"
 #include "tc.cuh"
+#include "chain.cuh"
 #include "smallk.cuh"
 #include "addsub.cuh"
 #include "actquant.cuh"
@@ -174,14 +175,16 @@ static TcTune tune_for(long long m, int cin, int cout, int stride)
     return it == g_shape_tune.end() ? g_tune : it->second;
 }
 
-// Depth-first execution of parts of a sequence (0 = off), set by prom_debug_seq_chain.
-static std::atomic<int> g_seq_chain{1};
+// Depth-first execution of parts of a sequence, set by prom_debug_seq_chain.  Off unless asked
+// for: on the network the library is timed on it is slower than one launch per layer.
+static std::atomic<int> g_seq_chain{0};
 
 static int round_up(int v, int a) { return (v + a - 1) / a * a; }
 
 // Everything of a plan that follows from (fold, nt, groups, occ); false when it does not fit.
 static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, const DeviceInfo &d,
-                         int fold, int nt, int groups, int occ, int want_stages, TcPlan &pl)
+                         int fold, int nt, int groups, int occ, int want_stages, TcPlan &pl,
+                         int cw_max = 128)
 {
     tc::Params &p = pl.p;
     memset(&p, 0, sizeof(p));
@@ -194,7 +197,7 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     const int subs = n_sub / groups;
     const int nt_pad = round_up(nt, 16);
     if (nt_pad > 256) return false;
-    const int cw = kf <= 32 ? 32 : (kf <= 64 ? 64 : 128);
+    const int cw = kf <= 32 ? 32 : (kf <= 64 || cw_max <= 64 ? 64 : 128);
     const int kc = (kf + cw - 1) / cw;
 
     // tile rows
@@ -586,25 +589,225 @@ static void seq_regions(const prom_layer *layers, int n, const SeqShape &s, size
     b += c;
 }
 
-// Bytes of prepared-operand images a sequence wants in its workspace (0 for layers the
-// tensor-core variant cannot run).
-static size_t seq_image_bytes(const prom_layer *layers, int n, const SeqShape &s, const DeviceInfo &d,
-                              std::vector<size_t> *offsets)
+// ---- depth-first chains (chain.cuh) ---------------------------------------------------------
+// A chain is a run of consecutive layers of a sequence that one launch of tc_chain_kernel takes
+// tile by tile through all of them: same number of rows in every layer (only the first may
+// subsample its input), channel counts that are multiples of 16, the clamp [0, 127], no
+// depthwise convolution and no skip connection, and few enough tiles that a CTA interleaves
+// at most chain::kMaxTasks of them.  Each layer of a chain writes to a buffer of its own in the
+// workspace (a ping-pong pair would be overwritten by tiles that are layers ahead).
+struct ChainPlan {
+    int first = 0, last = 0;             // layers [first, last]
+    int tm = 128, n_tasks = 0, grid = 0, box_r = 0;
+    std::vector<TcPlan> prep;            // per layer: the plan whose image layout the kernel reads
+};
+
+static int chain_nt(int cout)
 {
-    size_t total = 0;
-    for (int i = 0; i < n; ++i) {
-        TcPlan pl;
-        size_t bytes = 0;
-        if (tc_shape_plan(s.m[i], layers[i].cin, layers[i].cout, s.map[i], d, pl, kPlanPrepared))
-            bytes = round256((size_t)pl.p.groups * pl.p.image_stride);
-        if (offsets) offsets->push_back(bytes ? total : (size_t)-1);
-        total += bytes;
+    if (cout % 16) return 0;
+    if (cout <= chain::kNtMax) return cout;
+    for (int nt = chain::kNtMax; nt >= 16; nt -= 16)
+        if (cout % nt == 0) return nt;
+    return 0;
+}
+
+static bool chain_layer_ok(const prom_layer &l)
+{
+    return !l.dw_w && !l.add_block_input && l.cin % 16 == 0 && l.cin >= 32 && l.cout % 16 == 0 &&
+           l.rq.act_min == 0 && l.rq.act_max == 127 && chain_nt(l.cout) > 0;
+}
+
+static bool chain_prep_plan(long long m, int cin, int cout, const DeviceInfo &d, TcPlan &pl)
+{
+    const int nt = chain_nt(cout);
+    const RowMap plain{1, 1, 1, 1, 1};
+    return nt > 0 && tc_fill_plan(m, cin, cout, plain, d, 1, nt, cout / nt, 1, 0, pl, chain::kCwMax) &&
+           pl.p.cw <= chain::kCwMax && pl.p.nt_pad <= chain::kNtMax &&
+           (uint32_t)pl.p.nt_pad * 12u + 16u <= chain::kConstSlot;
+}
+
+static void find_chains(const prom_layer *layers, int n, const SeqShape &s, const DeviceInfo &d,
+                        std::vector<ChainPlan> &out)
+{
+    out.clear();
+    if (!g_seq_chain.load()) return;
+    int i = 0;
+    while (i < n) {
+        if (!chain_layer_ok(layers[i]) || s.m[i] <= 0) { ++i; continue; }
+        ChainPlan c;
+        c.first = i;
+        const RowMap &mp = s.map[i];
+        if (mp.stride != 1) {
+            if (mp.wo > 128) { ++i; continue; }
+            c.box_r = 128 / mp.wo;
+            const long long lines = s.m[i] / mp.wo;
+            if (c.box_r > lines) c.box_r = (int)lines;
+            c.tm = c.box_r * mp.wo;
+        }
+        const long long tasks = (s.m[i] + c.tm - 1) / c.tm;
+        if (tasks > (long long)chain::kMaxTasks * 2 * d.sms || s.m[i] + 256 >= (1ll << 31)) { ++i; continue; }
+        c.n_tasks = (int)tasks;
+        int j = i;
+        for (; j < n && j - i < chain::kMaxLayers; ++j) {
+            if (!chain_layer_ok(layers[j]) || s.m[j] != s.m[i] || (j > i && s.map[j].stride != 1)) break;
+            TcPlan pl;
+            if (!chain_prep_plan(s.m[j], layers[j].cin, layers[j].cout, d, pl)) break;
+            c.prep.push_back(pl);
+        }
+        if (j - i < 2) { ++i; continue; }
+        c.last = j - 1;
+        c.grid = c.n_tasks < 2 * d.sms ? c.n_tasks : 2 * d.sms;
+        out.push_back(c);
+        i = j;
     }
-    return total;
+}
+
+static bool make_x_map(CUtensorMap *map, const int8_t *x, int cin, long long rows, int cw, const RowMap *strided,
+                       int box_r)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const CUtensorMapSwizzle sw = cw == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : (cw == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    cuuint32_t es[3] = {1, 1, 1};
+    if (!strided) {
+        cuuint64_t dims[2] = {(cuuint64_t)cin, (cuuint64_t)rows};
+        cuuint64_t strides[1] = {(cuuint64_t)cin};
+        cuuint32_t box[2] = {(cuuint32_t)cw, 128};
+        return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(x), dims, strides, box, es,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
+    // [channel][wo, step stride*cin][batch*ho, step stride*win*cin]
+    const RowMap &mp = *strided;
+    cuuint64_t dims[3] = {(cuuint64_t)cin, (cuuint64_t)mp.wo, (cuuint64_t)(rows / mp.wo)};
+    cuuint64_t strides[2] = {(cuuint64_t)mp.stride * cin, (cuuint64_t)mp.stride * mp.win * cin};
+    cuuint32_t box[3] = {(cuuint32_t)cw, (cuuint32_t)mp.wo, (cuuint32_t)box_r};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t *>(x), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static bool make_y_map(CUtensorMap *map, int8_t *y, int nf, long long rows, int nt)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)nf, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)nf};
+    cuuint32_t box[2] = {(cuuint32_t)nt, 32};
+    cuuint32_t es[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, y, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Where everything of a sequence sits in the caller's workspace.
+struct SeqLayout {
+    size_t ra = 0, rb = 0, dw_off = 0;     // the two ping-pong regions (b ends with the depthwise buffer)
+    std::vector<size_t> img_off;           // per layer: prepared image of a one-launch layer, or -1
+    size_t img_total = 0;
+    std::vector<ChainPlan> chains;
+    std::vector<int> chain_of;             // per layer: its chain, or -1
+    std::vector<size_t> cimg_off, cbuf_off;   // per chain layer: images, output buffer
+    size_t cimg_total = 0, cbuf_total = 0;
+    size_t base() const { return ra + rb; }
+    size_t with_images() const { return round256(base()) + img_total; }
+    size_t with_chains() const { return round256(with_images()) + cimg_total + cbuf_total; }
+};
+
+static void seq_layout(const prom_layer *layers, int n, const SeqShape &s, const DeviceInfo &d, bool want_tc,
+                       SeqLayout &L, bool allow_chains = true)
+{
+    seq_regions(layers, n, s, L.ra, L.rb, &L.dw_off);
+    L.chain_of.assign(n, -1);
+    L.img_off.assign(n, (size_t)-1);
+    L.cimg_off.assign(n, 0);
+    L.cbuf_off.assign(n, 0);
+    if (!want_tc || !d.ok) return;
+    if (allow_chains) find_chains(layers, n, s, d, L.chains);
+    for (size_t c = 0; c < L.chains.size(); ++c)
+        for (int i = L.chains[c].first; i <= L.chains[c].last; ++i) L.chain_of[i] = (int)c;
+    for (int i = 0; i < n; ++i) {
+        if (L.chain_of[i] >= 0) {
+            const ChainPlan &c = L.chains[L.chain_of[i]];
+            const tc::Params &p = c.prep[i - c.first].p;
+            L.cimg_off[i] = L.cimg_total;
+            L.cimg_total += round256((size_t)p.groups * p.image_stride);
+            continue;
+        }
+        TcPlan pl;
+        if (tc_shape_plan(s.m[i], layers[i].cin, layers[i].cout, s.map[i], d, pl, kPlanPrepared)) {
+            L.img_off[i] = L.img_total;
+            L.img_total += round256((size_t)pl.p.groups * pl.p.image_stride);
+        }
+    }
+    for (int i = 0; i < n; ++i)
+        if (L.chain_of[i] >= 0 && i + 1 < n) {
+            L.cbuf_off[i] = L.cimg_total + L.cbuf_total;
+            L.cbuf_total += round256((size_t)s.m[i] * layers[i].cout);
+        }
 }
 
 extern "C" prom_status prom_dw_conv3x3_i8(const int8_t *, int, int, int, int, int, const int8_t *,
                                           const prom_requant *, int8_t *, void *);
+
+// One launch of tc_chain_kernel for layers [c.first, c.last]; conv[] holds every layer's pointers.
+static prom_status launch_chain(const prom_layer *layers, const SeqShape &s, const ChainPlan &c,
+                                const std::vector<Conv> &conv, uint8_t *const *images, bool pdl, bool pdl_next,
+                                cudaStream_t st)
+{
+    chain::Table t;
+    memset(&t, 0, sizeof(t));
+    t.m_rows = s.m[c.first];
+    t.n_layers = c.last - c.first + 1;
+    t.n_tasks = c.n_tasks;
+    t.tm = c.tm;
+    t.pdl = pdl ? 1 : 0;
+    t.pdl_next = pdl_next ? 1 : 0;
+    for (int i = c.first; i <= c.last; ++i) {
+        chain::Layer &L = t.layer[i - c.first];
+        const tc::Params &p = c.prep[i - c.first].p;
+        const bool strided = i == c.first && s.map[i].stride != 1;
+        if (!make_x_map(&L.xmap, conv[i].x, layers[i].cin, s.m[i], p.cw, strided ? &s.map[i] : nullptr, c.box_r))
+            return PROM_ERR_CUDA;
+        L.store_2d = p.n_sub > 1 ? 1 : 0;
+        if (L.store_2d) {
+            if (!make_y_map(&L.ymap, conv[i].y, layers[i].cout, s.m[i], p.nt)) return PROM_ERR_CUDA;
+        } else {
+            L.ymap = L.xmap;       // unused
+        }
+        L.image = images[i];
+        L.y = conv[i].y;
+        L.image_stride = p.image_stride;
+        L.wbias_off = p.off_wbias - p.off_w;
+        L.const_off = p.off_mult - p.off_w;
+        L.const_bytes = (uint32_t)p.nt_pad * 12u + 16u;
+        L.a_tx = strided ? (uint32_t)(p.cw * s.map[i].wo * c.box_r) : 128u * (uint32_t)p.cw;
+        L.n = layers[i].cout;
+        L.cw = p.cw; L.kc = p.kc; L.ksteps_last = p.ksteps_last;
+        L.nt = p.nt; L.nt_pad = p.nt_pad; L.n_sub = p.n_sub;
+        L.x3d = strided ? 1 : 0;
+        L.box_r = c.box_r;
+        L.act_min = layers[i].rq.act_min; L.act_max = layers[i].rq.act_max;
+    }
+    if (raise_smem_limit(chain::tc_chain_kernel, (int)chain::kSmemBytes) != cudaSuccess) return PROM_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)c.grid);
+    cfg.blockDim = dim3(chain::kThreads);
+    cfg.dynamicSmemBytes = chain::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    if (pdl) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, chain::tc_chain_kernel, t);
+    ++g_launches;
+    return cuda_status(e);
+}
 
 static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, int batch, int h0,
                            int w0, void *ws, size_t ws_bytes, int8_t *y_out, prom_variant variant,
@@ -612,15 +815,6 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
 {
     SeqShape s;
     if (!seq_shapes(layers, n, batch, h0, w0, s)) return PROM_ERR_SHAPE;
-    size_t ra, rb, dw_off;
-    seq_regions(layers, n, s, ra, rb, &dw_off);
-    if (ra + rb > 0) {
-        if (!ws) return PROM_ERR_NULL;
-        if (!aligned16(ws)) return PROM_ERR_ALIGN;
-        if (ws_bytes < ra + rb) return PROM_ERR_WORKSPACE;
-    }
-    int8_t *reg[2] = {static_cast<int8_t *>(ws), static_cast<int8_t *>(ws) + ra};
-    int8_t *dw_buf = static_cast<int8_t *>(ws) + dw_off;      // depthwise outputs
     // validate everything before the first launch
     for (int i = 0; i < n; ++i) {
         if (!layers[i].w_packed) return PROM_ERR_NULL;
@@ -636,37 +830,61 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
             return PROM_ERR_UNSUPPORTED;
     }
     DeviceInfo d = device_info();
+    const bool want_tc = variant == PROM_VARIANT_TC || variant == PROM_VARIANT_AUTO;
+    SeqLayout lay;
+    seq_layout(layers, n, s, d, want_tc, lay);
+    const size_t ra = lay.ra, rb = lay.rb;
+    if (ra + rb > 0) {
+        if (!ws) return PROM_ERR_NULL;
+        if (!aligned16(ws)) return PROM_ERR_ALIGN;
+        if (ws_bytes < ra + rb) return PROM_ERR_WORKSPACE;
+    }
     if (!d.ok) return PROM_ERR_CUDA;
+    int8_t *reg[2] = {static_cast<int8_t *>(ws), static_cast<int8_t *>(ws) + ra};
+    int8_t *dw_buf = static_cast<int8_t *>(ws) + lay.dw_off;      // depthwise outputs
+
+    // The images and the chains are optimisations: a workspace without room for them still works.
+    uint8_t *img_base = nullptr, *chain_base = nullptr;
+    if (ws && lay.img_total + lay.cimg_total > 0 && ws_bytes >= lay.with_images())
+        img_base = static_cast<uint8_t *>(ws) + round256(lay.base());
+    if (ws && !lay.chains.empty() && ws_bytes >= lay.with_chains())
+        chain_base = static_cast<uint8_t *>(ws) + round256(lay.with_images());
+    if (!chain_base && !lay.chains.empty()) {
+        // no room: plan again without chains (their layers then want one-launch images)
+        lay = SeqLayout();
+        seq_layout(layers, n, s, d, want_tc, lay, false);
+        img_base = nullptr;
+        if (ws && lay.img_total > 0 && ws_bytes >= lay.with_images())
+            img_base = static_cast<uint8_t *>(ws) + round256(lay.base());
+    }
 
     // plan: which layers run on the tensor cores, and where their prepared operands go
-    const bool want_tc = variant == PROM_VARIANT_TC || variant == PROM_VARIANT_AUTO;
     std::vector<Conv> conv(n);
     std::vector<TcPlan> plan(n);
     std::vector<char> is_tc(n, 0);
-    std::vector<size_t> img_off;
-    size_t img_total = want_tc ? seq_image_bytes(layers, n, s, d, &img_off) : 0;
-    // the images are an optimisation: a workspace without room for them still works
-    uint8_t *img_base = nullptr;
-    if (img_total > 0 && ws && ws_bytes >= round256(ra + rb) + img_total)
-        img_base = static_cast<uint8_t *>(ws) + round256(ra + rb);
+    std::vector<uint8_t *> chain_img(n, nullptr);
     const int8_t *cur = x0;
     long long in_rows = (long long)batch * h0 * w0;
     for (int i = 0; i < n; ++i) {
         Conv &c = conv[i];
+        const bool chained = lay.chain_of[i] >= 0;
         // behind a depthwise convolution the pointwise layer reads that convolution's output
         c.x = layers[i].dw_w ? dw_buf : cur; c.m = s.m[i]; c.cin = layers[i].cin; c.cout = layers[i].cout;
         c.map = s.map[i]; c.in_rows = layers[i].dw_w ? s.m[i] : in_rows;
         c.w = layers[i].w_packed; c.rq = layers[i].rq;
-        c.y = (i == n - 1) ? y_out : reg[i & 1];
+        c.y = (i == n - 1) ? y_out
+              : (chained ? reinterpret_cast<int8_t *>(chain_base + lay.cbuf_off[i]) : reg[i & 1]);
         c.st = st;
         c.pdl = i > 0;
         c.pdl_next = i + 1 < n;
         // The block's input is the output of layer i-2, which sits where this layer's output
-        // goes: the sum is formed in place.
+        // goes (unless a chain wrote it to a buffer of its own: then the sum reads from there).
         if (layers[i].add_block_input) c.res = i == 1 ? x0 : conv[i - 2].y;
-        if (want_tc && c.m > 0 && tc_shape_plan(c.m, c.cin, c.cout, c.map, d, plan[i], kPlanPrepared)) {
+        if (chained) {
+            chain_img[i] = chain_base + lay.cimg_off[i];
+        } else if (want_tc && c.m > 0 && tc_shape_plan(c.m, c.cin, c.cout, c.map, d, plan[i], kPlanPrepared)) {
             is_tc[i] = 1;
-            tc_bind(c, plan[i], img_base && img_off[i] != (size_t)-1 ? img_base + img_off[i] : nullptr);
+            tc_bind(c, plan[i], img_base && lay.img_off[i] != (size_t)-1 ? img_base + lay.img_off[i] : nullptr);
         } else if (variant == PROM_VARIANT_TC && c.m > 0) {
             return PROM_ERR_UNSUPPORTED;
         }
@@ -675,8 +893,8 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
     }
     if (want_tc && tc_set_attr(d) != PROM_OK) return PROM_ERR_CUDA;
 
-    // one launch prepares the operands of every tensor-core layer
-    if (img_base) {
+    // one launch prepares the operands of every tensor-core layer (of a chain: one image per subtile)
+    if (img_base || chain_base) {
         int i = 0;
         while (i < n) {
             tc::PrepTable t;
@@ -684,11 +902,22 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
             size_t smem = 0;
             int ctas = 0;
             for (; i < n && t.n < tc::kMaxPrepLayers; ++i) {
-                if (!is_tc[i]) continue;
+                const TcPlan *pl = nullptr;
+                if (lay.chain_of[i] >= 0) {
+                    const ChainPlan &c = lay.chains[lay.chain_of[i]];
+                    TcPlan tmp = c.prep[i - c.first];
+                    tc_bind(conv[i], tmp, chain_img[i]);
+                    t.layer[t.n] = tmp.p;
+                    pl = &c.prep[i - c.first];
+                } else if (is_tc[i] && plan[i].p.image) {
+                    t.layer[t.n] = plan[i].p;
+                    pl = &plan[i];
+                } else {
+                    continue;
+                }
                 t.first[t.n] = ctas;
-                t.layer[t.n] = plan[i].p;
-                ctas += plan[i].p.groups;
-                if (plan[i].smem > smem) smem = plan[i].smem;
+                ctas += pl->p.groups;
+                if (pl->smem > smem) smem = pl->smem;
                 ++t.n;
             }
             if (t.n == 0) break;
@@ -700,6 +929,13 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
     }
 
     for (int i = 0; i < n; ++i) {
+        if (lay.chain_of[i] >= 0) {
+            const ChainPlan &c = lay.chains[lay.chain_of[i]];
+            prom_status e = launch_chain(layers, s, c, conv, chain_img.data(), c.first > 0, c.last + 1 < n, st);
+            if (e != PROM_OK) return e;
+            i = c.last;
+            continue;
+        }
         if (layers[i].dw_w && s.m[i] > 0) {
             const int stride = layers[i].in_stride;
             const int8_t *src = i == 0 ? x0 : conv[i - 1].y;
@@ -1122,11 +1358,11 @@ size_t prom_layer_seq_workspace_bytes(const prom_layer *layers, int n, int batch
 {
     SeqShape s;
     if (!seq_shapes(layers, n, batch, h0, w0, s)) return 0;
-    size_t a, b;
-    seq_regions(layers, n, s, a, b);
     DeviceInfo d = device_info();
-    const size_t img = d.ok ? seq_image_bytes(layers, n, s, d, nullptr) : 0;
-    return img ? round256(a + b) + img : a + b;
+    SeqLayout lay;
+    seq_layout(layers, n, s, d, true, lay);
+    if (!lay.chains.empty()) return lay.with_chains();
+    return lay.img_total ? lay.with_images() : lay.base();
 }
 
 prom_status prom_pw_layer_seq(const prom_layer *layers, int n, const int8_t *x0_dev, int batch,
@@ -1270,6 +1506,20 @@ prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cyc
 }
 
 void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode ? 1 : 0); }
+
+int64_t prom_debug_layer_seq_output_offset(const prom_layer *layers, int n, int batch, int h0, int w0,
+                                           int layer, int *chained)
+{
+    SeqShape s;
+    if (!seq_shapes(layers, n, batch, h0, w0, s) || layer < 0 || layer >= n - 1) return -1;
+    DeviceInfo d = device_info();
+    SeqLayout lay;
+    seq_layout(layers, n, s, d, true, lay);
+    const bool in_chain = lay.chain_of[layer] >= 0;
+    if (chained) *chained = in_chain ? 1 : 0;
+    if (in_chain) return (int64_t)(round256(lay.with_images()) + lay.cbuf_off[layer]);
+    return (layer & 1) ? (int64_t)lay.ra : 0;
+}
 
 int prom_debug_once_per_device(int device, int key)
 {

@@ -605,6 +605,9 @@ __device__ __forceinline__ void build_image(const Params &p, const int g, const 
             *reinterpret_cast<uint4 *>(blk + swz_offset((uint32_t)c, 1u, 32u)) =
                 make_uint4(wd[4], wd[5], wd[6], wd[7]);
         }
+    else   // no bias step: the block is all zeros, so that a kernel which always issues the step adds nothing
+        for (int i = threadIdx.x; i < ncols_res * 2; i += kThreads)
+            *reinterpret_cast<uint4 *>(wbias_smem + (size_t)i * 16) = make_uint4(0u, 0u, 0u, 0u);
 
     // expand the resident weights from the packed copy into the K-major swizzled operand
     // layout: one table look-up per byte of four codes
