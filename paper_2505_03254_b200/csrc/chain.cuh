@@ -71,39 +71,6 @@ struct Table {
     Layer layer[kMaxLayers];
 };
 
-// The fast epilogue of tc.cuh over one subtile of a width known at compile time.
-template <int NT>
-__device__ __forceinline__ void epi_fast_fixed(uint32_t taddr, const int *cm, int shmax, uint8_t *dst_row,
-                                               uint32_t bar_release)
-{
-    constexpr bool wide = (NT & 15) == 0;
-    const long long r64 = 1ll << (32 + shmax);
-    constexpr int full = NT & ~31;
-#pragma unroll
-    for (int c = 0; c < full; c += 32) {
-        uint32_t v[32];
-        ptx::tmem_ld_x32(taddr + c, v);
-        ptx::tmem_wait_ld();
-        if (c + 32 == NT) tc::release_acc(bar_release);
-        tc::fast_piece<32>(v, cm + c, r64, shmax, dst_row + c, wide);
-    }
-    if constexpr ((NT & 16) != 0) {
-        uint32_t v[16];
-        ptx::tmem_ld_x16(taddr + full, v);
-        ptx::tmem_wait_ld();
-        if (full + 16 == NT) tc::release_acc(bar_release);
-        tc::fast_piece<16>(v, cm + full, r64, shmax, dst_row + full, wide);
-    }
-    if constexpr ((NT & 8) != 0) {
-        constexpr int c8 = NT & ~15;
-        uint32_t v[8];
-        ptx::tmem_ld_x8(taddr + c8, v);
-        ptx::tmem_wait_ld();
-        tc::release_acc(bar_release);
-        tc::fast_piece<8>(v, cm + c8, r64, shmax, dst_row + c8, wide);
-    }
-}
-
 // Any width (a multiple of 8): the same in chunks of 32, 16 and 8 columns.
 __device__ __noinline__ void epi_fast_any(int nt, uint32_t taddr, const int *cm, int shmax, uint8_t *dst_row,
                                           uint32_t bar_release)
@@ -160,7 +127,7 @@ __device__ __forceinline__ int reports_of(const Layer &L) { return L.n_sub >= 2 
 __global__ void __launch_bounds__(kThreads, 2) tc_chain_kernel(const __grid_constant__ Table t)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
     const uint32_t smem_base = ptx::smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -377,10 +344,10 @@ __global__ void __launch_bounds__(kThreads, 2) tc_chain_kernel(const __grid_cons
                         const uint32_t bar_rel = bar_tempty + 8 * grp;
                         if (fast && L.act_min == 0) {
                             switch (nt) {
-                            case 32: epi_fast_fixed<32>(t_lane, cms, shmax, my_row, bar_rel); break;
-                            case 64: epi_fast_fixed<64>(t_lane, cms, shmax, my_row, bar_rel); break;
-                            case 80: epi_fast_fixed<80>(t_lane, cms, shmax, my_row, bar_rel); break;
-                            case 96: epi_fast_fixed<96>(t_lane, cms, shmax, my_row, bar_rel); break;
+                            case 32: tc::epi_fast_fixed<32>(t_lane, cms, shmax, my_row, bar_rel); break;
+                            case 64: tc::epi_fast_fixed<64>(t_lane, cms, shmax, my_row, bar_rel); break;
+                            case 80: tc::epi_fast_fixed<80>(t_lane, cms, shmax, my_row, bar_rel); break;
+                            case 96: tc::epi_fast_fixed<96>(t_lane, cms, shmax, my_row, bar_rel); break;
                             default: epi_fast_any(nt, t_lane, cms, shmax, my_row, bar_rel); break;
                             }
                         } else {

@@ -276,6 +276,39 @@ __device__ __forceinline__ void epi_fast_subtile(const Params &p, uint32_t taddr
     }
 }
 
+// The fast epilogue over one subtile of a width known at compile time: straight-line code.
+template <int NT, bool SIGNED = false>
+__device__ __forceinline__ void epi_fast_fixed(uint32_t taddr, const int *cm, int shmax, uint8_t *dst_row,
+                                               uint32_t bar_release)
+{
+    constexpr bool wide = (NT & 15) == 0;
+    const long long r64 = 1ll << (32 + shmax);
+    constexpr int full = NT & ~31;
+#pragma unroll
+    for (int c = 0; c < full; c += 32) {
+        uint32_t v[32];
+        ptx::tmem_ld_x32(taddr + c, v);
+        ptx::tmem_wait_ld();
+        if (c + 32 == NT) release_acc(bar_release);
+        fast_piece<32, SIGNED>(v, cm + c, r64, shmax, dst_row + c, wide);
+    }
+    if constexpr ((NT & 16) != 0) {
+        uint32_t v[16];
+        ptx::tmem_ld_x16(taddr + full, v);
+        ptx::tmem_wait_ld();
+        if (full + 16 == NT) release_acc(bar_release);
+        fast_piece<16, SIGNED>(v, cm + full, r64, shmax, dst_row + full, wide);
+    }
+    if constexpr ((NT & 8) != 0) {
+        constexpr int c8 = NT & ~15;
+        uint32_t v[8];
+        ptx::tmem_ld_x8(taddr + c8, v);
+        ptx::tmem_wait_ld();
+        release_acc(bar_release);
+        fast_piece<8, SIGNED>(v, cm + c8, r64, shmax, dst_row + c8, wide);
+    }
+}
+
 // The exact epilogue over one subtile, in chunks of CH (32 or 16), then 16 and 8 columns.
 template <int CH>
 __device__ __noinline__ void epi_exact_subtile(int nt, int act_min, int act_max, uint32_t taddr,
@@ -689,8 +722,9 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // 1024-byte aligned base, by pointer arithmetic (a cast through an integer would make every
+    // access below a generic one)
+    uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
     const uint32_t smem_base = ptx::smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int CH = MINB >= 3 ? 16 : 32;     // columns per tensor-memory load in the epilogue
@@ -1001,7 +1035,13 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 if constexpr (MODE == 0 || MODE == 3 || MODE == 4) {
                     // the fast epilogue's clamp: [0, 127] in mode 0, [-128, 127] in mode 4, either in mode 3
                     const bool full_range = MODE == 4 || (MODE == 3 && p.act_min < 0);
-                    if (fast && !full_range) epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
+                    if (fast && !full_range) {
+                        // the widths of the network's large layers get straight-line code
+                        if (CH == 32 && p.nt == 96) epi_fast_fixed<96>(taddr, cms, shmax, my_row, bar_rel);
+                        else if (CH == 32 && p.nt == 64) epi_fast_fixed<64>(taddr, cms, shmax, my_row, bar_rel);
+                        else if (CH == 32 && p.nt == 48) epi_fast_fixed<48>(taddr, cms, shmax, my_row, bar_rel);
+                        else epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
+                    }
                     else if (fast) epi_fast_subtile<CH, true>(p, taddr, cms, shmax, my_row, bar_rel);
                     else epi_exact_subtile<CH>(p.nt, p.act_min, p.act_max, taddr, cms, cbs + ls * p.nt_pad, my_row, bar_rel);
                     if constexpr (MODE == 3) {
