@@ -790,9 +790,15 @@ def single_layer_configs(torch, binding, synth, bw, p_i8):
         y = torch.empty((m, cout), dtype=torch.int8, device="cuda")
         b, o = layer_bytes(m, cin, cout), layer_ops(m, cin, cout)
         roof = max(b / bw, o / p_i8) * 1e6
-        for variant in ("tc", "smallk", "addsub"):
+        prep = binding.pw_prepare(m, cin, wp, cout, rq)
+        for variant in ("tc", "tc_prepared", "addsub"):
             try:
-                fn = lambda: binding.pw_conv_i8(x, wp, cout, rq, y=y, variant=variant)
+                if variant == "tc_prepared":
+                    if prep is None:
+                        continue
+                    fn = lambda: binding.pw_conv_i8_prepared(x, cout, prep, y=y)
+                else:
+                    fn = lambda: binding.pw_conv_i8(x, wp, cout, rq, y=y, variant=variant)
                 fn()
             except binding.PromError:
                 continue

@@ -230,6 +230,35 @@ prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin,
                             const prom_requant *rq, int8_t *y_dev,
                             prom_variant variant, void *cuda_stream);
 
+/* The same layer with its operands prepared ahead of the call.  The paper's
+ * weights are quantised once, before inference (Figure 12, inference branch);
+ * the same holds for everything this library derives from them: the 2-bit
+ * codes expanded to the int8 operand layout of the tensor cores, the bias
+ * digits and the per-channel constants.  prom_pw_prepare writes that form of a
+ * layer into a caller-owned buffer once (one small kernel, asynchronous on the
+ * stream), and prom_pw_conv_i8_prepared runs the tensor-core variant from it,
+ * so that a call no longer rebuilds the operands in every CTA.
+ *   prom_pw_prepared_bytes  size of the buffer for a layer of m rows (the
+ *       launch plan, and with it the layout, depends on m, cin, cout and the
+ *       device); 0 when the tensor-core variant cannot run the shape
+ *   prom_pw_prepare         rq: constants and clamp as for prom_pw_conv_i8
+ *       (their ranges are checked on the device: PROM_ERR_BAD_REQUANT in
+ *       prom_last_device_status); prepared_dev: device, 16-byte aligned,
+ *       prepared_bytes >= prom_pw_prepared_bytes (PROM_ERR_WORKSPACE otherwise)
+ *   prom_pw_conv_i8_prepared  same m, cin, cout as at preparation; the clamp
+ *       [act_min, act_max] is given again and must equal the prepared one;
+ *       x_dev, y_dev as in prom_pw_conv_i8
+ * The buffer stays valid for any number of calls on the device it was
+ * prepared on; its contents are private to this build of the library.
+ * PROM_ERR_UNSUPPORTED where PROM_VARIANT_TC would be. */
+size_t prom_pw_prepared_bytes(int64_t m, int cin, int cout);
+prom_status prom_pw_prepare(int64_t m, int cin, const uint8_t *w_packed_dev, int cout,
+                            const prom_requant *rq, void *prepared_dev, size_t prepared_bytes,
+                            void *cuda_stream);
+prom_status prom_pw_conv_i8_prepared(const int8_t *x_dev, int64_t m, int cin, int cout,
+                                     const void *prepared_dev, int act_min, int act_max,
+                                     int8_t *y_dev, void *cuda_stream);
+
 /* The project convolution of an inverted-residual block with the block's
  * skip connection (Section 2): the layer of prom_pw_conv_i8, then
  *   y[r][o] = clamp(y[r][o] + res[r][o], -128, 127),

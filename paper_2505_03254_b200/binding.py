@@ -31,6 +31,7 @@ EXPORTS = [
     "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8", "prom_debug_tc_plan_shape", "prom_pw_conv_i8_res",
     "prom_debug_seq_chain", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
     "prom_debug_once_per_device", "prom_debug_layer_seq_output_offset",
+    "prom_pw_prepared_bytes", "prom_pw_prepare", "prom_pw_conv_i8_prepared",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -69,6 +70,12 @@ def lib():
         L.prom_pack_ternary.argtypes = [vp, i32, i32, vp, sz, vp]
         L.prom_pw_conv_i8.restype = i32
         L.prom_pw_conv_i8.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant), vp, i32, vp]
+        L.prom_pw_prepared_bytes.restype = sz
+        L.prom_pw_prepared_bytes.argtypes = [i64, i32, i32]
+        L.prom_pw_prepare.restype = i32
+        L.prom_pw_prepare.argtypes = [i64, i32, vp, i32, C.POINTER(PromRequant), vp, sz, vp]
+        L.prom_pw_conv_i8_prepared.restype = i32
+        L.prom_pw_conv_i8_prepared.argtypes = [vp, i64, i32, i32, vp, i32, i32, vp, vp]
         L.prom_pw_conv_i8_res.restype = i32
         L.prom_pw_conv_i8_res.argtypes = [vp, i64, i32, vp, i32, C.POINTER(PromRequant), vp, vp, i32, vp]
         L.prom_pw_conv_i8_acc32.restype = i32
@@ -342,6 +349,30 @@ def pw_conv_i8(x: torch.Tensor, w_packed: torch.Tensor, cout: int, rq: PromRequa
                                  _dev(w_packed, torch.uint8, "w_packed"), cout, C.byref(rq),
                                  _dev(y, torch.int8, "y"), _variant(variant), _stream(stream)),
            "prom_pw_conv_i8")
+    return y
+
+
+def pw_prepare(m: int, cin: int, w_packed: torch.Tensor, cout: int, rq: PromRequant, stream=None):
+    """prom_pw_prepare: the layer's prepared operands (a uint8 CUDA tensor), or None when the
+    tensor-core variant cannot run the shape."""
+    nbytes = int(lib().prom_pw_prepared_bytes(m, cin, cout))
+    if nbytes == 0:
+        return None
+    buf = torch.empty((nbytes,), dtype=torch.uint8, device=w_packed.device)
+    _check(lib().prom_pw_prepare(m, cin, _dev(w_packed, torch.uint8, "w_packed"), cout, C.byref(rq),
+                                 buf.data_ptr(), nbytes, _stream(stream)), "prom_pw_prepare")
+    return buf
+
+
+def pw_conv_i8_prepared(x: torch.Tensor, cout: int, prepared: torch.Tensor, act_min: int = 0, act_max: int = 127,
+                        y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """prom_pw_conv_i8_prepared on device tensors; x is [m, cin] int8."""
+    m, cin = x.shape
+    if y is None:
+        y = torch.empty((m, cout), dtype=torch.int8, device=x.device)
+    _check(lib().prom_pw_conv_i8_prepared(_dev(x, torch.int8, "x"), m, cin, cout,
+                                          _dev(prepared, torch.uint8, "prepared"), act_min, act_max,
+                                          _dev(y, torch.int8, "y"), _stream(stream)), "prom_pw_conv_i8_prepared")
     return y
 
 

@@ -1289,6 +1289,74 @@ prom_status prom_pw_conv_i8(const int8_t *x_dev, int64_t m, int cin, const uint8
     return run_conv(c, variant);
 }
 
+// ---- one layer with operands prepared ahead of the call --------------------------------------
+static bool prepared_plan(long long m, int cin, int cout, const DeviceInfo &d, TcPlan &pl)
+{
+    return m > 0 && tc_shape_plan(m, cin, cout, RowMap{1, 1, 1, 1, 1}, d, pl, kPlanPrepared);
+}
+
+size_t prom_pw_prepared_bytes(int64_t m, int cin, int cout)
+{
+    if (m < 1 || cin < 1 || cin > 4096 || cout < 1 || cout > 4096) return 0;
+    DeviceInfo d = device_info();
+    if (!d.ok) { d.sms = 148; d.smem_optin = 232448; d.smem_total = 233472; d.ok = true; }
+    TcPlan pl;
+    if (!prepared_plan(m, cin, cout, d, pl)) return 0;
+    return round256((size_t)pl.p.groups * pl.p.image_stride);
+}
+
+prom_status prom_pw_prepare(int64_t m, int cin, const uint8_t *w_packed_dev, int cout, const prom_requant *rq,
+                            void *prepared_dev, size_t prepared_bytes, void *cuda_stream)
+{
+    if (!w_packed_dev || !prepared_dev) return PROM_ERR_NULL;
+    prom_status e = check_requant(rq);
+    if (e != PROM_OK) return e;
+    if (m < 1 || cin < 1 || cin > 4096 || cout < 1 || cout > 4096) return PROM_ERR_SHAPE;
+    if (!aligned16(w_packed_dev) || !aligned16(prepared_dev)) return PROM_ERR_ALIGN;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    TcPlan pl;
+    if (!prepared_plan(m, cin, cout, d, pl)) return PROM_ERR_UNSUPPORTED;
+    if (prepared_bytes < round256((size_t)pl.p.groups * pl.p.image_stride)) return PROM_ERR_WORKSPACE;
+    if (tc_set_attr(d) != PROM_OK) return PROM_ERR_CUDA;
+    Conv c;
+    c.x = nullptr; c.m = m; c.cin = cin; c.cout = cout; c.map = RowMap{1, 1, 1, 1, 1}; c.in_rows = m;
+    c.w = w_packed_dev; c.rq = *rq; c.y = nullptr; c.st = static_cast<cudaStream_t>(cuda_stream);
+    c.pdl = false; c.pdl_next = false;
+    tc_bind(c, pl, static_cast<uint8_t *>(prepared_dev));
+    tc::PrepTable t;
+    memset(&t, 0, sizeof(t));
+    t.n = 1;
+    t.first[0] = 0;
+    t.first[1] = pl.p.groups;
+    t.layer[0] = pl.p;
+    tc::tc_prep_kernel<<<pl.p.groups, tc::kThreads, pl.smem, c.st>>>(t);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+prom_status prom_pw_conv_i8_prepared(const int8_t *x_dev, int64_t m, int cin, int cout, const void *prepared_dev,
+                                     int act_min, int act_max, int8_t *y_dev, void *cuda_stream)
+{
+    if (act_min < -128 || act_max > 127 || act_min > act_max) return PROM_ERR_BAD_REQUANT;
+    if (cin < 1 || cin > 4096 || cout < 1 || cout > 4096 || m < 0 || m > (1ll << 40)) return PROM_ERR_SHAPE;
+    if (m == 0) return PROM_OK;
+    if (!x_dev || !prepared_dev || !y_dev) return PROM_ERR_NULL;
+    if (!aligned16(x_dev) || !aligned16(prepared_dev) || !aligned16(y_dev)) return PROM_ERR_ALIGN;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    TcPlan pl;
+    if (!prepared_plan(m, cin, cout, d, pl)) return PROM_ERR_UNSUPPORTED;
+    if (tc_set_attr(d) != PROM_OK) return PROM_ERR_CUDA;
+    Conv c;
+    c.x = x_dev; c.m = m; c.cin = cin; c.cout = cout; c.map = RowMap{1, 1, 1, 1, 1}; c.in_rows = m;
+    c.w = nullptr; c.rq = prom_requant{nullptr, nullptr, nullptr, act_min, act_max}; c.y = y_dev;
+    c.st = static_cast<cudaStream_t>(cuda_stream);
+    c.pdl = false; c.pdl_next = false;
+    tc_bind(c, pl, const_cast<uint8_t *>(static_cast<const uint8_t *>(prepared_dev)));
+    return tc_launch_planned(c, pl);
+}
+
 prom_status prom_pw_conv_i8_res(const int8_t *x_dev, int64_t m, int cin, const uint8_t *w_packed_dev,
                                 int cout, const prom_requant *rq, const int8_t *res_dev,
                                 int8_t *y_dev, prom_variant variant, void *cuda_stream)

@@ -706,7 +706,8 @@ __device__ __forceinline__ void build_image(const Params &p, const int g, const 
         if (bad_consts && threadIdx.x == 0) raise_status(PROM_ERR_BAD_REQUANT);
     }
     if (threadIdx.x == 0) {
-        hdr[0] = shmax; hdr[1] = fast ? 1 : 0; hdr[2] = bad_consts ? 1 : 0; hdr[3] = 0;
+        hdr[0] = shmax; hdr[1] = fast ? 1 : 0; hdr[2] = bad_consts ? 1 : 0;
+        hdr[3] = ((p.act_min & 0xFF) << 8) | (p.act_max & 0xFF);     // the clamp these operands were built for
     }
 }
 
@@ -815,7 +816,11 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
     const uint32_t tmem_base = solo ? 0u : *tmem_slot;
     const int shmax = solo || no_image ? 0 : vw.hdr[0];
     const bool fast = solo || no_image ? false : vw.hdr[1] != 0;
-    const bool bad_consts = solo ? false : (no_image || vw.hdr[2] != 0);
+    // operands prepared for another clamp than this launch's are refused like bad constants
+    const bool wrong_clamp = !solo && split && !no_image &&
+                             vw.hdr[3] != (((p.act_min & 0xFF) << 8) | (p.act_max & 0xFF));
+    if (wrong_clamp && threadIdx.x == 32) raise_status(PROM_ERR_BAD_REQUANT);
+    const bool bad_consts = solo ? false : (no_image || wrong_clamp || vw.hdr[2] != 0);
     if (bad_consts && threadIdx.x == 32) flags[0] = 1;      // stops the producer too
 
     // instruction descriptor: s8 x s8 -> s32, both K-major, M = 128, N = nt_pad

@@ -268,3 +268,44 @@ def test_seeded_shape_fuzz(oracle):
             assert binding.last_device_status() == binding.PROM_OK, (case, m, cin, cout, variant)
             bad = np.argwhere(y.cpu().numpy() != want)
             assert len(bad) == 0, (case, m, cin, cout, variant, lo, hi, bad[:3].tolist())
+
+
+@pytest.mark.parametrize("m,cin,cout", TC_SHAPES)
+def test_tc_from_prepared_operands(oracle, m, cin, cout):
+    """The operands written once by prom_pw_prepare, then two calls from them."""
+    x, lay = make_case(24, m, cin, cout)
+    xd, wp, consts = to_device(x, lay)
+    want = oracle_y(oracle, x, lay)
+    prep = binding.pw_prepare(m, cin, wp, cout, binding.make_requant(*consts))
+    assert prep is not None and prep.numel() == binding.lib().prom_pw_prepared_bytes(m, cin, cout)
+    for _ in range(2):
+        y = torch.full((m, cout), -77, dtype=torch.int8, device="cuda")
+        binding.pw_conv_i8_prepared(xd, cout, prep, y=y)
+        torch.cuda.synchronize()
+        assert first_mismatch(y.cpu().numpy(), want) is None
+
+
+def test_prepared_operands_clamps_and_refusals(oracle):
+    m, cin, cout = 517, 64, 48
+    x, lay = make_case(25, m, cin, cout, shift_lo=0, shift_hi=20)
+    xd, wp, consts = to_device(x, lay)
+    for lo, hi in [(-128, 127), (0, 127), (-5, 90)]:
+        prep = binding.pw_prepare(m, cin, wp, cout, binding.make_requant(*consts, lo, hi))
+        y = binding.pw_conv_i8_prepared(xd, cout, prep, lo, hi)
+        torch.cuda.synchronize()
+        assert first_mismatch(y.cpu().numpy(), oracle_y(oracle, x, lay, lo, hi)) is None, (lo, hi)
+    # operands prepared for one clamp, call made with another: refused on the device
+    y = torch.full((m, cout), -77, dtype=torch.int8, device="cuda")
+    binding.pw_conv_i8_prepared(xd, cout, prep, 0, 127, y=y)
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == binding.PROM_ERR_BAD_REQUANT
+    assert bool((y == -77).all())
+    # shapes the tensor-core variant cannot run have no prepared form
+    assert binding.lib().prom_pw_prepared_bytes(65, 20, 12) == 0
+    assert binding.pw_prepare(65, 20, wp, 12, binding.make_requant(*consts)) is None
+    rc = binding.lib().prom_pw_prepare(65, 20, wp.data_ptr(), 12, binding.make_requant(*consts), wp.data_ptr(), 1 << 20, None)
+    assert rc == binding.PROM_ERR_UNSUPPORTED
+    # too small a buffer
+    small = torch.empty((256,), dtype=torch.uint8, device="cuda")
+    rc = binding.lib().prom_pw_prepare(m, cin, wp.data_ptr(), cout, binding.make_requant(*consts), small.data_ptr(), 256, None)
+    assert rc == binding.PROM_ERR_WORKSPACE
