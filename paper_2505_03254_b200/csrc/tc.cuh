@@ -1045,6 +1045,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                         if (CH == 32 && p.nt == 96) epi_fast_fixed<96>(taddr, cms, shmax, my_row, bar_rel);
                         else if (CH == 32 && p.nt == 64) epi_fast_fixed<64>(taddr, cms, shmax, my_row, bar_rel);
                         else if (CH == 32 && p.nt == 48) epi_fast_fixed<48>(taddr, cms, shmax, my_row, bar_rel);
+                        else if (CH == 32 && p.nt == 32) epi_fast_fixed<32>(taddr, cms, shmax, my_row, bar_rel);
+                        else if (CH == 32 && p.nt == 80) epi_fast_fixed<80>(taddr, cms, shmax, my_row, bar_rel);
                         else epi_fast_subtile<CH>(p, taddr, cms, shmax, my_row, bar_rel);
                     }
                     else if (fast) epi_fast_subtile<CH, true>(p, taddr, cms, shmax, my_row, bar_rel);
