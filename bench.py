@@ -720,6 +720,7 @@ def body_with_depthwise_timing(torch, binding, synth, bw, skips=False):
     ws = torch.empty((seq.workspace_bytes(BATCH, 112, 112),), dtype=torch.uint8, device="cuda")
     y = torch.empty((BATCH, 7, 7, 1280), dtype=torch.int8, device="cuda")
     side = torch.cuda.Stream()
+    torch.cuda.synchronize()          # the inputs were made on the default stream
     with torch.cuda.stream(side):
         binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
     torch.cuda.synchronize()
@@ -760,6 +761,7 @@ def depth_first_timing(torch, binding, synth):
             ws = torch.empty((max(16, seq.workspace_bytes(BATCH, hin, win)),), dtype=torch.uint8, device="cuda")
             y = torch.empty((BATCH, ll.h, ll.w, ll.cout), dtype=torch.int8, device="cuda")
             side = torch.cuda.Stream()
+            torch.cuda.synchronize()          # the inputs were made on the default stream
             with torch.cuda.stream(side):
                 binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
             torch.cuda.synchronize()
@@ -770,9 +772,11 @@ def depth_first_timing(torch, binding, synth):
                 g.replay()
             res[mode] = time_region(torch, g.replay, 200, False) / 200 * 1e3
             outs.append(y.clone())
+            res[("status", mode)] = binding.last_device_status()
         binding.debug_seq_chain(0)
         rows.append({"layers": f"{lo + 1}..{hi}", "us_one_launch_per_layer": round(res[0], 1),
-                     "us_depth_first": round(res[1], 1), "same_output": bool(torch.equal(outs[0], outs[1]))})
+                     "us_depth_first": round(res[1], 1), "same_output": bool(torch.equal(outs[0], outs[1])),
+                     "device_status": [res[("status", 0)], res[("status", 1)]]})
     return rows
 
 
@@ -968,6 +972,7 @@ def run_widths(args):
         ws = torch.empty((seq.workspace_bytes(BATCH, 112, 112),), dtype=torch.uint8, device="cuda")
         y = torch.empty((BATCH, 7, 7, c1), dtype=torch.int8, device="cuda")
         side = torch.cuda.Stream()
+        torch.cuda.synchronize()          # the inputs were made on the default stream
         with torch.cuda.stream(side):
             binding.pw_layer_seq(seq, x0, ws, y_out=y, stream=side)
         torch.cuda.synchronize()
