@@ -140,6 +140,20 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin,
                                   uint8_t *packed_dev, size_t packed_bytes,
                                   float *alpha_dev, void *cuda_stream);
 
+/* The same quantiser over several weight matrices (all the layers of a network)
+ * in one launch: the per-layer call is bound by launch latency, not by the few
+ * megabytes it moves.  jobs: host array of n entries, each as the arguments of
+ * prom_quantize_ternary (alpha_dev may be NULL).  Everything is checked before
+ * the launch.  Asynchronous on `cuda_stream`. */
+typedef struct {
+    const float *w_dev;
+    int cout, cin;
+    uint8_t *packed_dev;
+    size_t packed_bytes;
+    float *alpha_dev;
+} prom_quantize_job;
+prom_status prom_quantize_ternary_batch(const prom_quantize_job *jobs, int n, void *cuda_stream);
+
 /* The int8 depthwise 3x3 convolution between a block's expand and project convolutions
  * (paper, Section 2: depthwise-separable blocks; Section 3.1: its weights are 8-bit, Eq. 4-5).
  * Per channel, with one pixel of zero padding and stride 1 or 2,

@@ -31,7 +31,7 @@ EXPORTS = [
     "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8", "prom_debug_tc_plan_shape", "prom_pw_conv_i8_res",
     "prom_debug_seq_chain", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
     "prom_debug_once_per_device", "prom_debug_layer_seq_output_offset",
-    "prom_pw_prepared_bytes", "prom_pw_prepare", "prom_pw_conv_i8_prepared",
+    "prom_pw_prepared_bytes", "prom_pw_prepare", "prom_pw_conv_i8_prepared", "prom_quantize_ternary_batch",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -45,6 +45,11 @@ class PromLayer(C.Structure):
     _fields_ = [("cin", C.c_int), ("cout", C.c_int), ("in_stride", C.c_int),
                 ("w_packed", C.c_void_p), ("rq", PromRequant),
                 ("dw_w", C.c_void_p), ("dw_rq", PromRequant), ("add_block_input", C.c_int)]
+
+
+class PromQuantizeJob(C.Structure):
+    _fields_ = [("w_dev", C.c_void_p), ("cout", C.c_int), ("cin", C.c_int), ("packed_dev", C.c_void_p),
+                ("packed_bytes", C.c_size_t), ("alpha_dev", C.c_void_p)]
 
 
 class PromError(RuntimeError):
@@ -124,6 +129,8 @@ def lib():
         L.prom_debug_alu_rate.argtypes = [i32, i32, vp, vp, i32, C.POINTER(C.c_int), vp]
         L.prom_debug_once_per_device.restype = i32
         L.prom_debug_once_per_device.argtypes = [i32, i32]
+        L.prom_quantize_ternary_batch.restype = i32
+        L.prom_quantize_ternary_batch.argtypes = [C.POINTER(PromQuantizeJob), i32, vp]
         L.prom_quantize_ternary.restype = i32
         L.prom_quantize_ternary.argtypes = [vp, i32, i32, vp, sz, vp, vp]
         L.prom_requant_from_scale.restype = i32
@@ -322,6 +329,20 @@ def quantize_ternary(w: torch.Tensor, want_alpha: bool = True, stream=None):
                                        packed.numel(), alpha.data_ptr() if want_alpha else None,
                                        _stream(stream)), "prom_quantize_ternary")
     return packed, alpha
+
+
+def quantize_ternary_batch(ws: Sequence[torch.Tensor], out=None, stream=None):
+    """prom_quantize_ternary_batch: a list of device float32 [cout, cin] matrices -> a list of
+    (packed uint8 [cout, ceil(cin/4)], alpha float32 [cout]); `out` may carry that list."""
+    if out is None:
+        out = [(torch.empty((w.shape[0], (w.shape[1] + 3) // 4), dtype=torch.uint8, device=w.device),
+                torch.empty((w.shape[0],), dtype=torch.float32, device=w.device)) for w in ws]
+    jobs = (PromQuantizeJob * len(ws))()
+    for j, (w, (packed, alpha)) in enumerate(zip(ws, out)):
+        jobs[j] = PromQuantizeJob(_dev(w, torch.float32, "w"), w.shape[0], w.shape[1], packed.data_ptr(),
+                                  packed.numel(), alpha.data_ptr())
+    _check(lib().prom_quantize_ternary_batch(jobs, len(ws), _stream(stream)), "prom_quantize_ternary_batch")
+    return out
 
 
 def requant_from_scale(scale: float):

@@ -1036,6 +1036,39 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin, uint8_t
     return cuda_status(cudaGetLastError());
 }
 
+prom_status prom_quantize_ternary_batch(const prom_quantize_job *jobs, int n, void *cuda_stream)
+{
+    if (!jobs) return PROM_ERR_NULL;
+    if (n < 0) return PROM_ERR_SHAPE;
+    for (int i = 0; i < n; ++i) {
+        const prom_quantize_job &j = jobs[i];
+        if (!j.w_dev || !j.packed_dev) return PROM_ERR_NULL;
+        if (j.cout < 1 || j.cin < 1 || j.cout > 4096 || j.cin > 4096) return PROM_ERR_SHAPE;
+        if (j.packed_bytes < prom_packed_bytes(j.cout, j.cin)) return PROM_ERR_WORKSPACE;
+    }
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    for (int base = 0; base < n; base += quant::kMaxJobs) {
+        quant::Jobs t;
+        memset(&t, 0, sizeof(t));
+        t.n = n - base < quant::kMaxJobs ? n - base : quant::kMaxJobs;
+        int rows = 0;
+        for (int i = 0; i < t.n; ++i) {
+            const prom_quantize_job &j = jobs[base + i];
+            t.first_row[i] = rows;
+            rows += j.cout;
+            t.cin[i] = j.cin; t.w[i] = j.w_dev; t.packed[i] = j.packed_dev; t.alpha[i] = j.alpha_dev;
+        }
+        t.first_row[t.n] = rows;
+        const int grid = rows < d.sms * 16 ? rows : d.sms * 16;
+        quant::quantize_ternary_batch_kernel<<<grid, quant::kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+            t, 1e-5);
+        ++g_launches;
+        if (cudaGetLastError() != cudaSuccess) return PROM_ERR_CUDA;
+    }
+    return PROM_OK;
+}
+
 prom_status prom_dw_conv3x3_i8(const int8_t *x_dev, int batch, int h, int w, int c, int stride,
                                const int8_t *w_dev, const prom_requant *rq, int8_t *y_dev,
                                void *cuda_stream)

@@ -78,3 +78,24 @@ def test_nan_weight_is_reported():
     w[1, 3] = float("nan")
     binding.quantize_ternary(w.cuda())
     assert binding.last_device_status() == binding.PROM_ERR_BAD_WEIGHT
+
+
+def test_all_matrices_in_one_launch(oracle):
+    """prom_quantize_ternary_batch over matrices of different shapes equals the per-matrix call
+    and the oracle, codes and scales."""
+    shapes = [(16, 32), (96, 16), (37, 145), (1, 1), (1280, 320), (24, 96), (5, 3)]
+    g = torch.Generator().manual_seed(77)
+    ws = [(torch.randn(s, generator=g) * math.sqrt(2.0 / s[0])).cuda() for s in shapes]
+    outs = binding.quantize_ternary_batch(ws)
+    torch.cuda.synchronize()
+    for w, (packed, alpha) in zip(ws, outs):
+        p1, a1 = binding.quantize_ternary(w)
+        torch.cuda.synchronize()
+        assert torch.equal(packed, p1) and torch.equal(alpha, a1)
+        q, al = oracle.quantize_ternary(w.cpu().numpy())
+        got, bad = oracle.unpack(packed.cpu().numpy(), *w.shape)
+        assert bad == 0 and np.array_equal(got, q)
+    # argument checks happen before anything is launched
+    jobs = (binding.PromQuantizeJob * 1)(binding.PromQuantizeJob(ws[0].data_ptr(), 16, 32, outs[0][0].data_ptr(), 3, None))
+    assert binding.lib().prom_quantize_ternary_batch(jobs, 1, None) == binding.PROM_ERR_WORKSPACE
+    assert binding.lib().prom_quantize_ternary_batch(None, 1, None) == binding.PROM_ERR_NULL
