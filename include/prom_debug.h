@@ -49,6 +49,12 @@ int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
  * Process-wide. */
 void prom_debug_seq_chain(int mode);
 
+/* Which kernel prom_dw_conv3x3_i8 runs: 0 = the library's choice (default: TMA
+ * patches and tensor-core taps for stride 1 with a channel count that is a
+ * multiple of 16, CUDA cores otherwise), 1 = CUDA cores only, 2 = tensor cores
+ * or PROM_ERR_UNSUPPORTED.  Results do not depend on it.  Process-wide. */
+void prom_debug_dw_variant(int variant);
+
 /* Where layer `layer`'s output ([rows][cout] int8) sits in the workspace of a
  * prom_pw_layer_seq call whose workspace has prom_layer_seq_workspace_bytes
  * bytes, with AUTO or TC as the variant: the byte offset from the workspace's

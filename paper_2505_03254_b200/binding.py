@@ -32,6 +32,7 @@ EXPORTS = [
     "prom_debug_seq_chain", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
     "prom_debug_once_per_device", "prom_debug_layer_seq_output_offset",
     "prom_pw_prepared_bytes", "prom_pw_prepare", "prom_pw_conv_i8_prepared", "prom_quantize_ternary_batch",
+    "prom_debug_dw_variant",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -116,6 +117,8 @@ def lib():
         L.prom_debug_tc_plan.argtypes = [i32, i32, i32, i32, i32]
         L.prom_debug_tc_plan_query.restype = i32
         L.prom_debug_tc_plan_query.argtypes = [i64, i32, i32, C.POINTER(C.c_int)]
+        L.prom_debug_dw_variant.restype = None
+        L.prom_debug_dw_variant.argtypes = [i32]
         L.prom_debug_seq_chain.restype = None
         L.prom_debug_seq_chain.argtypes = [i32]
         L.prom_debug_layer_seq_output_offset.restype = i64
@@ -258,6 +261,11 @@ def debug_tc_plan_query(m: int, cin: int, cout: int):
         return None
     keys = ("fold", "nt", "groups", "grid", "stages", "nbuf", "smem", "cw", "est_us_x100")
     return dict(zip(keys, list(out)))
+
+
+def debug_dw_variant(variant: int = 0) -> None:
+    """prom_debug_dw_variant: 0 = the library's choice, 1 = CUDA cores, 2 = tensor cores or refuse."""
+    lib().prom_debug_dw_variant(int(variant))
 
 
 def debug_seq_chain(mode: int = 0) -> None:

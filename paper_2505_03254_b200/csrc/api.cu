@@ -25,6 +25,7 @@
 #include "addsub.cuh"
 #include "actquant.cuh"
 #include "depthwise.cuh"
+#include "dwtc.cuh"
 #include "quantize.cuh"
 #include "peak.cuh"
 
@@ -751,6 +752,48 @@ static void seq_layout(const prom_layer *layers, int n, const SeqShape &s, const
 extern "C" prom_status prom_dw_conv3x3_i8(const int8_t *, int, int, int, int, int, const int8_t *,
                                           const prom_requant *, int8_t *, void *);
 
+// ---- depthwise 3x3 on the tensor cores (dwtc.cuh) ---------------------------------------------
+// 0: the library's choice, 1: CUDA cores only, 2: tensor cores or PROM_ERR_UNSUPPORTED
+static std::atomic<int> g_dw_variant{0};
+
+static prom_status launch_dw_tc(const int8_t *x, int batch, int h, int w, int c, const int8_t *wt,
+                                const prom_requant *rq, int8_t *y, const DeviceInfo &d, cudaStream_t st)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return PROM_ERR_UNSUPPORTED;
+    const int slices = c / 16;
+    int ns = dwtc::kMaxSlices;
+    while (slices % ns) --ns;
+    dwtc::Params p;
+    memset(&p, 0, sizeof(p));
+    p.batch = batch; p.h = h; p.w = w; p.c = c; p.ns = ns; p.groups = slices / ns;
+    p.tiles_y = (h + dwtc::kTileH - 1) / dwtc::kTileH;
+    p.tiles_x = (w + dwtc::kTileW - 1) / dwtc::kTileW;
+    p.tiles = (long long)batch * p.tiles_y * p.tiles_x;
+    p.wt = wt; p.bias = rq->bias; p.mult = rq->mult; p.shift = rq->shift; p.lo = rq->act_min; p.hi = rq->act_max;
+    p.y = y;
+    if (p.groups > 2 * d.sms || p.tiles >= (1ll << 31)) return PROM_ERR_UNSUPPORTED;
+    // {channel in slice, x, y, slice, image}: the slice is a dimension of its own (16 bytes apart),
+    // so that the patches of a group's slices land one after the other in shared memory
+    CUtensorMap map;
+    cuuint64_t dims[5] = {16, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)slices, (cuuint64_t)batch};
+    cuuint64_t strides[4] = {(cuuint64_t)c, (cuuint64_t)w * c, 16, (cuuint64_t)h * w * c};
+    cuuint32_t box[5] = {16, (cuuint32_t)dwtc::kPatchW, (cuuint32_t)dwtc::kPatchH, (cuuint32_t)ns, 1};
+    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<int8_t *>(x), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return PROM_ERR_UNSUPPORTED;
+    if (raise_smem_limit(dwtc::dw3x3_tc_kernel, (int)dwtc::kSmemBytes) != cudaSuccess) return PROM_ERR_CUDA;
+    long long workers = (2ll * d.sms) / p.groups;
+    if (workers < 1) workers = 1;
+    if (workers > p.tiles) workers = p.tiles;
+    const int grid = (int)(workers * p.groups);
+    dwtc::dw3x3_tc_kernel<<<grid, dwtc::kThreads, dwtc::kSmemBytes, st>>>(map, p);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
 // One launch of tc_chain_kernel for layers [c.first, c.last]; conv[] holds every layer's pointers.
 static prom_status launch_chain(const prom_layer *layers, const SeqShape &s, const ChainPlan &c,
                                 const std::vector<Conv> &conv, uint8_t *const *images, bool pdl, bool pdl_next,
@@ -1086,6 +1129,14 @@ prom_status prom_dw_conv3x3_i8(const int8_t *x_dev, int batch, int h, int w, int
     if ((long long)batch * h * w * c >= (1ll << 40)) return PROM_ERR_SHAPE;
     DeviceInfo d = device_info();
     if (!d.ok) return PROM_ERR_CUDA;
+    // stride 1 and whole slices of 16 channels: TMA patches and tensor-core taps
+    const int dw_variant = g_dw_variant.load();
+    if (dw_variant != 1 && stride == 1 && (c & 15) == 0 && !(dw_variant == 0 && (long long)batch * h * w < 128)) {
+        const prom_status e = launch_dw_tc(x_dev, batch, h, w, c, w_dev, rq, y_dev, d,
+                                           static_cast<cudaStream_t>(cuda_stream));
+        if (e != PROM_ERR_UNSUPPORTED) return e;
+    }
+    if (dw_variant == 2) return PROM_ERR_UNSUPPORTED;
     const int rows = dw::rows_per_unit(stride);
     const long long units = (long long)batch * ((ho + rows - 1) / rows) * ((wo + dw::kStrip - 1) / dw::kStrip);
     if (units >= (1ll << 31)) return PROM_ERR_SHAPE;
@@ -1607,6 +1658,8 @@ prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cyc
 }
 
 void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode ? 1 : 0); }
+
+void prom_debug_dw_variant(int variant) { g_dw_variant.store(variant < 0 || variant > 2 ? 0 : variant); }
 
 int64_t prom_debug_layer_seq_output_offset(const prom_layer *layers, int n, int batch, int h0, int w0,
                                            int layer, int *chained)

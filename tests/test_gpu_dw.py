@@ -89,3 +89,39 @@ def test_seeded_shape_fuzz(oracle):
         stride = int(rng.choice([1, 2]))
         lo, hi = (0, 127) if case % 2 else (-128, 127)
         _run(oracle, *_case(100 + case, b, h, w, c), stride, lo, hi)
+
+
+@pytest.mark.parametrize("b,h,w,c", [
+    (2, 14, 14, 96), (1, 7, 7, 960), (3, 28, 28, 144), (2, 9, 13, 32), (1, 16, 8, 16), (2, 33, 17, 64),
+    (1, 56, 56, 48), (4, 5, 40, 80), (1, 1, 130, 16),
+])
+def test_stride_1_on_the_tensor_cores(oracle, b, h, w, c):
+    """The TMA + tcgen05 form (stride 1, whole slices of 16 channels) forced, against the oracle
+    and against the CUDA-core kernel: tiles that end inside the image on both axes, one to four
+    slices per CTA, several channel groups, images smaller than a tile."""
+    x, wt, bias, mult, shift = _case(41, b, h, w, c)
+    try:
+        for lo, hi in ((0, 127), (-128, 127), (3, 100)):
+            binding.debug_dw_variant(2)
+            _run(oracle, x, wt, bias, mult, shift, 1, lo, hi)
+            binding.debug_dw_variant(1)
+            _run(oracle, x, wt, bias, mult, shift, 1, lo, hi)
+    finally:
+        binding.debug_dw_variant(0)
+
+
+def test_tensor_core_form_refuses_what_it_cannot_take():
+    x = torch.zeros((1, 8, 8, 24), dtype=torch.int8, device="cuda")
+    w = torch.zeros((24, 3, 3), dtype=torch.int8, device="cuda")
+    z = torch.zeros((24,), dtype=torch.int32, device="cuda")
+    rq = binding.make_requant(z, z + (1 << 30), torch.zeros((24,), dtype=torch.int8, device="cuda"))
+    try:
+        binding.debug_dw_variant(2)
+        for stride in (1, 2):                       # 24 channels: no whole slices; stride 2: not built
+            with pytest.raises(binding.PromError) as e:
+                binding.dw_conv3x3_i8(x, w, rq, stride=stride)
+            assert e.value.code == binding.PROM_ERR_UNSUPPORTED
+    finally:
+        binding.debug_dw_variant(0)
+    binding.dw_conv3x3_i8(x, w, rq, stride=1)       # the library's choice still runs it
+    torch.cuda.synchronize()
