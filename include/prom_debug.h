@@ -55,6 +55,17 @@ void prom_debug_seq_chain(int mode);
  * or PROM_ERR_UNSUPPORTED.  Results do not depend on it.  Process-wide. */
 void prom_debug_dw_variant(int variant);
 
+/* Which kernel the tensor-core variant of a single pointwise call runs: 0 = the
+ * library's choice (the row-resident kernel, which keeps 128 rows with all their
+ * input channels in shared memory and streams the weight matrix past them, for
+ * layers with Cin >= 512, Cout >= 256 (nearly a multiple of 128 unless Cin >= 768)
+ * and at least four tiles of 128 rows per SM;
+ * the weight-resident kernel otherwise), 1 = the weight-resident kernel only, 2 = the row-resident kernel
+ * or PROM_ERR_UNSUPPORTED (it takes plain matrices with Cin and Cout multiples
+ * of 16, 128 <= Cin <= 1024, Cout >= 64, no residual).  Results do not depend on
+ * it.  Process-wide. */
+void prom_debug_tc_wide(int mode);
+
 /* Where layer `layer`'s output ([rows][cout] int8) sits in the workspace of a
  * prom_pw_layer_seq call whose workspace has prom_layer_seq_workspace_bytes
  * bytes, with AUTO or TC as the variant: the byte offset from the workspace's

@@ -32,7 +32,7 @@ EXPORTS = [
     "prom_debug_seq_chain", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
     "prom_debug_once_per_device", "prom_debug_layer_seq_output_offset",
     "prom_pw_prepared_bytes", "prom_pw_prepare", "prom_pw_conv_i8_prepared", "prom_quantize_ternary_batch",
-    "prom_debug_dw_variant",
+    "prom_debug_dw_variant", "prom_debug_tc_wide",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -119,6 +119,8 @@ def lib():
         L.prom_debug_tc_plan_query.argtypes = [i64, i32, i32, C.POINTER(C.c_int)]
         L.prom_debug_dw_variant.restype = None
         L.prom_debug_dw_variant.argtypes = [i32]
+        L.prom_debug_tc_wide.restype = None
+        L.prom_debug_tc_wide.argtypes = [i32]
         L.prom_debug_seq_chain.restype = None
         L.prom_debug_seq_chain.argtypes = [i32]
         L.prom_debug_layer_seq_output_offset.restype = i64
@@ -266,6 +268,12 @@ def debug_tc_plan_query(m: int, cin: int, cout: int):
 def debug_dw_variant(variant: int = 0) -> None:
     """prom_debug_dw_variant: 0 = the library's choice, 1 = CUDA cores, 2 = tensor cores or refuse."""
     lib().prom_debug_dw_variant(int(variant))
+
+
+def debug_tc_wide(mode: int = 0) -> None:
+    """prom_debug_tc_wide: 0 = the library's choice, 1 = the weight-resident kernel only, 2 = the
+    row-resident kernel or refuse."""
+    lib().prom_debug_tc_wide(int(mode))
 
 
 def debug_seq_chain(mode: int = 0) -> None:

@@ -26,6 +26,7 @@
 #include "actquant.cuh"
 #include "depthwise.cuh"
 #include "dwtc.cuh"
+#include "wide.cuh"
 #include "quantize.cuh"
 #include "peak.cuh"
 
@@ -489,10 +490,177 @@ static prom_status tc_launch_planned(const Conv &c, TcPlan &pl, int mode = 0)
     return cuda_status(e);
 }
 
+static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// ---- the row-resident variant for contraction-bound layers (wide.cuh) ----------------------------
+// 0: the library's choice, 1: never, 2: whenever the shape allows it
+static std::atomic<int> g_wide_mode{0};
+
+// Global scratch of the variant (the expanded weight matrix, bias digits, constants), one buffer
+// per (device, stream), grown on demand and kept until prom_shutdown().
+struct WideKey {
+    int dev;
+    cudaStream_t st;
+    bool operator<(const WideKey &o) const { return dev != o.dev ? dev < o.dev : st < o.st; }
+};
+struct WideBuf { uint8_t *p = nullptr; size_t bytes = 0; };
+static std::mutex g_wide_mu;
+static std::map<WideKey, WideBuf> g_wide_cache;
+
+static uint8_t *wide_scratch_for(cudaStream_t st, size_t bytes)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    std::lock_guard<std::mutex> lk(g_wide_mu);
+    WideBuf &b = g_wide_cache[WideKey{dev, st}];
+    if (b.bytes < bytes) {
+        if (b.p) {
+            cudaStreamSynchronize(st);      // an earlier call may still be reading it
+            cudaFree(b.p);
+            b.p = nullptr; b.bytes = 0;
+        }
+        if (cudaMalloc(reinterpret_cast<void **>(&b.p), bytes) != cudaSuccess) return nullptr;
+        b.bytes = bytes;
+    }
+    return b.p;
+}
+
+static void wide_release_cache()
+{
+    std::lock_guard<std::mutex> lk(g_wide_mu);
+    for (auto &kv : g_wide_cache)
+        if (kv.second.p) cudaFree(kv.second.p);
+    g_wide_cache.clear();
+}
+
+struct WidePlan {
+    wide::Params p;
+    int grid;
+    size_t smem;
+    int k_pad;
+};
+
+// Shapes the variant takes: a plain matrix, whole 16-channel slices on both sides, K within the
+// resident chunks.  `worth` says whether the library picks it by itself.
+static bool wide_plan(const Conv &c, const DeviceInfo &d, WidePlan &pl, bool &worth)
+{
+    if (c.map.stride != 1 || c.res || c.pdl || c.pdl_next) return false;
+    if ((c.cin & 15) || (c.cout & 15) || c.cin < wide::kChunk || c.cin > wide::kChunk * wide::kMaxKc) return false;
+    if (c.cout < 64) return false;
+    if (c.m >= (1ll << 31) - 256) return false;
+    wide::Params &p = pl.p;
+    memset(&p, 0, sizeof(p));
+    p.m = c.m; p.cin = c.cin; p.cout = c.cout;
+    p.kc = (c.cin + wide::kChunk - 1) / wide::kChunk;
+    p.ksteps_last = (c.cin - (p.kc - 1) * wide::kChunk + 31) / 32;
+    p.n_mtiles = (int)((c.m + 127) / 128);
+    p.n_ctiles = (c.cout + wide::kNt - 1) / wide::kNt;
+    pl.k_pad = p.kc * wide::kChunk;
+    // shared memory: resident chunks, weight ring, constants, staging slabs, the bias step's A block, barriers
+    const uint32_t a_bytes = (uint32_t)p.kc * wide::kStageBytes;
+    const uint32_t const_bytes = (wide::kAccs * wide::kConstBytes + 1023u) & ~1023u;
+    const uint32_t fixed = const_bytes + wide::kEpiWarps * wide::kSlabBytes + tc::kAConstBytes + 1024;
+    const long long room = (long long)d.smem_optin - 1024 - a_bytes - fixed;
+    int stages = (int)(room / wide::kStageBytes);
+    if (stages > wide::kMaxStages) stages = wide::kMaxStages;
+    stages &= ~1;                       // one half of the ring per issuing thread
+    if (stages < 4) return false;
+    p.stages = stages;
+    p.off_w = a_bytes;
+    p.off_aconst = p.off_w + (uint32_t)stages * wide::kStageBytes;
+    p.off_const = p.off_aconst + tc::kAConstBytes;
+    p.off_out = p.off_const + const_bytes;
+    p.off_bars = p.off_out + wide::kEpiWarps * wide::kSlabBytes;
+    pl.smem = p.off_bars + 1024 + 1024;
+    // few row tiles: CTAs share a row tile's columns
+    int groups = 1;
+    for (int g = 1; g <= p.n_ctiles; ++g)
+        if (p.n_ctiles % g == 0 && (long long)p.n_mtiles * g <= d.sms) groups = g;
+    p.groups = groups;
+    long long workers = d.sms / groups;
+    if (workers > p.n_mtiles) workers = p.n_mtiles;
+    if (workers < 1) workers = 1;
+    pl.grid = (int)(workers * groups);
+    p.act_min = c.rq.act_min; p.act_max = c.rq.act_max;
+    // measured on B200: it beats the weight-resident kernel from Cin = 512 on when there are
+    // several row tiles per SM (1.4 to 1.7 times at Cin = 960); below that both are bound by the
+    // cost of issuing tcgen05 instructions and the weight-resident kernel issues fewer per output
+    // (a last column tile that is mostly padding costs it that margin unless Cin is large)
+    const bool full_cols = 10 * c.cout > 9 * p.n_ctiles * wide::kNt;
+    worth = c.cin >= 512 && c.cout >= 256 && p.n_mtiles >= 4 * d.sms && (full_cols || c.cin >= 768);
+    return true;
+}
+
+static prom_status launch_wide(const Conv &c, const DeviceInfo &d, WidePlan &pl)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return PROM_ERR_UNSUPPORTED;
+    wide::Params &p = pl.p;
+    const size_t w8_bytes = (size_t)p.n_ctiles * wide::kNt * pl.k_pad;
+    const size_t wb_bytes = (size_t)p.n_ctiles * wide::kWbiasBytes;
+    const size_t cs_bytes = round256((size_t)p.n_ctiles * wide::kConstBytes);
+    uint8_t *scratch = wide_scratch_for(c.st, w8_bytes + wb_bytes + cs_bytes);
+    if (!scratch) return PROM_ERR_CUDA;
+    wide::PrepParams pp;
+    memset(&pp, 0, sizeof(pp));
+    pp.cin = c.cin; pp.cout = c.cout; pp.k_pad = pl.k_pad; pp.w_packed = c.w;
+    pp.bias = c.rq.bias; pp.mult = c.rq.mult; pp.shift = c.rq.shift;
+    pp.act_min = c.rq.act_min; pp.act_max = c.rq.act_max;
+    pp.w8 = reinterpret_cast<int8_t *>(scratch); pp.wbias = scratch + w8_bytes; pp.consts = scratch + w8_bytes + wb_bytes;
+    p.wbias = pp.wbias; p.consts = pp.consts;
+    CUtensorMap xmap, wmap, ymap;
+    cuuint32_t es[2] = {1, 1};
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)c.cin, (cuuint64_t)c.m};
+        cuuint64_t strides[1] = {(cuuint64_t)c.cin};
+        cuuint32_t box[2] = {(cuuint32_t)wide::kChunk, 128};
+        if (enc(&xmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(c.x), dims, strides, box, es,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PROM_ERR_UNSUPPORTED;
+    }
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)pl.k_pad, (cuuint64_t)p.n_ctiles * wide::kNt};
+        cuuint64_t strides[1] = {(cuuint64_t)pl.k_pad};
+        cuuint32_t box[2] = {(cuuint32_t)wide::kChunk, (cuuint32_t)wide::kNt};
+        if (enc(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, pp.w8, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
+            CUDA_SUCCESS)
+            return PROM_ERR_UNSUPPORTED;
+    }
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)c.cout, (cuuint64_t)c.m};
+        cuuint64_t strides[1] = {(cuuint64_t)c.cout};
+        cuuint32_t box[2] = {wide::kEpiCols, 32};
+        if (enc(&ymap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, c.y, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
+            CUDA_SUCCESS)
+            return PROM_ERR_UNSUPPORTED;
+    }
+    if (raise_smem_limit(wide::wide_conv_kernel, d.smem_optin) != cudaSuccess) return PROM_ERR_CUDA;
+    wide::wide_prep_kernel<<<p.n_ctiles, 256, 0, c.st>>>(pp);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return PROM_ERR_CUDA;
+    wide::wide_conv_kernel<<<pl.grid, wide::kThreads, pl.smem, c.st>>>(xmap, wmap, ymap, p);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
 static prom_status launch_tc(const Conv &c)
 {
     DeviceInfo d = device_info();
     if (!d.ok) return PROM_ERR_CUDA;
+    const int wide_mode = g_wide_mode.load();
+    if (wide_mode != 1) {
+        WidePlan wp;
+        bool worth = false;
+        if (wide_plan(c, d, wp, worth) && (worth || wide_mode == 2)) {
+            const prom_status e = launch_wide(c, d, wp);
+            if (e != PROM_ERR_UNSUPPORTED) return e;
+        } else if (wide_mode == 2) {
+            return PROM_ERR_UNSUPPORTED;
+        }
+    }
     TcPlan pl;
     if (!tc_shape_plan(c.m, c.cin, c.cout, c.map, d, pl)) return PROM_ERR_UNSUPPORTED;
     if (tc_set_attr(d) != PROM_OK) return PROM_ERR_CUDA;
@@ -530,7 +698,6 @@ static prom_status run_conv(const Conv &c, prom_variant v)
     }
 }
 
-static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 // Shapes of a sequence; false when it does not chain.
 struct SeqShape {
@@ -1661,6 +1828,8 @@ void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode ? 1 : 0); }
 
 void prom_debug_dw_variant(int variant) { g_dw_variant.store(variant < 0 || variant > 2 ? 0 : variant); }
 
+void prom_debug_tc_wide(int mode) { g_wide_mode.store(mode < 0 || mode > 2 ? 0 : mode); }
+
 int64_t prom_debug_layer_seq_output_offset(const prom_layer *layers, int n, int batch, int h0, int w0,
                                            int layer, int *chained)
 {
@@ -1698,7 +1867,11 @@ int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9)
     return 1;
 }
 
-void prom_shutdown(void) { addsub::release_cache(); }
+void prom_shutdown(void)
+{
+    addsub::release_cache();
+    wide_release_cache();
+}
 
 const char *prom_status_string(prom_status s)
 {
