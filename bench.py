@@ -178,6 +178,43 @@ def alu_rate_probe(torch, binding, iters=2000):
     return out
 
 
+def mma_issue_probe(torch, binding, iters=4096):
+    """SM clocks per tcgen05.mma.kind::i8 of shape 128 x N x 32, per SM and per issuing thread, for
+    1, 2 and 4 issuing threads (as far as tensor memory holds their accumulators)."""
+    cycles = torch.zeros((4096,), dtype=torch.int64, device="cuda")
+    out = []
+    for n in (16, 32, 64, 128, 256):
+        for warps in (1, 2, 4):
+            if warps * 2 * max(n, 64) > 512:
+                continue
+            binding.debug_mma_issue_rate(n, warps, 64, cycles)
+            grid = binding.debug_mma_issue_rate(n, warps, iters, cycles)
+            torch.cuda.synchronize()
+            cyc = int(cycles[:4 * grid].max().item())
+            out.append({"n": n, "issuing_threads": warps, "cycles_per_mma_per_sm": round(cyc / (4.0 * iters * warps), 1),
+                        "cycles_per_mma_per_thread": round(cyc / (4.0 * iters), 1)})
+    return out
+
+
+def l2_copy_probe(torch, binding, iters=4096, region_mb=8):
+    """Bytes per SM clock that every SM pulls from an L2-resident region with 16 KB bulk copies,
+    against the number of copies it keeps in flight; and the total in TB/s by CUDA events."""
+    cycles = torch.zeros((1024,), dtype=torch.int64, device="cuda")
+    region = torch.ones((region_mb << 20,), dtype=torch.uint8, device="cuda")
+    out = []
+    for stages in (1, 2, 3, 4, 6, 8):
+        binding.debug_l2_copy_rate(region, 256, stages, cycles)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        grid = binding.debug_l2_copy_rate(region, iters, stages, cycles)
+        e1.record()
+        e1.synchronize()
+        cyc = int(cycles[:grid].max().item())
+        out.append({"copies_in_flight": stages, "bytes_per_clk_per_sm": round(iters * 16384 / cyc, 1),
+                    "tb_per_s_all_sms": round(iters * 16384 * grid / (e0.elapsed_time(e1) * 1e-3) / 1e12, 2)})
+    return out
+
+
 def build_network(seed, synth, binding=None, device=None, width=1.0):
     """Layer table plus per-layer weights/constants: host arrays for the oracle,
     and (when a binding is given) packed device tensors for the library."""
@@ -1021,6 +1058,10 @@ def run_aux(args):
         out["nominal_tops"] = NOMINAL_I8_TOPS
     elif args.aux == "alu_rate":
         out = alu_rate_probe(torch, binding)
+    elif args.aux == "mma_issue":
+        out = mma_issue_probe(torch, binding)
+    elif args.aux == "l2_copy":
+        out = l2_copy_probe(torch, binding)
     elif args.aux == "depth_first":
         out = depth_first_timing(torch, binding, synth)
     elif args.aux == "act_quantizer":
@@ -1048,7 +1089,7 @@ def main():
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
     ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
-    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate", "depth_first"],
+    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate", "depth_first", "mma_issue", "l2_copy"],
                     help="run one of the legs that are off the timed step, alone")
     ap.add_argument("--widths", default=None, help="comma-separated width multipliers: time the sequence at each")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")

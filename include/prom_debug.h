@@ -103,6 +103,23 @@ prom_status prom_debug_i8_mma_rate(int iters, long long *cycles_dev, int cycles_
 prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cycles_dev,
                                 int cycles_len, int *grid_out, void *cuda_stream);
 
+/* Two more probes behind figures that the design doc argues with.
+ *   mma_issue_rate: how often an SM accepts a tcgen05.mma.kind::i8 of shape
+ *     128 x n x 32 (n a multiple of 16, 16..256) when `warps` threads (1..4, one
+ *     per warp, each with two accumulators of its own: warps * 2 * max(n, 64)
+ *     <= 512 tensor-memory columns, else PROM_ERR_SHAPE) issue iters x 4 of them
+ *     each.  cycles_dev[4 * cta + w] = SM clocks of warp w; cycles_len >= 4 x the
+ *     grid size.
+ *   l2_copy_rate: what one SM can pull from L2.  One thread per SM keeps `stages`
+ *     (1..8) bulk copies of 16 KB in flight out of region_dev (device, 16-byte
+ *     aligned, region_bytes a multiple of 16 KB and at least that; keep it below
+ *     the L2 size), iters copies per SM.  cycles_dev[cta] = SM clocks.
+ * Both write the grid size to *grid_out and are asynchronous on the stream. */
+prom_status prom_debug_mma_issue_rate(int n, int warps, int iters, long long *cycles_dev, int cycles_len,
+                                      int *grid_out, void *cuda_stream);
+prom_status prom_debug_l2_copy_rate(const void *region_dev, uint64_t region_bytes, int iters, int stages,
+                                    long long *cycles_dev, int cycles_len, int *grid_out, void *cuda_stream);
+
 /* Bookkeeping check, no CUDA call: returns 1 the first time (device, key) is
  * asked about on the table used for per-device kernel attributes, 0
  * afterwards (the table behind this entry is a separate instance). */

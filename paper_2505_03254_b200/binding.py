@@ -32,7 +32,7 @@ EXPORTS = [
     "prom_debug_seq_chain", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
     "prom_debug_once_per_device", "prom_debug_layer_seq_output_offset",
     "prom_pw_prepared_bytes", "prom_pw_prepare", "prom_pw_conv_i8_prepared", "prom_quantize_ternary_batch",
-    "prom_debug_dw_variant", "prom_debug_tc_wide",
+    "prom_debug_dw_variant", "prom_debug_tc_wide", "prom_debug_mma_issue_rate", "prom_debug_l2_copy_rate",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -132,6 +132,10 @@ def lib():
         L.prom_debug_i8_mma_rate.argtypes = [i32, vp, i32, C.POINTER(C.c_int), vp]
         L.prom_debug_alu_rate.restype = i32
         L.prom_debug_alu_rate.argtypes = [i32, i32, vp, vp, i32, C.POINTER(C.c_int), vp]
+        L.prom_debug_mma_issue_rate.restype = i32
+        L.prom_debug_mma_issue_rate.argtypes = [i32, i32, i32, vp, i32, C.POINTER(C.c_int), vp]
+        L.prom_debug_l2_copy_rate.restype = i32
+        L.prom_debug_l2_copy_rate.argtypes = [vp, C.c_uint64, i32, i32, vp, i32, C.POINTER(C.c_int), vp]
         L.prom_debug_once_per_device.restype = i32
         L.prom_debug_once_per_device.argtypes = [i32, i32]
         L.prom_quantize_ternary_batch.restype = i32
@@ -315,6 +319,25 @@ def debug_alu_rate(op: int, iters: int, sink: torch.Tensor, cycles: torch.Tensor
     _check(lib().prom_debug_alu_rate(int(op), int(iters), _dev(sink, torch.int32, "sink"),
                                      _dev(cycles, torch.int64, "cycles"), cycles.numel(), C.byref(grid),
                                      _stream(stream)), "prom_debug_alu_rate")
+    return int(grid.value)
+
+
+def debug_mma_issue_rate(n: int, warps: int, iters: int, cycles: torch.Tensor, stream=None) -> int:
+    """prom_debug_mma_issue_rate: cycles[4 * cta + w] = SM clocks of issuing warp w.  Returns the grid size."""
+    grid = C.c_int(0)
+    _check(lib().prom_debug_mma_issue_rate(int(n), int(warps), int(iters), _dev(cycles, torch.int64, "cycles"),
+                                           cycles.numel(), C.byref(grid), _stream(stream)),
+           "prom_debug_mma_issue_rate")
+    return int(grid.value)
+
+
+def debug_l2_copy_rate(region: torch.Tensor, iters: int, stages: int, cycles: torch.Tensor, stream=None) -> int:
+    """prom_debug_l2_copy_rate: every SM copies 16 KB pieces of `region` (device uint8) into its shared
+    memory, `stages` at a time.  Returns the grid size."""
+    grid = C.c_int(0)
+    _check(lib().prom_debug_l2_copy_rate(_dev(region, torch.uint8, "region"), region.numel(), int(iters),
+                                         int(stages), _dev(cycles, torch.int64, "cycles"), cycles.numel(),
+                                         C.byref(grid), _stream(stream)), "prom_debug_l2_copy_rate")
     return int(grid.value)
 
 

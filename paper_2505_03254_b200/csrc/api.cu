@@ -1824,6 +1824,45 @@ prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cyc
     return cuda_status(cudaGetLastError());
 }
 
+prom_status prom_debug_mma_issue_rate(int n, int warps, int iters, long long *cycles_dev, int cycles_len,
+                                      int *grid_out, void *cuda_stream)
+{
+    if (!cycles_dev || !grid_out) return PROM_ERR_NULL;
+    if (n < 16 || n > 256 || (n & 15) || warps < 1 || warps > 4 || iters < 1 || iters > (1 << 20))
+        return PROM_ERR_SHAPE;
+    if (warps * 2 * (n > 64 ? n : 64) > 512) return PROM_ERR_SHAPE;     // tensor-memory columns
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    if (cycles_len < 4 * d.sms) return PROM_ERR_WORKSPACE;
+    *grid_out = d.sms;
+    if (raise_smem_limit(peak::mma_issue_rate_kernel, peak::kMmaSmem) != cudaSuccess) return PROM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(cycles_dev, 0, sizeof(long long) * 4 * (size_t)d.sms, st) != cudaSuccess) return PROM_ERR_CUDA;
+    peak::mma_issue_rate_kernel<<<d.sms, peak::kMmaThreads, peak::kMmaSmem, st>>>(iters, n, warps, cycles_dev);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
+prom_status prom_debug_l2_copy_rate(const void *region_dev, uint64_t region_bytes, int iters, int stages,
+                                    long long *cycles_dev, int cycles_len, int *grid_out, void *cuda_stream)
+{
+    if (!region_dev || !cycles_dev || !grid_out) return PROM_ERR_NULL;
+    if (!aligned16(region_dev)) return PROM_ERR_ALIGN;
+    if (region_bytes < peak::kCopyBytes || region_bytes % peak::kCopyBytes || iters < 1 || iters > (1 << 20) ||
+        stages < 1 || stages > peak::kCopyMaxStages)
+        return PROM_ERR_SHAPE;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    if (cycles_len < d.sms) return PROM_ERR_WORKSPACE;
+    *grid_out = d.sms;
+    const int smem = peak::kCopyMaxStages * (int)peak::kCopyBytes + 256;
+    if (raise_smem_limit(peak::l2_copy_rate_kernel, smem) != cudaSuccess) return PROM_ERR_CUDA;
+    peak::l2_copy_rate_kernel<<<d.sms, 32, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
+        static_cast<const uint8_t *>(region_dev), (unsigned long long)region_bytes, iters, stages, cycles_dev);
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
 void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode ? 1 : 0); }
 
 void prom_debug_dw_variant(int variant) { g_dw_variant.store(variant < 0 || variant > 2 ? 0 : variant); }

@@ -112,4 +112,102 @@ __global__ void __launch_bounds__(kAluThreads, 2) alu_rate_kernel(int iters, int
     if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
 }
 
+// How often an SM accepts a tcgen05.mma: `nwarps` threads (lane 0 of warps 0..nwarps-1) each issue
+// `iters` rounds of four 128 x n x 32 MMAs on fixed shared-memory operands into two accumulators
+// of their own (tensor-memory columns [w * 2 * stride, (w + 1) * 2 * stride), stride = max(n, 64);
+// the host checks that nwarps * 2 * stride <= 512), then commit and wait (bounded).
+// cycles[4 * blockIdx.x + w] = SM clocks of warp w from its first issue to its drain.
+__global__ void __launch_bounds__(kMmaThreads, 1) mma_issue_rate_kernel(int iters, int n, int nwarps, long long *cycles)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+    __shared__ uint64_t bar[4];
+    __shared__ uint32_t tmem_slot;
+    for (int i = threadIdx.x; i < (kMmaM + kMmaN) * kMmaRowBytes / 4; i += kMmaThreads)
+        reinterpret_cast<uint32_t *>(smem)[i] = 0x01010101u * (uint32_t)(i & 3);
+    if (threadIdx.x < 4) {
+        ptx::mbar_init(ptx::smem_u32(&bar[threadIdx.x]), 1);
+        ptx::mbar_init_fence();
+    }
+    if (threadIdx.x < 32) ptx::tmem_alloc(ptx::smem_u32(&tmem_slot), 512u);
+    ptx::fence_proxy_async_smem();
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    const int warp = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0 && warp < nwarps) {
+        const uint32_t a_addr = ptx::smem_u32(smem), b_addr = a_addr + kMmaM * kMmaRowBytes;
+        const uint64_t hi = (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+        const uint64_t a0 = hi | (uint64_t)((a_addr >> 4) & 0x3FFFu), b0 = hi | (uint64_t)((b_addr >> 4) & 0x3FFFu);
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+        const uint32_t stride = n > 64 ? (uint32_t)n : 64u;
+        const uint32_t bar_addr = ptx::smem_u32(&bar[warp]);
+        const long long t0 = clock64();
+        for (int it = 0; it < iters; ++it) {
+            const uint32_t d = tmem + (uint32_t)warp * 2u * stride + (uint32_t)(it & 1) * stride;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) ptx::mma_i8(d, a0 + 2 * ks, b0 + 2 * ks, idesc, 1u);
+        }
+        ptx::mma_commit(bar_addr);
+        const unsigned long long g0 = ptx::globaltimer();
+        bool done = false;
+        while (!(done = ptx::mbar_try_wait(bar_addr, 0u)) && ptx::globaltimer() - g0 < kDrainLimitNs) {}
+        if (!done) raise_status(PROM_ERR_TIMEOUT);
+        cycles[4 * blockIdx.x + warp] = clock64() - t0;
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, 512u);
+    }
+}
+
+// What an SM can pull out of L2: one thread per CTA (one CTA per SM) keeps `stages` bulk copies
+// of 16 KB in flight from a region of global memory that fits L2 (every CTA starts at another
+// offset and wraps around), `iters` copies in all; all waits bounded.
+// cycles[blockIdx.x] = SM clocks from the first copy to the last arrival.
+constexpr uint32_t kCopyBytes = 16384;
+constexpr int kCopyMaxStages = 8;
+__global__ void __launch_bounds__(32, 1)
+l2_copy_rate_kernel(const uint8_t *src, unsigned long long region, int iters, int stages, long long *cycles)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((128u - (ptx::smem_u32(smem_raw) & 127u)) & 127u);
+    __shared__ uint64_t bar[kCopyMaxStages];
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < stages; ++i) ptx::mbar_init(ptx::smem_u32(&bar[i]), 1);
+        ptx::mbar_init_fence();
+        const unsigned long long nchunks = region / kCopyBytes;
+        unsigned long long c = ((unsigned long long)blockIdx.x * 7ull) % nchunks;
+        bool ok = true;
+        const long long t0 = clock64();
+        // ring position and phase advance by additions (a division per copy would be what is measured)
+        int s = 0;
+        uint32_t ph = 1;                            // parity of the stage's previous use; no wait in round 0
+        const uint32_t bar0 = ptx::smem_u32(&bar[0]), dst0 = ptx::smem_u32(smem);
+        for (int it = 0; it < iters + stages && ok; ++it) {
+            const uint32_t b = bar0 + 8u * (uint32_t)s;
+            if (it >= stages) {
+                const unsigned long long g0 = ptx::globaltimer();
+                while (!ptx::mbar_try_wait(b, ph))
+                    if (ptx::globaltimer() - g0 > kDrainLimitNs) { ok = false; break; }
+            }
+            if (it < iters && ok) {
+                ptx::mbar_expect_tx(b, kCopyBytes);
+                ptx::bulk_load(dst0 + (uint32_t)s * kCopyBytes, src + c * kCopyBytes, kCopyBytes, b);
+                if (++c == nchunks) c = 0;
+            }
+            if (++s == stages) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) {
+            raise_status(PROM_ERR_TIMEOUT);
+            const unsigned long long g0 = ptx::globaltimer();        // let what is in flight land
+            while (ptx::globaltimer() - g0 < 100000ull) {}
+        }
+        cycles[blockIdx.x] = clock64() - t0;
+    }
+}
+
 }}  // namespace prom::peak
