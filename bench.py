@@ -178,6 +178,30 @@ def alu_rate_probe(torch, binding, iters=2000):
     return out
 
 
+def write_bandwidth_probe(torch, gib=1):
+    """What the GPU sustains when it only writes: a fill and a memset of `gib` GiB, best of 5 each
+    (GB/s).  A copy moves read + write bytes at the copy bandwidth, i.e. half of it each way; a
+    kernel that writes far more than it reads (an expand layer) is held to this figure instead."""
+    n = gib << 30
+    buf = torch.empty((n,), dtype=torch.uint8, device="cuda")
+    out = {}
+    for name, fn in (("fill", lambda: buf.fill_(3)), ("memset", lambda: buf.zero_())):
+        ts = []
+        for i in range(7):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            e1.synchronize()
+            if i >= 2:
+                ts.append(e0.elapsed_time(e1))
+        out[name + "_gbs"] = round(n / min(ts) / 1e6, 1)
+    del buf
+    out["gbs"] = max(out["fill_gbs"], out["memset_gbs"])
+    out["how"] = f"torch fill_ / zero_ over {gib} GiB of uint8, best of 5, CUDA events"
+    return out
+
+
 def mma_issue_probe(torch, binding, iters=4096):
     """SM clocks per tcgen05.mma.kind::i8 of shape 128 x N x 32, per SM and per issuing thread, for
     1, 2 and 4 issuing threads (as far as tensor memory holds their accumulators)."""
@@ -531,6 +555,16 @@ def run_gpu(args):
                 "us_per_launch": ms_per_step * 1e3 / (launches / args.steps),
                 "step_roofline_us": sum(roof_us),
                 "step_roofline_frac": sum(roof_us) / (ms_per_step * 1e3)}
+
+    # The copy bandwidth is read + write; on its own the write path sustains less than the copy's
+    # total (measured here), and the expand layers write six times what they read.  Beside the
+    # figure against the copy bandwidth, the step's roofline with the write path as a third roof.
+    if rank == 0:
+        wr = write_bandwidth_probe(torch)
+        roof_w_us = [max(r, m * l.cout / (wr["gbs"] * 1e9) * 1e6) for r, m, l in zip(roof_us, ms_layers, table)]
+        roofline["write_path"] = {"gbs": wr["gbs"], "probe": wr, "step_roofline_us": sum(roof_w_us),
+                                  "step_roofline_frac": sum(roof_w_us) / (ms_per_step * 1e3),
+                                  "layers_bound_by_it": sum(1 for a, b in zip(roof_w_us, roof_us) if a > b)}
 
     # second roof of the requantising epilogue: one 32-bit high multiply per output, at the rate
     # the probe above measured on this GPU (lanes per clock per SM) and the sampled SM clock
@@ -1058,6 +1092,8 @@ def run_aux(args):
         out["nominal_tops"] = NOMINAL_I8_TOPS
     elif args.aux == "alu_rate":
         out = alu_rate_probe(torch, binding)
+    elif args.aux == "write_bw":
+        out = write_bandwidth_probe(torch)
     elif args.aux == "mma_issue":
         out = mma_issue_probe(torch, binding)
     elif args.aux == "l2_copy":
@@ -1089,7 +1125,7 @@ def main():
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
     ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
-    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate", "depth_first", "mma_issue", "l2_copy"],
+    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate", "depth_first", "mma_issue", "l2_copy", "write_bw"],
                     help="run one of the legs that are off the timed step, alone")
     ap.add_argument("--widths", default=None, help="comma-separated width multipliers: time the sequence at each")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")

@@ -62,9 +62,11 @@ void prom_debug_dw_variant(int variant);
  * and at least four tiles of 128 rows per SM;
  * the weight-resident kernel otherwise), 1 = the weight-resident kernel only, 2 = the row-resident kernel
  * or PROM_ERR_UNSUPPORTED (it takes plain matrices with Cin and Cout multiples
- * of 16, 128 <= Cin <= 1024, Cout >= 64, no residual).  Results do not depend on
- * it.  Process-wide. */
-void prom_debug_tc_wide(int mode);
+ * of 16, 128 <= Cin <= 1024, Cout >= 64, no residual).  blocks: 128-channel
+ * blocks per column tile of that kernel, 1 (MMA N = 128) or 2 (N = 256; refused
+ * where four 32 KB stages do not fit beside the resident rows), 0 = the
+ * planner's choice.  Results do not depend on either.  Process-wide. */
+void prom_debug_tc_wide(int mode, int blocks);
 
 /* Where layer `layer`'s output ([rows][cout] int8) sits in the workspace of a
  * prom_pw_layer_seq call whose workspace has prom_layer_seq_workspace_bytes

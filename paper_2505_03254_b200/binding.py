@@ -120,7 +120,7 @@ def lib():
         L.prom_debug_dw_variant.restype = None
         L.prom_debug_dw_variant.argtypes = [i32]
         L.prom_debug_tc_wide.restype = None
-        L.prom_debug_tc_wide.argtypes = [i32]
+        L.prom_debug_tc_wide.argtypes = [i32, i32]
         L.prom_debug_seq_chain.restype = None
         L.prom_debug_seq_chain.argtypes = [i32]
         L.prom_debug_layer_seq_output_offset.restype = i64
@@ -274,10 +274,11 @@ def debug_dw_variant(variant: int = 0) -> None:
     lib().prom_debug_dw_variant(int(variant))
 
 
-def debug_tc_wide(mode: int = 0) -> None:
-    """prom_debug_tc_wide: 0 = the library's choice, 1 = the weight-resident kernel only, 2 = the
-    row-resident kernel or refuse."""
-    lib().prom_debug_tc_wide(int(mode))
+def debug_tc_wide(mode: int = 0, blocks: int = 0) -> None:
+    """prom_debug_tc_wide: mode 0 = the library's choice, 1 = the weight-resident kernel only, 2 = the
+    row-resident kernel or refuse; blocks = 128-channel blocks per column tile of that kernel (1, 2,
+    0 = the planner's choice)."""
+    lib().prom_debug_tc_wide(int(mode), int(blocks))
 
 
 def debug_seq_chain(mode: int = 0) -> None:

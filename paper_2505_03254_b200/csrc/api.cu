@@ -495,6 +495,7 @@ static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
 // ---- the row-resident variant for contraction-bound layers (wide.cuh) ----------------------------
 // 0: the library's choice, 1: never, 2: whenever the shape allows it
 static std::atomic<int> g_wide_mode{0};
+static std::atomic<int> g_wide_nb{0};        // 0: the planner's choice; 1 or 2: forced (tests)
 
 // Global scratch of the variant (the expanded weight matrix, bias digits, constants), one buffer
 // per (device, stream), grown on demand and kept until prom_shutdown().
@@ -554,20 +555,28 @@ static bool wide_plan(const Conv &c, const DeviceInfo &d, WidePlan &pl, bool &wo
     p.kc = (c.cin + wide::kChunk - 1) / wide::kChunk;
     p.ksteps_last = (c.cin - (p.kc - 1) * wide::kChunk + 31) / 32;
     p.n_mtiles = (int)((c.m + 127) / 128);
-    p.n_ctiles = (c.cout + wide::kNt - 1) / wide::kNt;
     pl.k_pad = p.kc * wide::kChunk;
     // shared memory: resident chunks, weight ring, constants, staging slabs, the bias step's A block, barriers
     const uint32_t a_bytes = (uint32_t)p.kc * wide::kStageBytes;
     const uint32_t const_bytes = (wide::kAccs * wide::kConstBytes + 1023u) & ~1023u;
     const uint32_t fixed = const_bytes + wide::kEpiWarps * wide::kSlabBytes + tc::kAConstBytes + 1024;
     const long long room = (long long)d.smem_optin - 1024 - a_bytes - fixed;
-    int stages = (int)(room / wide::kStageBytes);
+    // 128-channel column tiles.  256-channel tiles (half as many tcgen05 instructions per output;
+    // on request, where four stages of 32 KB fit beside the resident rows) measured slower: tensor
+    // memory then holds one accumulator per issuing thread, so a thread's MMAs cannot overlap the
+    // read-out of its previous tile (1.6 M x 384 -> 1280: 1416 against 1090 us, x 512 -> 256: 490
+    // against 300 us).
+    int nb = g_wide_nb.load();
+    if (nb == 0) nb = 1;
+    p.nb = nb;
+    int stages = (int)(room / (nb * wide::kStageBytes));
     if (stages > wide::kMaxStages) stages = wide::kMaxStages;
     stages &= ~1;                       // one half of the ring per issuing thread
     if (stages < 4) return false;
     p.stages = stages;
+    p.n_ctiles = (c.cout + nb * wide::kNt - 1) / (nb * wide::kNt);
     p.off_w = a_bytes;
-    p.off_aconst = p.off_w + (uint32_t)stages * wide::kStageBytes;
+    p.off_aconst = p.off_w + (uint32_t)stages * nb * wide::kStageBytes;
     p.off_const = p.off_aconst + tc::kAConstBytes;
     p.off_out = p.off_const + const_bytes;
     p.off_bars = p.off_out + wide::kEpiWarps * wide::kSlabBytes;
@@ -586,7 +595,7 @@ static bool wide_plan(const Conv &c, const DeviceInfo &d, WidePlan &pl, bool &wo
     // several row tiles per SM (1.4 to 1.7 times at Cin = 960); below that both are bound by the
     // cost of issuing tcgen05 instructions and the weight-resident kernel issues fewer per output
     // (a last column tile that is mostly padding costs it that margin unless Cin is large)
-    const bool full_cols = 10 * c.cout > 9 * p.n_ctiles * wide::kNt;
+    const bool full_cols = 10 * c.cout > 9 * p.n_ctiles * nb * wide::kNt;
     worth = c.cin >= 512 && c.cout >= 256 && p.n_mtiles >= 4 * d.sms && (full_cols || c.cin >= 768);
     return true;
 }
@@ -596,9 +605,10 @@ static prom_status launch_wide(const Conv &c, const DeviceInfo &d, WidePlan &pl)
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return PROM_ERR_UNSUPPORTED;
     wide::Params &p = pl.p;
-    const size_t w8_bytes = (size_t)p.n_ctiles * wide::kNt * pl.k_pad;
-    const size_t wb_bytes = (size_t)p.n_ctiles * wide::kWbiasBytes;
-    const size_t cs_bytes = round256((size_t)p.n_ctiles * wide::kConstBytes);
+    const int blocks = p.n_ctiles * p.nb;           // of 128 channels
+    const size_t w8_bytes = (size_t)blocks * wide::kNt * pl.k_pad;
+    const size_t wb_bytes = (size_t)blocks * wide::kWbiasBytes;
+    const size_t cs_bytes = round256((size_t)blocks * wide::kConstBytes);
     uint8_t *scratch = wide_scratch_for(c.st, w8_bytes + wb_bytes + cs_bytes);
     if (!scratch) return PROM_ERR_CUDA;
     wide::PrepParams pp;
@@ -620,9 +630,9 @@ static prom_status launch_wide(const Conv &c, const DeviceInfo &d, WidePlan &pl)
             return PROM_ERR_UNSUPPORTED;
     }
     {
-        cuuint64_t dims[2] = {(cuuint64_t)pl.k_pad, (cuuint64_t)p.n_ctiles * wide::kNt};
+        cuuint64_t dims[2] = {(cuuint64_t)pl.k_pad, (cuuint64_t)blocks * wide::kNt};
         cuuint64_t strides[1] = {(cuuint64_t)pl.k_pad};
-        cuuint32_t box[2] = {(cuuint32_t)wide::kChunk, (cuuint32_t)wide::kNt};
+        cuuint32_t box[2] = {(cuuint32_t)wide::kChunk, (cuuint32_t)(p.nb * wide::kNt)};
         if (enc(&wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, pp.w8, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
             CUDA_SUCCESS)
@@ -638,7 +648,7 @@ static prom_status launch_wide(const Conv &c, const DeviceInfo &d, WidePlan &pl)
             return PROM_ERR_UNSUPPORTED;
     }
     if (raise_smem_limit(wide::wide_conv_kernel, d.smem_optin) != cudaSuccess) return PROM_ERR_CUDA;
-    wide::wide_prep_kernel<<<p.n_ctiles, 256, 0, c.st>>>(pp);
+    wide::wide_prep_kernel<<<blocks, 256, 0, c.st>>>(pp);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return PROM_ERR_CUDA;
     wide::wide_conv_kernel<<<pl.grid, wide::kThreads, pl.smem, c.st>>>(xmap, wmap, ymap, p);
@@ -1867,7 +1877,11 @@ void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode ? 1 : 0); }
 
 void prom_debug_dw_variant(int variant) { g_dw_variant.store(variant < 0 || variant > 2 ? 0 : variant); }
 
-void prom_debug_tc_wide(int mode) { g_wide_mode.store(mode < 0 || mode > 2 ? 0 : mode); }
+void prom_debug_tc_wide(int mode, int blocks)
+{
+    g_wide_mode.store(mode < 0 || mode > 2 ? 0 : mode);
+    g_wide_nb.store(blocks == 1 || blocks == 2 ? blocks : 0);
+}
 
 int64_t prom_debug_layer_seq_output_offset(const prom_layer *layers, int n, int batch, int h0, int w0,
                                            int layer, int *chained)

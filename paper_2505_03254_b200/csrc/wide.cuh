@@ -48,11 +48,12 @@ struct Params {
     int cin, cout;
     int kc, ksteps_last;        // chunks of K; 32-byte MMA steps in the last one
     int n_mtiles, n_ctiles;     // row tiles, column tiles
+    int nb;                     // 128-channel blocks per column tile: 1 (MMA N = 128) or 2 (N = 256)
     int groups;                 // CTAs that share a row tile's columns; n_ctiles % groups == 0
     int stages;                 // of the weight ring
     uint32_t off_w, off_const, off_out, off_aconst, off_bars;
-    const uint8_t *wbias;       // [n_ctiles][kWbiasBytes]
-    const uint8_t *consts;      // [n_ctiles][kConstBytes]
+    const uint8_t *wbias;       // [n_ctiles * nb][kWbiasBytes]
+    const uint8_t *consts;      // [n_ctiles * nb][kConstBytes]
     int act_min, act_max;
 };
 
@@ -181,6 +182,12 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
     const int nworkers = gridDim.x / p.groups;
     const int cols = p.n_ctiles / p.groups;                       // column tiles g, g + groups, ...
     const uint32_t half = (uint32_t)p.stages >> 1;                // stages per issuing thread
+    // With 128-channel tiles the k-th unit of thread t uses slot t + 2 (k & 1) of four (accumulator,
+    // constants); with 256-channel tiles a thread has the one slot t, twice as wide.
+    const uint32_t nb = (uint32_t)p.nb, nt = nb * (uint32_t)kNt;
+    const uint32_t w_stage = nb * kStageBytes;
+    auto slot_of = [&](uint32_t t, uint32_t k) { return nb == 1u ? t + 2u * (k & 1u) : t; };
+    auto phase_of = [&](uint32_t k) { return nb == 1u ? (k >> 1) & 1u : k & 1u; };
 
     // ---- prologue -----------------------------------------------------------------------------
     if (warp == 0) {
@@ -194,9 +201,9 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
         } else if (lane < kMaxKc + kMaxStages + kAccs) {
             const int b = lane - kMaxKc - kMaxStages;
             ptx::mbar_init(bar_tfull + 8 * b, 1);
-            ptx::mbar_init(bar_tempty + 8 * b, 4);
+            ptx::mbar_init(bar_tempty + 8 * b, 4 * p.nb);      // the warps that read the slot
             ptx::mbar_init(bar_cfull + 8 * b, 1);
-            ptx::mbar_init(bar_cempty + 8 * b, 4);
+            ptx::mbar_init(bar_cempty + 8 * b, 4 * p.nb);
         } else if (lane == 31) {
             ptx::mbar_init(bar_drain, 2);
             flags[0] = 0;
@@ -229,7 +236,7 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                 bar = bar_wfull + 8 * st;
                 ptx::mbar_expect_tx(bar, tx);
                 if (++hs[t] == half) { hs[t] = 0; hph[t] ^= 1u; }
-                return smem_base + p.off_w + st * kStageBytes;
+                return smem_base + p.off_w + st * w_stage;
             };
             for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers, aph ^= 1u) {
                 for (int lc0 = 0; lc0 < cols && ok; lc0 += 2) {
@@ -237,11 +244,11 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                     int ct[2];
                     for (int t = 0; t < nu && ok; ++t) {
                         ct[t] = g + (lc0 + t) * p.groups;
-                        const uint32_t slot = (uint32_t)t + 2u * (k[t] & 1u);
-                        if (!tc::wait_bar(bar_cempty + 8 * slot, ((k[t] >> 1) & 1u) ^ 1u, flags)) { ok = false; break; }
-                        ptx::mbar_expect_tx(bar_cfull + 8 * slot, kConstBytes);
-                        ptx::bulk_load(smem_base + p.off_const + slot * kConstBytes, p.consts + (size_t)ct[t] * kConstBytes,
-                                       kConstBytes, bar_cfull + 8 * slot);
+                        const uint32_t slot = slot_of((uint32_t)t, k[t]);
+                        if (!tc::wait_bar(bar_cempty + 8 * slot, phase_of(k[t]) ^ 1u, flags)) { ok = false; break; }
+                        ptx::mbar_expect_tx(bar_cfull + 8 * slot, nb * kConstBytes);
+                        ptx::bulk_load(smem_base + p.off_const + slot * nb * kConstBytes,
+                                       p.consts + (size_t)ct[t] * nb * kConstBytes, nb * kConstBytes, bar_cfull + 8 * slot);
                         ++k[t];
                     }
                     for (int c = 0; c < p.kc && ok; ++c) {
@@ -252,14 +259,14 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                         }
                         for (int t = 0; t < nu && ok; ++t) {
                             uint32_t bar = 0;
-                            const uint32_t dst = w_slot(t, kStageBytes, bar);
-                            if (ok) ptx::tma_load_2d(dst, &wmap, c * kChunk, ct[t] * kNt, bar);
+                            const uint32_t dst = w_slot(t, w_stage, bar);
+                            if (ok) ptx::tma_load_2d(dst, &wmap, c * kChunk, ct[t] * (int)nt, bar);
                         }
                     }
                     for (int t = 0; t < nu && ok; ++t) {
                         uint32_t bar = 0;
-                        const uint32_t dst = w_slot(t, kWbiasBytes, bar);
-                        if (ok) ptx::bulk_load(dst, p.wbias + (size_t)ct[t] * kWbiasBytes, kWbiasBytes, bar);
+                        const uint32_t dst = w_slot(t, nb * kWbiasBytes, bar);
+                        if (ok) ptx::bulk_load(dst, p.wbias + (size_t)ct[t] * nb * kWbiasBytes, nb * kWbiasBytes, bar);
                     }
                 }
             }
@@ -273,19 +280,20 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
         // ---- MMA issuers ------------------------------------------------------------------------------
         if (lane == 0) {
             const uint32_t t = warp == 1 ? 0u : 1u;
-            // s8 x s8 -> s32, both K-major, M = 128, N = 128
-            const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kNt >> 3) << 17) | ((128u >> 4) << 24);
+            // s8 x s8 -> s32, both K-major, M = 128, N = 128 or 256
+            const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((nt >> 3) << 17) | ((128u >> 4) << 24);
             const uint64_t d_128 = tc::smem_desc(0u, 128u), d_32 = tc::smem_desc(0u, 32u);
             const uint64_t ac_desc = d_32 | (uint64_t)((smem_base + p.off_aconst) >> 4);
-            const uint32_t a_lo0 = smem_base >> 4, w_lo0 = (smem_base + p.off_w) >> 4, step = kStageBytes >> 4;
+            const uint32_t a_lo0 = smem_base >> 4, w_lo0 = (smem_base + p.off_w) >> 4;
+            const uint32_t a_step = kStageBytes >> 4, w_step = w_stage >> 4;
             uint32_t hs = 0, hph = 0, k = 0, aph = 0;
             bool ok = true;
             for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers, aph ^= 1u) {
                 for (int lc = (int)t; lc < cols && ok; lc += 2, ++k) {
-                    const uint32_t acc = t + 2u * (k & 1u);
-                    if (!tc::wait_bar(bar_tempty + 8 * acc, ((k >> 1) & 1u) ^ 1u, flags)) { ok = false; break; }
+                    const uint32_t acc = slot_of(t, k);
+                    if (!tc::wait_bar(bar_tempty + 8 * acc, phase_of(k) ^ 1u, flags)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
-                    const uint32_t d_tmem = tmem_base + acc * 128u;
+                    const uint32_t d_tmem = tmem_base + acc * nt;
                     const bool first = lc == (int)t, last = lc + 2 >= cols;     // of this thread in the row tile
                     uint32_t accum = 0;
                     for (int c = 0; c < p.kc; ++c) {
@@ -293,7 +301,7 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                         if (first && !tc::wait_bar(bar_afull + 8 * c, aph, flags)) { ok = false; break; }
                         if (!tc::wait_bar(bar_wfull + 8 * st, hph, flags)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
-                        const uint32_t a_lo = a_lo0 + (uint32_t)c * step, w_lo = w_lo0 + st * step;
+                        const uint32_t a_lo = a_lo0 + (uint32_t)c * a_step, w_lo = w_lo0 + st * w_step;
                         const int nks = c == p.kc - 1 ? p.ksteps_last : 4;
                         for (int ks = 0; ks < nks; ++ks) {
                             ptx::mma_i8(d_tmem, d_128 | (uint64_t)(a_lo + 2 * ks), d_128 | (uint64_t)(w_lo + 2 * ks), idesc, accum);
@@ -308,7 +316,7 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                     const uint32_t st = 2u * hs + t;
                     if (!tc::wait_bar(bar_wfull + 8 * st, hph, flags)) { ok = false; break; }
                     ptx::tc_fence_after_sync();
-                    ptx::mma_i8(d_tmem, ac_desc, d_32 | (uint64_t)(w_lo0 + st * step), idesc, 1u);
+                    ptx::mma_i8(d_tmem, ac_desc, d_32 | (uint64_t)(w_lo0 + st * w_step), idesc, 1u);
                     ptx::mma_commit(bar_wempty + 8 * st);
                     if (++hs == half) { hs = 0; hph ^= 1u; }
                     ptx::mma_commit(bar_tfull + 8 * acc);
@@ -320,14 +328,20 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
         }
     } else {
         // ---- epilogue ---------------------------------------------------------------------------------
-        const int q = warp & 3, grp = (warp - 2) >> 2;          // grp = this group's accumulator
-        const int t = grp & 1;                                  // the issuing thread it follows
+        // Group grp follows issuing thread grp & 1.  With 128-channel tiles it takes that thread's
+        // units with k & 1 == grp >> 1 (slot grp); with 256-channel tiles it takes every unit of the
+        // thread and the half grp >> 1 of its 256 columns.
+        const int q = warp & 3, grp = (warp - 2) >> 2;
+        const int t = grp & 1, h = grp >> 1;
         uint8_t *slab = smem + p.off_out + (size_t)(warp - 2) * kSlabBytes;
         uint8_t *my_row = slab + lane * kEpiCols;
         const uint32_t slab_addr = ptx::smem_u32(slab);
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
-        const uint32_t acc = (uint32_t)grp;
-        const uint8_t *cst = smem + p.off_const + acc * kConstBytes;
+        const uint32_t acc = nb == 1u ? (uint32_t)grp : (uint32_t)t;          // slot: barriers, accumulator
+        const uint32_t blk = nb == 1u ? (uint32_t)grp : 2u * (uint32_t)t + (uint32_t)h;   // 128-column block of constants
+        const uint32_t tcol = blk * 128u;                                       // its accumulator columns
+        const int col_in_tile = nb == 1u ? 0 : h * kNt;
+        const uint8_t *cst = smem + p.off_const + blk * kConstBytes;
         const int *cm = reinterpret_cast<const int *>(cst);
         const int2 *cbs = reinterpret_cast<const int2 *>(cst + kNt * 4);
         const int *hdr = reinterpret_cast<const int *>(cst + kNt * 12);
@@ -336,9 +350,9 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
         for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers) {
             const int row0 = mt * 128 + q * 32;
             for (int lc = t; lc < cols && ok; lc += 2, ++k) {
-                if ((int)(k & 1u) != (grp >> 1)) continue;
-                const int col0 = (g + lc * p.groups) * kNt;
-                const uint32_t ph = (k >> 1) & 1u;
+                if (nb == 1u && (int)(k & 1u) != h) continue;
+                const int col0 = (g + lc * p.groups) * (int)nt + col_in_tile;
+                const uint32_t ph = phase_of(k);
                 if (!tc::wait_bar<true>(bar_cfull + 8 * acc, ph, flags)) { ok = false; break; }
                 if (!tc::wait_bar<true>(bar_tfull + 8 * acc, ph, flags)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
@@ -355,7 +369,7 @@ wide_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant
                     // the previous store has read the slab
                     ptx::bulk_wait_read0();
                     __syncwarp();
-                    const uint32_t taddr = t_lane + acc * 128u + pc * kEpiCols;
+                    const uint32_t taddr = t_lane + tcol + pc * kEpiCols;
                     if (fast) tc::epi_fast_fixed<32>(taddr, cm + pc * kEpiCols, shmax, my_row, rel);
                     else tc::epi_exact_subtile<32>(32, p.act_min, p.act_max, taddr, cm + pc * kEpiCols,
                                                    cbs + pc * kEpiCols, my_row, rel);

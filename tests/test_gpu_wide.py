@@ -38,13 +38,28 @@ SHAPES = [
     (37965, 256, 256),      # two and three row tiles per CTA, ragged end
     (5000, 1024, 128),      # the largest K
     (129, 208, 448),
+    (40000, 512, 640),      # N = 256: two and a half column tiles, the resident rows at their limit
 ]
 
 
+@pytest.fixture(params=[1, 2], ids=["n128", "n256"])
+def blocks(request):
+    """128-channel blocks per column tile: MMAs of N = 128 or N = 256."""
+    binding.debug_tc_wide(2, request.param)
+    yield request.param
+    binding.debug_tc_wide(2, 0)
+
+
 @pytest.mark.parametrize("m,cin,cout", SHAPES)
-def test_matches_oracle(oracle, m, cin, cout):
+def test_matches_oracle(oracle, blocks, m, cin, cout):
     x, lay = make_case(7000 + cin + cout, m, cin, cout, 0.5, act="i8")
     xd, wp, consts = to_device(x, lay)
+    if blocks == 2 and cin > 512:
+        # four 32 KB stages do not fit beside the resident rows
+        with pytest.raises(binding.PromError) as e:
+            binding.pw_conv_i8(xd, wp, cout, binding.make_requant(*consts), variant="tc")
+        assert e.value.code == binding.PROM_ERR_UNSUPPORTED
+        return
     got = run_variant(xd, wp, consts, cout, "tc")
     assert binding.last_device_status() == binding.PROM_OK
     assert first_mismatch(got, oracle_y(oracle, x, lay)) is None, (m, cin, cout)
@@ -64,7 +79,7 @@ def test_same_bytes_as_the_weight_resident_kernel():
 
 
 @pytest.mark.parametrize("lo,hi", [(-128, 127), (-5, 90), (0, 127)])
-def test_clamps_and_wide_shift_spans(oracle, lo, hi):
+def test_clamps_and_wide_shift_spans(oracle, blocks, lo, hi):
     """Shifts 1..20 inside one column tile and a signed clamp: the 64-bit epilogue; the third case
     mixes a tile on the one-multiply form with tiles on the 64-bit form."""
     m, cin, cout = 3000, 256, 384
@@ -76,7 +91,7 @@ def test_clamps_and_wide_shift_spans(oracle, lo, hi):
     assert first_mismatch(got, oracle_y(oracle, x, lay, lo, hi)) is None
 
 
-def test_large_m_sampled_rows(oracle):
+def test_large_m_sampled_rows(oracle, blocks):
     m, cin, cout = 200704, 384, 320
     seed = synth.BASE_SEED + 5
     x = synth.act_uniform_i8(seed, (m, cin), device="cuda")
