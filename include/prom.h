@@ -29,8 +29,12 @@
  *   - Every pointer named *_dev is device memory of the current CUDA device,
  *     owned by the caller; *_host is host memory (pinned for overlap).
  *   - The library allocates nothing the caller must free.  It keeps small
- *     internal caches (tensor-map plans, index lists of the add/sub variant)
- *     that prom_shutdown() releases.
+ *     internal caches (tensor-map plans; per device and stream, the index
+ *     lists of the add/sub variant and the expanded weight matrix of the
+ *     row-resident tensor-core kernel, which single calls with Cin >= 512 and
+ *     Cout >= 256 on many rows use: device memory obtained with cudaMalloc on
+ *     first use, so the first such call on a stream should not be made while
+ *     that stream is being captured) that prom_shutdown() releases.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
  *     Convolution calls are asynchronous on that stream.
  *   - Errors are return codes; nothing aborts or traps.  Argument errors are
