@@ -105,7 +105,8 @@ prom_status prom_debug_i8_mma_rate(int iters, long long *cycles_dev, int cycles_
 prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cycles_dev,
                                 int cycles_len, int *grid_out, void *cuda_stream);
 
-/* Two more probes behind figures that the design doc argues with.
+/* Two more probes: rates that bound kernels made of small MMAs and kernels
+ * that stream an operand out of L2.
  *   mma_issue_rate: how often an SM accepts a tcgen05.mma.kind::i8 of shape
  *     128 x n x 32 (n a multiple of 16, 16..256) when `warps` threads (1..4, one
  *     per warp, each with two accumulators of its own: warps * 2 * max(n, 64)

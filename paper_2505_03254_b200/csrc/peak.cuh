@@ -185,7 +185,7 @@ l2_copy_rate_kernel(const uint8_t *src, unsigned long long region, int iters, in
         const long long t0 = clock64();
         // ring position and phase advance by additions (a division per copy would be what is measured)
         int s = 0;
-        uint32_t ph = 1;                            // parity of the stage's previous use; no wait in round 0
+        uint32_t ph = 1;                            // parity of the stage's previous use; no wait in the first pass over the ring
         const uint32_t bar0 = ptx::smem_u32(&bar[0]), dst0 = ptx::smem_u32(smem);
         for (int it = 0; it < iters + stages && ok; ++it) {
             const uint32_t b = bar0 + 8u * (uint32_t)s;
