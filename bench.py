@@ -239,6 +239,35 @@ def l2_copy_probe(torch, binding, iters=4096, region_mb=8):
     return out
 
 
+def mma_beside_probe(torch, binding, iters=4096):
+    """128 x 128 x 32 MMAs beside bulk copies into the same SM's shared memory, and beside warps that
+    read tensor memory: SM clocks per MMA, bytes per clock of the copies, bytes per clock of the reads."""
+    out = torch.zeros((8 * 1024,), dtype=torch.int64, device="cuda")
+    region = torch.ones((8 << 20,), dtype=torch.uint8, device="cuda")
+    rows = {"beside_copies": [], "beside_reads": []}
+    for stages in (0, 1, 2, 3):
+        binding.debug_mma_beside(0, 64, 0, stages, region, out)
+        grid = binding.debug_mma_beside(0, iters, 0, stages, region, out)
+        torch.cuda.synchronize()
+        o = out[:8 * grid].view(grid, 8)
+        cyc = int(o[:, 0].max().item())
+        rows["beside_copies"].append({"copies_in_flight": stages, "cycles_per_mma": round(cyc / (4.0 * iters), 1),
+                                      "copy_bytes_per_clk_per_sm": round(float(o[:, 3].double().mean().item()) * 16384 / cyc, 1)})
+    for nwarps in (4, 8, 16):
+        for mma in (0, 1):
+            binding.debug_mma_beside(1, 64, nwarps, mma, None, out)
+            grid = binding.debug_mma_beside(1, iters, nwarps, mma, None, out)
+            torch.cuda.synchronize()
+            o = out[:8 * grid].view(grid, 8)
+            cyc = int(o[:, 0].max().item())
+            n_mma = o[:, 1].double()
+            c_mma = o[:, 2].double()
+            rows["beside_reads"].append({"reading_warps": nwarps, "mmas": bool(mma),
+                                         "read_bytes_per_clk_per_sm": round(iters * nwarps * 4096.0 / cyc, 1),
+                                         "cycles_per_mma": round(float((c_mma / n_mma.clamp(min=1)).max().item()), 1) if mma else None})
+    return rows
+
+
 def build_network(seed, synth, binding=None, device=None, width=1.0):
     """Layer table plus per-layer weights/constants: host arrays for the oracle,
     and (when a binding is given) packed device tensors for the library."""
@@ -1094,6 +1123,8 @@ def run_aux(args):
         out = alu_rate_probe(torch, binding)
     elif args.aux == "write_bw":
         out = write_bandwidth_probe(torch)
+    elif args.aux == "mma_beside":
+        out = mma_beside_probe(torch, binding)
     elif args.aux == "mma_issue":
         out = mma_issue_probe(torch, binding)
     elif args.aux == "l2_copy":
@@ -1125,7 +1156,7 @@ def main():
     ap.add_argument("--no-detail", action="store_true", help="skip per-layer and single-layer timing")
     ap.add_argument("--sweep", default=None, help="write the single-layer sweep to this file")
     ap.add_argument("--single", default=None, help="M,K,N[,variant[,zero_frac]]: time one layer")
-    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate", "depth_first", "mma_issue", "l2_copy", "write_bw"],
+    ap.add_argument("--aux", default=None, choices=["act_quantizer", "dynamic_layer", "depthwise", "body", "i8_peak", "alu_rate", "depth_first", "mma_issue", "l2_copy", "write_bw", "mma_beside"],
                     help="run one of the legs that are off the timed step, alone")
     ap.add_argument("--widths", default=None, help="comma-separated width multipliers: time the sequence at each")
     ap.add_argument("--sweep-small", action="store_true", help="sweep without the largest M")

@@ -123,6 +123,23 @@ prom_status prom_debug_mma_issue_rate(int n, int warps, int iters, long long *cy
 prom_status prom_debug_l2_copy_rate(const void *region_dev, uint64_t region_bytes, int iters, int stages,
                                     long long *cycles_dev, int cycles_len, int *grid_out, void *cuda_stream);
 
+/* What shares an SM with the MMAs, one CTA per SM.
+ *   mode 0: one thread issues iters x 4 tcgen05.mma.kind::i8 of shape
+ *     128 x 128 x 32 while a second thread keeps `stages` (0 = none, 1..3) bulk
+ *     copies of 16 KB in flight out of region_dev (as for l2_copy_rate) into
+ *     other shared memory, until the MMAs are done.
+ *   mode 1: nwarps (4, 8 or 16) warps each read iters times 32 lanes x 32
+ *     columns of tensor memory (tcgen05.ld 32x32b.x32, wait, fold) while, if
+ *     stages == 1, another thread issues the same MMAs into other columns until
+ *     the readers are done (stages == 0: no MMAs).
+ * out_dev[8 * cta + i], out_len >= 8 x the grid size: i = 0 SM clocks of the
+ * measured loop (mode 1: of the slowest reading warp), 1 = MMAs issued,
+ * 2 = SM clocks of the MMA loop, 3 = copies issued.  Asynchronous on the
+ * stream; all waits bounded. */
+prom_status prom_debug_mma_beside(int mode, int iters, int nwarps, int stages, const void *region_dev,
+                                  uint64_t region_bytes, long long *out_dev, int out_len, int *grid_out,
+                                  void *cuda_stream);
+
 /* Bookkeeping check, no CUDA call: returns 1 the first time (device, key) is
  * asked about on the table used for per-device kernel attributes, 0
  * afterwards (the table behind this entry is a separate instance). */

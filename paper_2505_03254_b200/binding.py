@@ -33,6 +33,7 @@ EXPORTS = [
     "prom_debug_once_per_device", "prom_debug_layer_seq_output_offset",
     "prom_pw_prepared_bytes", "prom_pw_prepare", "prom_pw_conv_i8_prepared", "prom_quantize_ternary_batch",
     "prom_debug_dw_variant", "prom_debug_tc_wide", "prom_debug_mma_issue_rate", "prom_debug_l2_copy_rate",
+    "prom_debug_mma_beside",
 ]
 STATIC_SCRATCH_BYTES = 6 << 20
 
@@ -136,6 +137,8 @@ def lib():
         L.prom_debug_mma_issue_rate.argtypes = [i32, i32, i32, vp, i32, C.POINTER(C.c_int), vp]
         L.prom_debug_l2_copy_rate.restype = i32
         L.prom_debug_l2_copy_rate.argtypes = [vp, C.c_uint64, i32, i32, vp, i32, C.POINTER(C.c_int), vp]
+        L.prom_debug_mma_beside.restype = i32
+        L.prom_debug_mma_beside.argtypes = [i32, i32, i32, i32, vp, C.c_uint64, vp, i32, C.POINTER(C.c_int), vp]
         L.prom_debug_once_per_device.restype = i32
         L.prom_debug_once_per_device.argtypes = [i32, i32]
         L.prom_quantize_ternary_batch.restype = i32
@@ -339,6 +342,18 @@ def debug_l2_copy_rate(region: torch.Tensor, iters: int, stages: int, cycles: to
     _check(lib().prom_debug_l2_copy_rate(_dev(region, torch.uint8, "region"), region.numel(), int(iters),
                                          int(stages), _dev(cycles, torch.int64, "cycles"), cycles.numel(),
                                          C.byref(grid), _stream(stream)), "prom_debug_l2_copy_rate")
+    return int(grid.value)
+
+
+def debug_mma_beside(mode: int, iters: int, nwarps: int, stages: int, region, out: torch.Tensor, stream=None) -> int:
+    """prom_debug_mma_beside: MMAs beside bulk copies (mode 0) or beside tensor-memory reads (mode 1);
+    out[8 * cta + i] as in the header.  Returns the grid size."""
+    grid = C.c_int(0)
+    rp = _dev(region, torch.uint8, "region") if region is not None else None
+    rb = region.numel() if region is not None else 0
+    _check(lib().prom_debug_mma_beside(int(mode), int(iters), int(nwarps), int(stages), rp, rb,
+                                       _dev(out, torch.int64, "out"), out.numel(), C.byref(grid), _stream(stream)),
+           "prom_debug_mma_beside")
     return int(grid.value)
 
 

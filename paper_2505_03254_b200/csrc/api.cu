@@ -1873,6 +1873,42 @@ prom_status prom_debug_l2_copy_rate(const void *region_dev, uint64_t region_byte
     return cuda_status(cudaGetLastError());
 }
 
+prom_status prom_debug_mma_beside(int mode, int iters, int nwarps, int stages, const void *region_dev,
+                                  uint64_t region_bytes, long long *out_dev, int out_len, int *grid_out,
+                                  void *cuda_stream)
+{
+    if (!out_dev || !grid_out) return PROM_ERR_NULL;
+    if ((mode != 0 && mode != 1) || iters < 1 || iters > (1 << 20)) return PROM_ERR_SHAPE;
+    if (mode == 0) {
+        if (stages < 0 || stages > 3) return PROM_ERR_SHAPE;
+        if (stages > 0) {
+            if (!region_dev) return PROM_ERR_NULL;
+            if (!aligned16(region_dev)) return PROM_ERR_ALIGN;
+            if (region_bytes < peak::kCopyBytes || region_bytes % peak::kCopyBytes) return PROM_ERR_SHAPE;
+        }
+    } else if ((nwarps != 4 && nwarps != 8 && nwarps != 16) || (stages != 0 && stages != 1)) {
+        return PROM_ERR_SHAPE;
+    }
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    if (out_len < 8 * d.sms) return PROM_ERR_WORKSPACE;
+    *grid_out = d.sms;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(out_dev, 0, sizeof(long long) * 8 * (size_t)d.sms, st) != cudaSuccess) return PROM_ERR_CUDA;
+    const uint8_t *src = static_cast<const uint8_t *>(region_dev);
+    if (mode == 0) {
+        if (raise_smem_limit(peak::beside_mma_kernel<0>, peak::kBesideSmem) != cudaSuccess) return PROM_ERR_CUDA;
+        peak::beside_mma_kernel<0><<<d.sms, peak::kBesideThreads, peak::kBesideSmem, st>>>(
+            iters, 0, stages, src, (unsigned long long)region_bytes, out_dev);
+    } else {
+        if (raise_smem_limit(peak::beside_mma_kernel<1>, peak::kBesideSmem) != cudaSuccess) return PROM_ERR_CUDA;
+        peak::beside_mma_kernel<1><<<d.sms, peak::kBesideThreads, peak::kBesideSmem, st>>>(
+            iters, nwarps, stages, src, (unsigned long long)region_bytes, out_dev);
+    }
+    ++g_launches;
+    return cuda_status(cudaGetLastError());
+}
+
 void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode ? 1 : 0); }
 
 void prom_debug_dw_variant(int variant) { g_dw_variant.store(variant < 0 || variant > 2 ? 0 : variant); }

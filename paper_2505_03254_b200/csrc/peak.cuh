@@ -210,4 +210,126 @@ l2_copy_rate_kernel(const uint8_t *src, unsigned long long region, int iters, in
     }
 }
 
+// Two things that share an SM with the MMAs.
+// MODE 0: warp 0 issues `iters` rounds of four 128 x 128 x 32 MMAs (fixed operands, accumulator
+// columns 384..511) while lane 0 of warp 1 keeps `stages` (0 = no copies, else 1..3) bulk copies
+// of 16 KB in flight from `src` into a ring of its own until the MMAs are done.
+// MODE 1: warps 0..nwarps-1 (4, 8 or 16) each read `iters` times 32 lanes x 32 columns out of the
+// accumulator columns 0..383 with tcgen05.ld 32x32b.x32, wait and fold the registers, while (if
+// `stages` != 0) lane 0 of warp 16 issues MMAs into columns 384..511 until the readers are done.
+// out[8 * cta + 0] = SM clocks of the measured loop (the slowest reader in mode 1), [1] = MMAs
+// issued, [2] = SM clocks of the MMA loop, [3] = copies issued.  All loops and waits are bounded.
+constexpr int kBesideThreads = 32 * 17;
+constexpr uint32_t kBesideOperands = (kMmaM + 128) * kMmaRowBytes;            // A and B: 32 KB
+constexpr int kBesideSmem = (int)kBesideOperands + 3 * (int)kCopyBytes + 1024 + 64;
+template <int MODE>
+__global__ void __launch_bounds__(kBesideThreads, 1)
+beside_mma_kernel(int iters, int nwarps, int stages, const uint8_t *src, unsigned long long region, long long *out)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
+    __shared__ uint64_t bar_mma, bar_ld[3];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int done;                                   // readers (mode 1) or the MMA thread (mode 0) finished
+    __shared__ long long reader_max;
+    for (int i = threadIdx.x; i < (int)kBesideOperands / 4; i += kBesideThreads)
+        reinterpret_cast<uint32_t *>(smem)[i] = 0x01010101u * (uint32_t)(i & 3);
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_u32(&bar_mma), 1);
+        for (int i = 0; i < 3; ++i) ptx::mbar_init(ptx::smem_u32(&bar_ld[i]), 1);
+        ptx::mbar_init_fence();
+        done = 0;
+        reader_max = 0;
+    }
+    if (threadIdx.x < 32) ptx::tmem_alloc(ptx::smem_u32(&tmem_slot), 512u);
+    ptx::fence_proxy_async_smem();
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *vdone = &done;
+    const int mma_warp = MODE == 0 ? 0 : 16;
+    if (warp == mma_warp && lane == 0 && (MODE == 0 || stages != 0)) {
+        const uint32_t a_addr = ptx::smem_u32(smem), b_addr = a_addr + kMmaM * kMmaRowBytes;
+        const uint64_t hi = (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+        const uint64_t a0 = hi | (uint64_t)((a_addr >> 4) & 0x3FFFu), b0 = hi | (uint64_t)((b_addr >> 4) & 0x3FFFu);
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+        const int rounds = MODE == 0 ? iters : (1 << 22);  // mode 1: until the readers are done
+        long long n = 0;
+        const long long t0 = clock64();
+        for (int it = 0; it < rounds && (MODE == 0 || *vdone < nwarps); ++it) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) ptx::mma_i8(tmem + 384u, a0 + 2 * ks, b0 + 2 * ks, idesc, 1u);
+            n += 4;
+        }
+        const long long t1 = clock64();
+        ptx::mma_commit(ptx::smem_u32(&bar_mma));
+        const unsigned long long g0 = ptx::globaltimer();
+        bool ok = false;
+        while (!(ok = ptx::mbar_try_wait(ptx::smem_u32(&bar_mma), 0u)) && ptx::globaltimer() - g0 < kDrainLimitNs) {}
+        if (!ok) raise_status(PROM_ERR_TIMEOUT);
+        out[8 * blockIdx.x + 1] = n;
+        out[8 * blockIdx.x + 2] = t1 - t0;
+        if (MODE == 0) {
+            out[8 * blockIdx.x + 0] = clock64() - t0;
+            *vdone = 1;
+        }
+    } else if (MODE == 0 && warp == 1 && lane == 0 && stages != 0) {
+        const uint32_t ring = ptx::smem_u32(smem) + kBesideOperands;
+        const unsigned long long nchunks = region / kCopyBytes;
+        unsigned long long c = ((unsigned long long)blockIdx.x * 7ull) % nchunks;
+        long long copies = 0;
+        int s = 0;
+        uint32_t ph = 1;
+        bool ok = true;
+        for (int it = 0; it < (1 << 22) && ok && !*vdone; ++it) {
+            const uint32_t b = ptx::smem_u32(&bar_ld[s]);
+            if (it >= stages) {
+                const unsigned long long g0 = ptx::globaltimer();
+                while (!ptx::mbar_try_wait(b, ph))
+                    if (ptx::globaltimer() - g0 > kDrainLimitNs) { ok = false; break; }
+            }
+            if (!ok) break;
+            ptx::mbar_expect_tx(b, kCopyBytes);
+            ptx::bulk_load(ring + (uint32_t)s * kCopyBytes, src + c * kCopyBytes, kCopyBytes, b);
+            if (++c == nchunks) c = 0;
+            ++copies;
+            if (++s == stages) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) raise_status(PROM_ERR_TIMEOUT);
+        const unsigned long long g0 = ptx::globaltimer();        // let what is in flight land
+        while (ptx::globaltimer() - g0 < 100000ull) {}
+        out[8 * blockIdx.x + 3] = copies;
+    } else if (MODE == 1 && warp < nwarps) {
+        // a warp reads its own lane quarter; the warps of a quarter start 96 columns apart
+        const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        uint32_t acc = 0, col = (uint32_t)(warp >> 2) * 96u;
+        const long long t0 = clock64();
+        for (int it = 0; it < iters; ++it) {
+            uint32_t v[32];
+            ptx::tmem_ld_x32(t_lane + col, v);             // columns col .. col + 31 <= 383
+            ptx::tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) acc ^= v[j];
+            col += 32u;
+            if (col > 352u) col = 0u;
+        }
+        const long long t1 = clock64();
+        if (acc == 0x12345678u) out[8 * blockIdx.x + 7] = 1;                   // keeps the loads alive
+        if (lane == 0) {
+            atomicMax(reinterpret_cast<unsigned long long *>(&reader_max), (unsigned long long)(t1 - t0));
+            __threadfence_block();
+            atomicAdd(&done, 1);
+        }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (MODE == 1 && threadIdx.x == 0) out[8 * blockIdx.x + 0] = reader_max;
+    if (threadIdx.x < 32) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem, 512u);
+    }
+}
+
 }}  // namespace prom::peak
