@@ -329,7 +329,10 @@ static bool tc_search_plan(long long m, int cin, int cout, const RowMap &map, co
     const TcTune tn = tune_for(m, cin, cout, map.stride);
     int fold = 1;
     if (map.stride == 1) {
-        if ((cin & 15) || ((cout & 15) && m % 2 == 0)) fold = 2;
+        // Rows that are not 16-byte multiples cannot be described to TMA: two rows are folded into
+        // one.  On the output side that is only needed when the row does not fit one subtile
+        // (a slab of 32 whole rows is then one contiguous, 16-byte aligned range of Y anyway).
+        if ((cin & 15) || ((cout & 15) && cout > 256 && m % 2 == 0)) fold = 2;
         if (m % fold) return false;
         while (fold * 2 <= 8 && fold * 2 * cin <= 128 && fold * 2 * cout <= 128 &&
                m % (fold * 2) == 0)

@@ -683,15 +683,14 @@ __device__ __forceinline__ void build_image(const Params &p, const int g, const 
                             val.w = tb[w >> 24];
                         }
                     } else {
-                        // cin is 8 modulo 16: a piece may straddle two diagonal blocks
+                        // cin is 8 modulo 16: a piece may straddle two diagonal blocks; the part of
+                        // it that lies in this channel's block pn is the K range [pn k0, (pn + 1) k0)
                         const uint32_t mag = t == 0 ? 1u : (2u << t), neg = 256u - mag;
                         uint32_t wd[4] = {0, 0, 0, 0};
-                        for (int e = 0; e < 16; ++e) {
-                            const int kk = kbase + e;
-                            if (kk >= p.kf) break;
-                            const int pke = kk / p.k0, k = kk - pke * p.k0;
-                            if (pke != pn) continue;
-                            int wv = weight_at(wq, rowb, row, k);
+                        const int k_lo = pn * p.k0, k_hi = min(k_lo + p.k0, p.kf);
+                        const int e_lo = max(0, k_lo - kbase), e_hi = min(16, k_hi - kbase);
+                        for (int e = e_lo; e < e_hi; ++e) {
+                            int wv = weight_at(wq, rowb, row, kbase + e - k_lo);
                             if (wv == -2) { invalid = 1; wv = 0; }
                             const uint32_t byte = wv == 0 ? 0u : (wv > 0 ? mag : neg);
                             wd[e >> 2] |= byte << (8 * (e & 3));
