@@ -51,7 +51,7 @@ void prom_debug_seq_chain(int mode);
 
 /* Which kernel prom_dw_conv3x3_i8 runs: 0 = the library's choice (default: TMA
  * patches and tensor-core taps for stride 1 with a channel count that is a
- * multiple of 16, CUDA cores otherwise), 1 = CUDA cores only, 2 = tensor cores
+ * multiple of 16 and images of at least 100 pixels, CUDA cores otherwise), 1 = CUDA cores only, 2 = tensor cores
  * or PROM_ERR_UNSUPPORTED.  Results do not depend on it.  Process-wide. */
 void prom_debug_dw_variant(int variant);
 

@@ -929,15 +929,32 @@ static void seq_layout(const prom_layer *layers, int n, const SeqShape &s, const
         }
 }
 
-extern "C" prom_status prom_dw_conv3x3_i8(const int8_t *, int, int, int, int, int, const int8_t *,
-                                          const prom_requant *, int8_t *, void *);
 
 // ---- depthwise 3x3 on the tensor cores (dwtc.cuh) ---------------------------------------------
 // 0: the library's choice, 1: CUDA cores only, 2: tensor cores or PROM_ERR_UNSUPPORTED
 static std::atomic<int> g_dw_variant{0};
 
+// Launch configuration of a kernel that may be chained to its predecessor in the stream with
+// programmatic dependent launch (attr must outlive the launch call).
+static void fill_launch_cfg(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int grid, int threads, size_t smem,
+                            cudaStream_t st, bool pdl)
+{
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    if (pdl) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+}
+
 static prom_status launch_dw_tc(const int8_t *x, int batch, int h, int w, int c, const int8_t *wt,
-                                const prom_requant *rq, int8_t *y, const DeviceInfo &d, cudaStream_t st)
+                                const prom_requant *rq, int8_t *y, const DeviceInfo &d, cudaStream_t st,
+                                bool pdl, bool pdl_next)
 {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return PROM_ERR_UNSUPPORTED;
@@ -969,9 +986,73 @@ static prom_status launch_dw_tc(const int8_t *x, int batch, int h, int w, int c,
     if (workers < 1) workers = 1;
     if (workers > p.tiles) workers = p.tiles;
     const int grid = (int)(workers * p.groups);
-    dwtc::dw3x3_tc_kernel<<<grid, dwtc::kThreads, dwtc::kSmemBytes, st>>>(map, p);
+    p.pdl = pdl ? 1 : 0;
+    p.pdl_next = pdl_next ? 1 : 0;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fill_launch_cfg(cfg, attr, grid, dwtc::kThreads, dwtc::kSmemBytes, st, pdl);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, dwtc::dw3x3_tc_kernel, map, p);
     ++g_launches;
-    return cuda_status(cudaGetLastError());
+    return cuda_status(e);
+}
+
+// pdl / pdl_next: the call is a link of a layer sequence (programmatic dependent launch behind the
+// kernel that writes x; the next kernel of the stream is launched that way)
+static prom_status dw_conv3x3(const int8_t *x_dev, int batch, int h, int w, int c, int stride,
+                              const int8_t *w_dev, const prom_requant *rq, int8_t *y_dev, void *cuda_stream,
+                              bool pdl, bool pdl_next)
+{
+    if (batch < 0 || h < 1 || w < 1 || c < 1 || c > 4096 || (stride != 1 && stride != 2)) return PROM_ERR_SHAPE;
+    if (c & 3) return PROM_ERR_UNSUPPORTED;
+    if (!rq) return PROM_ERR_NULL;
+    prom_status e = check_requant(rq);
+    if (e != PROM_OK) return e;
+    if (batch == 0) return PROM_OK;
+    if (!x_dev || !w_dev || !y_dev) return PROM_ERR_NULL;
+    if (!aligned16(x_dev) || !aligned16(y_dev)) return PROM_ERR_ALIGN;
+    if (reinterpret_cast<const void *>(x_dev) == reinterpret_cast<const void *>(y_dev)) return PROM_ERR_ALIGN;
+    const int ho = (h - 1) / stride + 1, wo = (w - 1) / stride + 1;
+    if ((long long)batch * h * w * c >= (1ll << 40)) return PROM_ERR_SHAPE;
+    DeviceInfo d = device_info();
+    if (!d.ok) return PROM_ERR_CUDA;
+    // stride 1 and whole slices of 16 channels: TMA patches and tensor-core taps
+    const int dw_variant = g_dw_variant.load();
+    // (left to itself the library keeps images of fewer than 100 pixels on the CUDA cores: a 7 x 7
+    // image fills 49 of a tile's 128 rows, and [128,7,7,960] takes 18.6 us there against 14.8 us)
+    if (dw_variant != 1 && stride == 1 && (c & 15) == 0 &&
+        !(dw_variant == 0 && ((long long)batch * h * w < 128 || h * w < 100))) {
+        const prom_status e = launch_dw_tc(x_dev, batch, h, w, c, w_dev, rq, y_dev, d,
+                                           static_cast<cudaStream_t>(cuda_stream), pdl, pdl_next);
+        if (e != PROM_ERR_UNSUPPORTED) return e;
+    }
+    if (dw_variant == 2) return PROM_ERR_UNSUPPORTED;
+    const int rows = dw::rows_per_unit(stride);
+    const long long units = (long long)batch * ((ho + rows - 1) / rows) * ((wo + dw::kStrip - 1) / dw::kStrip);
+    if (units >= (1ll << 31)) return PROM_ERR_SHAPE;
+    const long long total = units * (c >> 2);
+    // a multiple of c / 4 threads, so that a thread keeps its channels: blocks in multiples of
+    // (c / 4) / gcd(c / 4, threads per block)
+    int step = c >> 2;
+    for (int a = step, b = dw::kThreads; b;) { const int r = a % b; a = b; b = r; if (!b) step = (c >> 2) / a; }
+    long long blocks = (total + dw::kThreads - 1) / dw::kThreads;
+    const long long cap = (long long)d.sms * 16;
+    if (blocks > cap) blocks = cap;
+    blocks = (blocks + step - 1) / step * step;
+    const int grid = (int)blocks;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fill_launch_cfg(cfg, attr, grid, dw::kThreads, 0, st, pdl);
+    const int f_pdl = pdl ? 1 : 0, f_next = pdl_next ? 1 : 0;
+    cudaError_t le;
+    if (stride == 1)
+        le = cudaLaunchKernelEx(&cfg, dw::dw3x3_kernel<1>, x_dev, batch, h, w, c, ho, wo, w_dev, rq->bias, rq->mult,
+                                rq->shift, rq->act_min, rq->act_max, y_dev, f_pdl, f_next);
+    else
+        le = cudaLaunchKernelEx(&cfg, dw::dw3x3_kernel<2>, x_dev, batch, h, w, c, ho, wo, w_dev, rq->bias, rq->mult,
+                                rq->shift, rq->act_min, rq->act_max, y_dev, f_pdl, f_next);
+    ++g_launches;
+    return cuda_status(le);
 }
 
 // One launch of tc_chain_kernel for layers [c.first, c.last]; conv[] holds every layer's pointers.
@@ -1162,8 +1243,10 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
         if (layers[i].dw_w && s.m[i] > 0) {
             const int stride = layers[i].in_stride;
             const int8_t *src = i == 0 ? x0 : conv[i - 1].y;
-            prom_status de = prom_dw_conv3x3_i8(src, batch, s.h[i] * stride, s.w[i] * stride, layers[i].cin,
-                                                stride, layers[i].dw_w, &layers[i].dw_rq, dw_buf, st);
+            // chained like the pointwise kernels: behind layer i-1's kernel (which releases its
+            // dependents at entry) and in front of layer i's, which waits for it before its loads
+            prom_status de = dw_conv3x3(src, batch, s.h[i] * stride, s.w[i] * stride, layers[i].cin, stride,
+                                        layers[i].dw_w, &layers[i].dw_rq, dw_buf, st, i > 0, true);
             if (de != PROM_OK) return de;
         }
         prom_status e = is_tc[i] ? tc_launch_planned(conv[i], plan[i]) : run_conv(conv[i], variant);
@@ -1296,49 +1379,7 @@ prom_status prom_dw_conv3x3_i8(const int8_t *x_dev, int batch, int h, int w, int
                                const int8_t *w_dev, const prom_requant *rq, int8_t *y_dev,
                                void *cuda_stream)
 {
-    if (batch < 0 || h < 1 || w < 1 || c < 1 || c > 4096 || (stride != 1 && stride != 2)) return PROM_ERR_SHAPE;
-    if (c & 3) return PROM_ERR_UNSUPPORTED;
-    if (!rq) return PROM_ERR_NULL;
-    prom_status e = check_requant(rq);
-    if (e != PROM_OK) return e;
-    if (batch == 0) return PROM_OK;
-    if (!x_dev || !w_dev || !y_dev) return PROM_ERR_NULL;
-    if (!aligned16(x_dev) || !aligned16(y_dev)) return PROM_ERR_ALIGN;
-    if (reinterpret_cast<const void *>(x_dev) == reinterpret_cast<const void *>(y_dev)) return PROM_ERR_ALIGN;
-    const int ho = (h - 1) / stride + 1, wo = (w - 1) / stride + 1;
-    if ((long long)batch * h * w * c >= (1ll << 40)) return PROM_ERR_SHAPE;
-    DeviceInfo d = device_info();
-    if (!d.ok) return PROM_ERR_CUDA;
-    // stride 1 and whole slices of 16 channels: TMA patches and tensor-core taps
-    const int dw_variant = g_dw_variant.load();
-    if (dw_variant != 1 && stride == 1 && (c & 15) == 0 && !(dw_variant == 0 && (long long)batch * h * w < 128)) {
-        const prom_status e = launch_dw_tc(x_dev, batch, h, w, c, w_dev, rq, y_dev, d,
-                                           static_cast<cudaStream_t>(cuda_stream));
-        if (e != PROM_ERR_UNSUPPORTED) return e;
-    }
-    if (dw_variant == 2) return PROM_ERR_UNSUPPORTED;
-    const int rows = dw::rows_per_unit(stride);
-    const long long units = (long long)batch * ((ho + rows - 1) / rows) * ((wo + dw::kStrip - 1) / dw::kStrip);
-    if (units >= (1ll << 31)) return PROM_ERR_SHAPE;
-    const long long total = units * (c >> 2);
-    // a multiple of c / 4 threads, so that a thread keeps its channels: blocks in multiples of
-    // (c / 4) / gcd(c / 4, threads per block)
-    int step = c >> 2;
-    for (int a = step, b = dw::kThreads; b;) { const int r = a % b; a = b; b = r; if (!b) step = (c >> 2) / a; }
-    long long blocks = (total + dw::kThreads - 1) / dw::kThreads;
-    const long long cap = (long long)d.sms * 16;
-    if (blocks > cap) blocks = cap;
-    blocks = (blocks + step - 1) / step * step;
-    const int grid = (int)blocks;
-    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    if (stride == 1)
-        dw::dw3x3_kernel<1><<<grid, dw::kThreads, 0, st>>>(x_dev, batch, h, w, c, ho, wo, w_dev, rq->bias,
-                                                           rq->mult, rq->shift, rq->act_min, rq->act_max, y_dev);
-    else
-        dw::dw3x3_kernel<2><<<grid, dw::kThreads, 0, st>>>(x_dev, batch, h, w, c, ho, wo, w_dev, rq->bias,
-                                                           rq->mult, rq->shift, rq->act_min, rq->act_max, y_dev);
-    ++g_launches;
-    return cuda_status(cudaGetLastError());
+    return dw_conv3x3(x_dev, batch, h, w, c, stride, w_dev, rq, y_dev, cuda_stream, false, false);
 }
 
 prom_status prom_pw_conv_i8_dyn(const int8_t *x_dev, int batch, int64_t rows_per_sample, int cin,

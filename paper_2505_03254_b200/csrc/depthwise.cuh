@@ -15,6 +15,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace prom { namespace dw {
 
@@ -48,8 +49,11 @@ __global__ void __launch_bounds__(kThreads, 3)
 dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int ho, int wo,
              const int8_t *__restrict__ wt, const int32_t *__restrict__ bias,
              const int32_t *__restrict__ mult, const int8_t *__restrict__ shift, int lo, int hi,
-             int8_t *__restrict__ y)
+             int8_t *__restrict__ y, int pdl, int pdl_next)
 {
+    // pdl: launched with programmatic dependent launch behind the kernel that writes x;
+    // pdl_next: the next kernel of the stream is launched that way and may start its prologue now
+    if (pdl_next) ptx::grid_dep_launch();
     constexpr int kRows = rows_per_unit(STRIDE);          // output rows of a unit
     constexpr int kRowsIn = STRIDE * (kRows - 1) + 3;     // input rows under them (3 or 4)
     constexpr int kCols = STRIDE * (kStrip - 1) + 3;      // input columns under a strip
@@ -84,6 +88,9 @@ dw3x3_kernel(const int8_t *__restrict__ x, int batch, int h, int w, int c, int h
 #pragma unroll
     for (int k = 0; k < 4; ++k) cb4[k] = cb[k] * 4;
 
+    // filters and constants are nobody's output; x is the previous kernel's (every thread waits, so
+    // that a grid without work still ends after its predecessor)
+    if (pdl) ptx::grid_dep_wait();
     const size_t pix = (size_t)c;                         // bytes from a pixel to the next
     // 32-bit unit indices (the host keeps the number of units below 2^31)
     const unsigned ustep = (unsigned)(nthreads / cw);

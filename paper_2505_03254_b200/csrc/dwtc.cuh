@@ -49,6 +49,8 @@ struct Params {
     const int8_t *shift;
     int lo, hi;
     int8_t *y;
+    int pdl;                // launched with programmatic dependent launch behind the kernel that writes x
+    int pdl_next;           // the next kernel of the stream is launched that way
 };
 
 // Unswizzled K-major operand: core matrices of 8 rows x 16 bytes; `k_off` bytes from a core
@@ -81,7 +83,9 @@ __global__ void __launch_bounds__(kThreads, 2) dw3x3_tc_kernel(const __grid_cons
     const int ch0 = g * p.ns * 16;                        // its first channel
     const int nch = p.ns * 16;
 
-    // ---- prologue ---------------------------------------------------------------------------
+    if (p.pdl_next) ptx::grid_dep_launch();
+
+    // ---- prologue (nothing here reads the previous kernel's output) -------------------------
     if (warp == 0) {
         if (lane < kStages) {
             ptx::mbar_init(bar_full + 8 * lane, 1);
@@ -133,6 +137,7 @@ __global__ void __launch_bounds__(kThreads, 2) dw3x3_tc_kernel(const __grid_cons
         if (lane == 0) {
             uint32_t slot = 0, ph = 0, issued = 0;
             bool ok = true;
+            if (p.pdl) ptx::grid_dep_wait();      // the loads are the only reads of x
             for (long long t = worker; t < p.tiles && ok; t += nworkers) {
                 const int b = (int)(t / tiles_img), r = (int)(t - (long long)b * tiles_img);
                 const int ty = r / p.tiles_x, tx = r - ty * p.tiles_x;
@@ -239,6 +244,8 @@ __global__ void __launch_bounds__(kThreads, 2) dw3x3_tc_kernel(const __grid_cons
     }
 
     // ---- teardown -------------------------------------------------------------------------------
+    // every CTA waits for the previous kernel before it ends, also one whose loader had no tile
+    if (p.pdl && threadIdx.x == 32) ptx::grid_dep_wait();
     ptx::tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
