@@ -1019,7 +1019,8 @@ def run_sweep(args):
 
 
 def run_single(args):
-    """One single layer M,K,N[,variant[,zero_frac]] launched a few times (for profiler captures)."""
+    """One single layer M,K,N[,variant[,zero_frac]] launched a few times (for profiler captures);
+    variant tc_prepared times prom_pw_conv_i8_prepared on operands prepared once."""
     import torch
     from paper_2505_03254_b200 import binding, build, synth
     torch.cuda.set_device(0)
@@ -1038,7 +1039,11 @@ def run_single(args):
     rq = binding.make_requant(lay["bias"], lay["mult"], lay["shift"])
     y = torch.empty((m, cout), dtype=torch.int8, device="cuda")
     flush = torch.empty((FLUSH_BYTES,), dtype=torch.uint8, device="cuda")
-    fn = lambda: binding.pw_conv_i8(x, wp, cout, rq, y=y, variant=variant)
+    if variant == "tc_prepared":
+        prep = binding.pw_prepare(m, cin, wp, cout, rq)
+        fn = lambda: binding.pw_conv_i8_prepared(x, cout, prep, y=y)
+    else:
+        fn = lambda: binding.pw_conv_i8(x, wp, cout, rq, y=y, variant=variant)
     med, mn = cold_time_us(torch, fn, flush, iters=max(1, args.steps), warm=max(1, args.warmup))
     b, o = layer_bytes(m, cin, cout), layer_ops(m, cin, cout)
     roof = max(b / bw, o / p_i8) * 1e6
