@@ -386,18 +386,30 @@ def quantize_ternary(w: torch.Tensor, want_alpha: bool = True, stream=None):
     return packed, alpha
 
 
-def quantize_ternary_batch(ws: Sequence[torch.Tensor], out=None, stream=None):
+class QuantizeJobs:
+    """The job table of prom_quantize_ternary_batch for a list of device float32 [cout, cin] matrices,
+    marshalled once (it holds raw pointers: the tensors are kept alive with it)."""
+
+    def __init__(self, ws: Sequence[torch.Tensor], out=None):
+        if out is None:
+            out = [(torch.empty((w.shape[0], (w.shape[1] + 3) // 4), dtype=torch.uint8, device=w.device),
+                    torch.empty((w.shape[0],), dtype=torch.float32, device=w.device)) for w in ws]
+        self.ws, self.out, self.n = list(ws), out, len(ws)
+        self.array = (PromQuantizeJob * self.n)()
+        for j, (w, (packed, alpha)) in enumerate(zip(ws, out)):
+            self.array[j] = PromQuantizeJob(_dev(w, torch.float32, "w"), w.shape[0], w.shape[1], packed.data_ptr(),
+                                            packed.numel(), alpha.data_ptr())
+
+
+def quantize_ternary_batch(ws: Optional[Sequence[torch.Tensor]] = None, out=None, stream=None,
+                           jobs: Optional[QuantizeJobs] = None):
     """prom_quantize_ternary_batch: a list of device float32 [cout, cin] matrices -> a list of
-    (packed uint8 [cout, ceil(cin/4)], alpha float32 [cout]); `out` may carry that list."""
-    if out is None:
-        out = [(torch.empty((w.shape[0], (w.shape[1] + 3) // 4), dtype=torch.uint8, device=w.device),
-                torch.empty((w.shape[0],), dtype=torch.float32, device=w.device)) for w in ws]
-    jobs = (PromQuantizeJob * len(ws))()
-    for j, (w, (packed, alpha)) in enumerate(zip(ws, out)):
-        jobs[j] = PromQuantizeJob(_dev(w, torch.float32, "w"), w.shape[0], w.shape[1], packed.data_ptr(),
-                                  packed.numel(), alpha.data_ptr())
-    _check(lib().prom_quantize_ternary_batch(jobs, len(ws), _stream(stream)), "prom_quantize_ternary_batch")
-    return out
+    (packed uint8 [cout, ceil(cin/4)], alpha float32 [cout]); `out` may carry that list, `jobs` a
+    table marshalled earlier (then ws and out are not looked at)."""
+    if jobs is None:
+        jobs = QuantizeJobs(ws, out)
+    _check(lib().prom_quantize_ternary_batch(jobs.array, jobs.n, _stream(stream)), "prom_quantize_ternary_batch")
+    return jobs.out
 
 
 def requant_from_scale(scale: float):

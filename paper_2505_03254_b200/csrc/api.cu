@@ -1335,7 +1335,8 @@ prom_status prom_quantize_ternary(const float *w_dev, int cout, int cin, uint8_t
     if (packed_bytes < prom_packed_bytes(cout, cin)) return PROM_ERR_WORKSPACE;
     DeviceInfo d = device_info();
     if (!d.ok) return PROM_ERR_CUDA;
-    const int grid = cout < d.sms * 8 ? cout : d.sms * 8;
+    const int want = (cout + quant::kWarps - 1) / quant::kWarps;        // a warp per row
+    const int grid = want < d.sms * 16 ? want : d.sms * 16;
     quant::quantize_ternary_kernel<<<grid, quant::kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
         w_dev, cout, cin, 1e-5, packed_dev, alpha_dev);
     ++g_launches;
@@ -1366,7 +1367,8 @@ prom_status prom_quantize_ternary_batch(const prom_quantize_job *jobs, int n, vo
             t.cin[i] = j.cin; t.w[i] = j.w_dev; t.packed[i] = j.packed_dev; t.alpha[i] = j.alpha_dev;
         }
         t.first_row[t.n] = rows;
-        const int grid = rows < d.sms * 16 ? rows : d.sms * 16;
+        const int want = (rows + quant::kWarps - 1) / quant::kWarps;      // a warp per row
+        const int grid = want < d.sms * 16 ? want : d.sms * 16;
         quant::quantize_ternary_batch_kernel<<<grid, quant::kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
             t, 1e-5);
         ++g_launches;
