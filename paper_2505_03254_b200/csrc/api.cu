@@ -300,10 +300,16 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
                                : ((double)pl.grid / d.sms > per_sm ? per_sm : (double)pl.grid / d.sms);
     const double epi_rate = 36e3 / ctas_per_sm;              // outputs per microsecond per CTA
     const double load_rate = 60e3 / ctas_per_sm;             // bytes per microsecond per CTA
-    const double t_epi = (double)tm * nt / epi_rate;
+    // subtile widths with a straight-line epilogue (tc.cuh: epi_fast_fixed); any other width that
+    // splits a row runs the looped epilogue, measured ~1 us per layer slower at 128 columns
+    const bool straight = nt == 96 || nt == 64 || nt == 48 || nt == 32 || nt == 80;
+    const double t_epi = (double)tm * nt / epi_rate * (straight || n_sub == 1 ? 1.0 : 1.5);
     const double t_load = (double)kc * tm * (kf < cw ? kf : cw) / load_rate;
-    const double t_first = (t_epi > t_load ? t_epi : t_load) + 0.1;
-    const double t_next = share_x ? t_epi + 0.1 : t_first;
+    // 0.8 us per unit for the hand-overs around it (barrier waits, fences, store issue): fitted to
+    // plans timed inside the chained step (32 -> 192 and 64 -> 384 prefer 96-column subtiles in
+    // fewer channel groups to 64-column ones)
+    const double t_first = (t_epi > t_load ? t_epi : t_load) + 0.8;
+    const double t_next = share_x ? t_epi + 0.8 : t_first;
     const double startup = 1.2 + (double)p.image_bytes / 80e3 * ctas_per_sm;
     const double fill = 1.0 + 0.1 * kc;                      // first load, first MMA
     const double last = 0.45 * ((nt + 31) / 32) + 0.8;       // draining the last accumulator, store
