@@ -299,7 +299,8 @@ static bool tc_fill_plan(long long m, int cin, int cout, const RowMap &map, cons
     const double ctas_per_sm = (double)pl.grid / d.sms < 1.0 ? 1.0
                                : ((double)pl.grid / d.sms > per_sm ? per_sm : (double)pl.grid / d.sms);
     const double epi_rate = 36e3 / ctas_per_sm;              // outputs per microsecond per CTA
-    const double load_rate = 60e3 / ctas_per_sm;             // bytes per microsecond per CTA
+    // an SM takes 58 bytes per clock from L2 (the copy-rate probe): 110 KB per microsecond
+    const double load_rate = 110e3 / ctas_per_sm;            // bytes per microsecond per CTA
     // subtile widths with a straight-line epilogue (tc.cuh: epi_fast_fixed); any other width that
     // splits a row runs the looped epilogue, measured ~1 us per layer slower at 128 columns
     const bool straight = nt == 96 || nt == 64 || nt == 48 || nt == 32 || nt == 80;
