@@ -843,15 +843,16 @@ def body_with_depthwise_timing(torch, binding, synth, bw, skips=False):
 
 def depth_first_timing(torch, binding, synth):
     """The three runs of late layers of the network (28x28, 14x14 and 7x7 feature maps) and the
-    whole step, each as a CUDA graph, with one launch per layer and with the depth-first launches
-    of prom_debug_seq_chain(1); outputs compared."""
+    whole step, each as a CUDA graph, with one launch per layer, with the depth-first launches
+    of prom_debug_seq_chain(1) and with the runs that stay in shared memory of
+    prom_debug_seq_chain(2); outputs compared."""
     table = synth.mobilenetv2_pointwise_layers()
     seed = synth.BASE_SEED + 3
     rows = []
     for lo, hi in ((6, 12), (12, 26), (26, 34), (0, 34)):
         res = {}
         outs = []
-        for mode in (0, 1):
+        for mode in (0, 1, 2):
             binding.debug_seq_chain(mode)
             dev = []
             for i, l in enumerate(table[lo:hi]):
@@ -879,8 +880,9 @@ def depth_first_timing(torch, binding, synth):
             res[("status", mode)] = binding.last_device_status()
         binding.debug_seq_chain(0)
         rows.append({"layers": f"{lo + 1}..{hi}", "us_one_launch_per_layer": round(res[0], 1),
-                     "us_depth_first": round(res[1], 1), "same_output": bool(torch.equal(outs[0], outs[1])),
-                     "device_status": [res[("status", 0)], res[("status", 1)]]})
+                     "us_depth_first": round(res[1], 1), "us_resident_runs": round(res[2], 1),
+                     "same_output": bool(torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])),
+                     "device_status": [res[("status", m)] for m in (0, 1, 2)]})
     return rows
 
 

@@ -46,6 +46,14 @@ int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
  * layer.  Results do not depend on the mode; the workspace size does
  * (prom_layer_seq_workspace_bytes follows the mode; a workspace that is too
  * small for the depth-first buffers falls back to one launch per layer).
+ * 2 = runs that stay in shared memory: consecutive layers on the same rows
+ * (only the first may subsample), channel counts multiples of 16, no depthwise
+ * convolution and no skip connection, alternately at most 384 output channels
+ * (the first layer and every second one after it) and at most 384 input
+ * channels (the layers in between), any clamp; one launch takes a tile of rows
+ * through all of them and only the run's last layer writes a tensor (to a
+ * buffer of its own in the workspace, or to y_out).  The inner layers have no
+ * output tensor: prom_debug_layer_seq_output_offset returns -2 for them.
  * Process-wide. */
 void prom_debug_seq_chain(int mode);
 
@@ -71,9 +79,10 @@ void prom_debug_tc_wide(int mode, int blocks);
 /* Where layer `layer`'s output ([rows][cout] int8) sits in the workspace of a
  * prom_pw_layer_seq call whose workspace has prom_layer_seq_workspace_bytes
  * bytes, with AUTO or TC as the variant: the byte offset from the workspace's
- * start, or -1 for the last layer (its output is y_out_dev) or a bad argument.
- * *chained (may be NULL) receives 1 when the layer runs inside a depth-first
- * launch.  A layer's output stays intact until the layer two further on has
+ * start, -1 for the last layer (its output is y_out_dev) or a bad argument,
+ * -2 for a layer inside a shared-memory run (prom_debug_seq_chain(2)) that is
+ * not the run's last: it writes no tensor.  *chained (may be NULL) receives 1
+ * when the layer runs inside a multi-layer launch.  A layer's output stays intact until the layer two further on has
  * run (ping-pong regions) or, inside a depth-first launch, until the next
  * call. */
 int64_t prom_debug_layer_seq_output_offset(const prom_layer *layers, int n, int batch, int h0,

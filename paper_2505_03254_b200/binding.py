@@ -286,13 +286,14 @@ def debug_tc_wide(mode: int = 0, blocks: int = 0) -> None:
 
 def debug_seq_chain(mode: int = 0) -> None:
     """prom_debug_seq_chain: 0 = one launch per layer (default), 1 = depth-first launches for
-    every run of layers that qualifies."""
+    every run of layers that qualifies, 2 = runs whose activations stay in shared memory."""
     lib().prom_debug_seq_chain(int(mode))
 
 
 def debug_layer_seq_output_offset(seq: "LayerSeq", batch: int, h0: int, w0: int, layer: int):
-    """prom_debug_layer_seq_output_offset: (byte offset of the layer's output in the workspace or
-    -1, whether the layer runs inside a depth-first launch)."""
+    """prom_debug_layer_seq_output_offset: (byte offset of the layer's output in the workspace, -1
+    for a bad argument or -2 for a layer inside a shared-memory run, which writes no tensor;
+    whether the layer runs inside a multi-layer launch)."""
     chained = C.c_int(0)
     off = lib().prom_debug_layer_seq_output_offset(seq.array, seq.n, batch, h0, w0, layer, C.byref(chained))
     return int(off), bool(chained.value)

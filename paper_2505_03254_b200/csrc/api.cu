@@ -27,6 +27,7 @@
 #include "depthwise.cuh"
 #include "dwtc.cuh"
 #include "wide.cuh"
+#include "stack.cuh"
 #include "quantize.cuh"
 #include "peak.cuh"
 
@@ -788,7 +789,102 @@ struct ChainPlan {
     int first = 0, last = 0;             // layers [first, last]
     int tm = 128, n_tasks = 0, grid = 0, box_r = 0;
     std::vector<TcPlan> prep;            // per layer: the plan whose image layout the kernel reads
+    // kind 1: the run stays in shared memory (stack.cuh); `prep` is then empty
+    int kind = 0;
+    stack::Table st;                     // everything but pointers and tensor maps
+    size_t smem = 0;
 };
+
+// Global scratch of one layer of a resident run: the int8 matrix, bias digits and constants that
+// wide_prep_kernel writes, column tile after column tile.
+struct StackScratch { size_t w8, wbias, consts, total; int n_ct, k_pad; };
+static StackScratch stack_scratch(int cin, int cout)
+{
+    StackScratch z;
+    z.n_ct = (cout + 127) / 128;
+    z.k_pad = (cin + 127) / 128 * 128;
+    z.w8 = (size_t)z.n_ct * 128 * z.k_pad;
+    z.wbias = (size_t)z.n_ct * stack::kWbiasBytes;
+    z.consts = round256((size_t)z.n_ct * stack::kConstBytes);
+    z.total = z.w8 + z.wbias + z.consts;
+    return z;
+}
+
+// The layers of a resident run alternate: P layers (the first and every second one after it; at
+// most 384 output channels) and E layers (at most 384 input channels).
+static bool stack_layer_ok(const prom_layer &l, bool is_p)
+{
+    if (l.dw_w || l.add_block_input || l.cin % 16 || l.cout % 16 || l.cin > 4096 || l.cout > 4096) return false;
+    return is_p ? l.cout <= 128 * stack::kNarrowMax : l.cin <= 128 * stack::kNarrowMax;
+}
+
+// Roles, accumulator slots, shared-memory layout and rings of a resident run over the layers
+// [c.first, c.last]; false when it does not fit.
+static bool stack_fill(const prom_layer *layers, const DeviceInfo &d, ChainPlan &c)
+{
+    stack::Table &t = c.st;
+    memset(&t, 0, sizeof(t));
+    const int n = c.last - c.first + 1;
+    if (n < 2 || n > stack::kMaxLayers) return false;
+    int narrow = 1, ring_chunks = 0;
+    for (int l = 0; l < n; ++l) {
+        const prom_layer &pl = layers[c.first + l];
+        stack::Layer &L = t.layer[l];
+        L.cout = pl.cout;
+        L.kc = (pl.cin + 127) / 128;
+        L.ksteps = (pl.cin + 31) / 32;
+        L.n_ct = (pl.cout + 127) / 128;
+        L.act_min = pl.rq.act_min; L.act_max = pl.rq.act_max;
+        L.streamed = (l & 1) ? 0 : 1;
+        L.out_mode = l == n - 1 ? 2 : (L.streamed ? 0 : 1);
+        if (L.streamed) {
+            if (L.n_ct > stack::kNarrowMax) return false;
+            L.ring_off = ring_chunks;
+            ring_chunks += L.kc;
+            if (L.out_mode == 0 && L.n_ct > narrow) narrow = L.n_ct;
+        } else if (L.kc > stack::kNarrowMax) {
+            return false;
+        }
+    }
+    // accumulators: a P layer keeps all of its units' live, two of the four slots unless it has three
+    // units; the E layer in front of it takes what is left
+    for (int l = 0; l < n; ++l) {
+        stack::Layer &L = t.layer[l];
+        if (L.streamed) {
+            L.nslots = L.n_ct == 3 ? 3 : 2;
+            L.slot0 = stack::kAccs - L.nslots;
+        } else {
+            const bool tight = l + 1 < n && t.layer[l + 1].n_ct == 3;
+            L.slot0 = 0;
+            L.nslots = tight ? 1 : 2;
+        }
+    }
+    t.n_layers = n;
+    t.tm = c.tm; t.box_r = c.box_r; t.x3d = c.box_r > 0 ? 1 : 0;
+    t.n_mtiles = c.n_tasks;
+    t.chunks_per_tile = ring_chunks;
+    t.ring = 3;
+    const uint32_t const_bytes = stack::kAccs * stack::kSlotBytes;
+    const uint32_t fixed = const_bytes + stack::kEpiWarps * stack::kSlabBytes + tc::kAConstBytes + 1024;
+    const uint32_t act_bytes = (uint32_t)(narrow + t.ring) * stack::kChunkBytes;
+    const long long room = (long long)d.smem_optin - 1024 - act_bytes - fixed;
+    int stages = (int)(room / stack::kChunkBytes);
+    if (stages > stack::kMaxStages) stages = stack::kMaxStages;
+    stages &= ~1;                   // one half of the ring per issuing thread
+    if (stages < 4) return false;
+    t.stages = stages;
+    t.off_nar = 0;
+    t.off_ring = (uint32_t)narrow * stack::kChunkBytes;
+    t.off_w = t.off_ring + (uint32_t)t.ring * stack::kChunkBytes;
+    t.off_aconst = t.off_w + (uint32_t)stages * stack::kChunkBytes;
+    t.off_const = t.off_aconst + tc::kAConstBytes;
+    t.off_out = t.off_const + const_bytes;
+    t.off_bars = t.off_out + stack::kEpiWarps * stack::kSlabBytes;
+    c.smem = t.off_bars + 1024 + 1024;
+    // one CTA per SM whatever the size: each allocates all of tensor memory
+    if (c.smem < (size_t)d.smem_optin / 2 + 2048) c.smem = (size_t)d.smem_optin / 2 + 2048;
+    return true;
+}
 
 static int chain_nt(int cout)
 {
@@ -818,8 +914,42 @@ static void find_chains(const prom_layer *layers, int n, const SeqShape &s, cons
                         std::vector<ChainPlan> &out)
 {
     out.clear();
-    if (!g_seq_chain.load()) return;
+    const int mode = g_seq_chain.load();
+    if (!mode) return;
     int i = 0;
+    while (mode == 2 && i < n) {
+        // runs that stay in shared memory: P, E, P, E, ...
+        if (!stack_layer_ok(layers[i], true) || s.m[i] <= 0 || s.m[i] + 256 >= (1ll << 31)) { ++i; continue; }
+        ChainPlan c;
+        c.kind = 1;
+        c.first = i;
+        const RowMap &mp = s.map[i];
+        if (mp.stride != 1) {
+            if (mp.wo > 128) { ++i; continue; }
+            c.box_r = 128 / mp.wo;
+            const long long lines = s.m[i] / mp.wo;
+            if (c.box_r > lines) c.box_r = (int)lines;
+            c.tm = c.box_r * mp.wo;
+        }
+        c.n_tasks = (int)((s.m[i] + c.tm - 1) / c.tm);
+        int j = i + 1;
+        while (j < n && j - i < stack::kMaxLayers && s.m[j] == s.m[i] && s.map[j].stride == 1 &&
+               stack_layer_ok(layers[j], ((j - i) & 1) == 0))
+            ++j;
+        // the longest run that fits
+        bool found = false;
+        for (; j - i >= 2 && !found; --j) {
+            // a skip connection into layer j reads the output of layer j - 2, which must exist
+            if (j < n && layers[j].add_block_input) continue;
+            c.last = j - 1;
+            found = stack_fill(layers, d, c);
+        }
+        if (!found) { ++i; continue; }
+        c.grid = c.n_tasks < d.sms ? c.n_tasks : d.sms;
+        out.push_back(c);
+        i = c.last + 1;
+    }
+    if (mode == 2) return;
     while (i < n) {
         if (!chain_layer_ok(layers[i]) || s.m[i] <= 0) { ++i; continue; }
         ChainPlan c;
@@ -918,8 +1048,12 @@ static void seq_layout(const prom_layer *layers, int n, const SeqShape &s, const
     for (int i = 0; i < n; ++i) {
         if (L.chain_of[i] >= 0) {
             const ChainPlan &c = L.chains[L.chain_of[i]];
-            const tc::Params &p = c.prep[i - c.first].p;
             L.cimg_off[i] = L.cimg_total;
+            if (c.kind == 1) {
+                L.cimg_total += round256(stack_scratch(layers[i].cin, layers[i].cout).total);
+                continue;
+            }
+            const tc::Params &p = c.prep[i - c.first].p;
             L.cimg_total += round256((size_t)p.groups * p.image_stride);
             continue;
         }
@@ -931,6 +1065,9 @@ static void seq_layout(const prom_layer *layers, int n, const SeqShape &s, const
     }
     for (int i = 0; i < n; ++i)
         if (L.chain_of[i] >= 0 && i + 1 < n) {
+            // (the inner layers of a resident run have no output tensor)
+            const ChainPlan &c = L.chains[L.chain_of[i]];
+            if (c.kind == 1 && i != c.last) continue;
             L.cbuf_off[i] = L.cimg_total + L.cbuf_total;
             L.cbuf_total += round256((size_t)s.m[i] * layers[i].cout);
         }
@@ -1120,6 +1257,46 @@ static prom_status launch_chain(const prom_layer *layers, const SeqShape &s, con
     return cuda_status(e);
 }
 
+// One launch of stack_kernel for the layers [c.first, c.last] of a resident run.
+static prom_status launch_stack(const prom_layer *layers, const SeqShape &s, const ChainPlan &c,
+                                const std::vector<Conv> &conv, uint8_t *const *scratch, const DeviceInfo &d,
+                                bool pdl, bool pdl_next, cudaStream_t st)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return PROM_ERR_CUDA;
+    stack::Table t = c.st;
+    t.m = s.m[c.first];
+    t.pdl = pdl ? 1 : 0;
+    t.pdl_next = pdl_next ? 1 : 0;
+    t.y = conv[c.last].y;
+    const bool strided = s.map[c.first].stride != 1;
+    if (!make_x_map(&t.xmap, conv[c.first].x, layers[c.first].cin, s.m[c.first], 128,
+                    strided ? &s.map[c.first] : nullptr, c.box_r))
+        return PROM_ERR_CUDA;
+    if (!make_y_map(&t.ymap, conv[c.last].y, layers[c.last].cout, s.m[c.last], 32)) return PROM_ERR_CUDA;
+    cuuint32_t es[2] = {1, 1};
+    for (int i = c.first; i <= c.last; ++i) {
+        stack::Layer &L = t.layer[i - c.first];
+        const StackScratch z = stack_scratch(layers[i].cin, layers[i].cout);
+        cuuint64_t dims[2] = {(cuuint64_t)z.k_pad, (cuuint64_t)z.n_ct * 128};
+        cuuint64_t strides[1] = {(cuuint64_t)z.k_pad};
+        cuuint32_t box[2] = {128, 128};
+        if (enc(&L.wmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, scratch[i], dims, strides, box, es,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PROM_ERR_CUDA;
+        L.wbias = scratch[i] + z.w8;
+        L.consts = scratch[i] + z.w8 + z.wbias;
+    }
+    if (raise_smem_limit(stack::stack_kernel, d.smem_optin) != cudaSuccess) return PROM_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fill_launch_cfg(cfg, attr, c.grid, stack::kThreads, c.smem, st, pdl);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, stack::stack_kernel, t);
+    ++g_launches;
+    return cuda_status(e);
+}
+
 static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, int batch, int h0,
                            int w0, void *ws, size_t ws_bytes, int8_t *y_out, prom_variant variant,
                            cudaStream_t st)
@@ -1216,6 +1393,7 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
                 const TcPlan *pl = nullptr;
                 if (lay.chain_of[i] >= 0) {
                     const ChainPlan &c = lay.chains[lay.chain_of[i]];
+                    if (c.kind == 1) continue;          // prepared by the batch below
                     TcPlan tmp = c.prep[i - c.first];
                     tc_bind(conv[i], tmp, chain_img[i]);
                     t.layer[t.n] = tmp.p;
@@ -1239,10 +1417,41 @@ static prom_status run_seq(const prom_layer *layers, int n, const int8_t *x0, in
         }
     }
 
+    // ... and one launch the operands of the runs that stay in shared memory
+    if (chain_base) {
+        int i = 0;
+        while (i < n) {
+            wide::PrepBatch b;
+            memset(&b, 0, sizeof(b));
+            int ctas = 0;
+            for (; i < n && b.n < wide::kMaxPrepLayers; ++i) {
+                if (lay.chain_of[i] < 0 || lay.chains[lay.chain_of[i]].kind != 1) continue;
+                const StackScratch z = stack_scratch(layers[i].cin, layers[i].cout);
+                wide::PrepParams &pp = b.layer[b.n];
+                pp.cin = layers[i].cin; pp.cout = layers[i].cout; pp.k_pad = z.k_pad; pp.w_packed = layers[i].w_packed;
+                pp.bias = layers[i].rq.bias; pp.mult = layers[i].rq.mult; pp.shift = layers[i].rq.shift;
+                pp.act_min = layers[i].rq.act_min; pp.act_max = layers[i].rq.act_max;
+                pp.w8 = reinterpret_cast<int8_t *>(chain_img[i]);
+                pp.wbias = chain_img[i] + z.w8;
+                pp.consts = chain_img[i] + z.w8 + z.wbias;
+                b.first[b.n] = ctas;
+                ctas += z.n_ct;
+                ++b.n;
+            }
+            if (b.n == 0) break;
+            b.first[b.n] = ctas;
+            wide::wide_prep_batch_kernel<<<ctas, 256, 0, st>>>(b);
+            ++g_launches;
+            if (cudaGetLastError() != cudaSuccess) return PROM_ERR_CUDA;
+        }
+    }
+
     for (int i = 0; i < n; ++i) {
         if (lay.chain_of[i] >= 0) {
             const ChainPlan &c = lay.chains[lay.chain_of[i]];
-            prom_status e = launch_chain(layers, s, c, conv, chain_img.data(), c.first > 0, c.last + 1 < n, st);
+            prom_status e = c.kind == 1
+                ? launch_stack(layers, s, c, conv, chain_img.data(), d, c.first > 0, c.last + 1 < n, st)
+                : launch_chain(layers, s, c, conv, chain_img.data(), c.first > 0, c.last + 1 < n, st);
             if (e != PROM_OK) return e;
             i = c.last;
             continue;
@@ -1962,7 +2171,7 @@ prom_status prom_debug_mma_beside(int mode, int iters, int nwarps, int stages, c
     return cuda_status(cudaGetLastError());
 }
 
-void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode ? 1 : 0); }
+void prom_debug_seq_chain(int mode) { g_seq_chain.store(mode == 2 ? 2 : (mode ? 1 : 0)); }
 
 void prom_debug_dw_variant(int variant) { g_dw_variant.store(variant < 0 || variant > 2 ? 0 : variant); }
 
@@ -1982,7 +2191,11 @@ int64_t prom_debug_layer_seq_output_offset(const prom_layer *layers, int n, int 
     seq_layout(layers, n, s, d, true, lay);
     const bool in_chain = lay.chain_of[layer] >= 0;
     if (chained) *chained = in_chain ? 1 : 0;
-    if (in_chain) return (int64_t)(round256(lay.with_images()) + lay.cbuf_off[layer]);
+    if (in_chain) {
+        const ChainPlan &c = lay.chains[lay.chain_of[layer]];
+        if (c.kind == 1 && layer != c.last) return -2;      // never written: it stays in shared memory
+        return (int64_t)(round256(lay.with_images()) + lay.cbuf_off[layer]);
+    }
     return (layer & 1) ? (int64_t)lay.ra : 0;
 }
 

@@ -67,12 +67,12 @@ struct PrepParams {
     uint8_t *wbias, *consts;
 };
 
-// One CTA per column tile.
-__global__ void __launch_bounds__(256, 1) wide_prep_kernel(const PrepParams p)
+// The operands of column tile `tile` of one layer; all 256 threads of the CTA take part.
+__device__ __forceinline__ void prep_tile(const PrepParams &p, const int tile)
 {
     __shared__ int s_mult[kNt], s_bias[kNt], s_shift[kNt];
     __shared__ int s_flags[4];      // shmin, shmax, bad, slow
-    const int tile = blockIdx.x, n0 = tile * kNt;
+    const int n0 = tile * kNt;
     if (threadIdx.x == 0) { s_flags[0] = 31; s_flags[1] = 0; s_flags[2] = 0; s_flags[3] = 0; }
     __syncthreads();
     if (threadIdx.x < kNt) {
@@ -147,6 +147,24 @@ __global__ void __launch_bounds__(256, 1) wide_prep_kernel(const PrepParams p)
         *reinterpret_cast<uint4 *>(p.w8 + (size_t)n * p.k_pad + j * 16) = val;
     }
     if (invalid) raise_status(PROM_ERR_BAD_WEIGHT);
+}
+
+// One CTA per column tile.
+__global__ void __launch_bounds__(256, 1) wide_prep_kernel(const PrepParams p) { prep_tile(p, (int)blockIdx.x); }
+
+// The same for several layers in one launch: CTA b belongs to the layer l with first[l] <= b < first[l + 1].
+constexpr int kMaxPrepLayers = 16;
+struct PrepBatch {
+    int n;
+    int first[kMaxPrepLayers + 1];
+    PrepParams layer[kMaxPrepLayers];
+};
+
+__global__ void __launch_bounds__(256, 1) wide_prep_batch_kernel(const __grid_constant__ PrepBatch t)
+{
+    int l = 0;
+    while (l + 1 < t.n && (int)blockIdx.x >= t.first[l + 1]) ++l;
+    prep_tile(t.layer[l], (int)blockIdx.x - t.first[l]);
 }
 
 // Two threads issue MMAs (warps 1 and 18), each with half of the weight ring (stages t, t + 2, ..),
