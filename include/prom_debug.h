@@ -56,6 +56,11 @@ int prom_debug_tc_plan_query(int64_t m, int cin, int cout, int *out9);
  * output tensor: prom_debug_layer_seq_output_offset returns -2 for them.
  * Process-wide. */
 void prom_debug_seq_chain(int mode);
+/* Order of the row tiles inside the tensor-core layers of prom_pw_layer_seq:
+ * 1 (default) = every second layer walks its tiles from the last to the first,
+ * so that it reads first what the layer before wrote last; 0 = every layer
+ * from the first to the last.  Results do not depend on it.  Process-wide. */
+void prom_debug_seq_order(int alternate);
 
 /* Which kernel prom_dw_conv3x3_i8 runs: 0 = the library's choice (default: TMA
  * patches and tensor-core taps for stride 1 with a channel count that is a

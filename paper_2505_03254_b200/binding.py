@@ -29,7 +29,7 @@ EXPORTS = [
     "prom_launch_count", "prom_shutdown", "prom_status_string",
     "prom_pw_conv_i8_addsub_static", "prom_debug_tc_plan", "prom_debug_tc_plan_query",
     "prom_quantize_ternary", "prom_requant_from_scale", "prom_quantize_act_absmax", "prom_pw_conv_i8_dyn", "prom_dw_conv3x3_i8", "prom_debug_tc_plan_shape", "prom_pw_conv_i8_res",
-    "prom_debug_seq_chain", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
+    "prom_debug_seq_chain", "prom_debug_seq_order", "prom_debug_wait_timeout", "prom_debug_i8_mma_rate", "prom_debug_alu_rate",
     "prom_debug_once_per_device", "prom_debug_layer_seq_output_offset",
     "prom_pw_prepared_bytes", "prom_pw_prepare", "prom_pw_conv_i8_prepared", "prom_quantize_ternary_batch",
     "prom_debug_dw_variant", "prom_debug_tc_wide", "prom_debug_mma_issue_rate", "prom_debug_l2_copy_rate",
@@ -124,6 +124,8 @@ def lib():
         L.prom_debug_tc_wide.argtypes = [i32, i32]
         L.prom_debug_seq_chain.restype = None
         L.prom_debug_seq_chain.argtypes = [i32]
+        L.prom_debug_seq_order.restype = None
+        L.prom_debug_seq_order.argtypes = [i32]
         L.prom_debug_layer_seq_output_offset.restype = i64
         L.prom_debug_layer_seq_output_offset.argtypes = [C.POINTER(PromLayer), i32, i32, i32, i32, i32,
                                                          C.POINTER(C.c_int)]
@@ -288,6 +290,12 @@ def debug_seq_chain(mode: int = 0) -> None:
     """prom_debug_seq_chain: 0 = one launch per layer (default), 1 = depth-first launches for
     every run of layers that qualifies, 2 = runs whose activations stay in shared memory."""
     lib().prom_debug_seq_chain(int(mode))
+
+
+def debug_seq_order(alternate: bool = True) -> None:
+    """prom_debug_seq_order: whether every second layer of a sequence walks its row tiles backwards
+    (the default)."""
+    lib().prom_debug_seq_order(1 if alternate else 0)
 
 
 def debug_layer_seq_output_offset(seq: "LayerSeq", batch: int, h0: int, w0: int, layer: int):

@@ -77,6 +77,7 @@ struct Params {
     int8_t *y;
     int pdl;            // launched with programmatic dependent launch
     int pdl_next;       // the next kernel in the stream is launched that way
+    int reverse;        // row tiles are taken from the last to the first
     // The dynamic layer (kernel modes 1 and 2): `mult` then holds the bit patterns of the
     // float per-channel factors alpha, bias and shift are not read, and rows belong to
     // samples of rows_per_sample rows each.
@@ -846,7 +847,8 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
                 // CTA follows from its loads, so it alone waits for that kernel to finish.
                 if (p.pdl) ptx::grid_dep_wait();
                 for (int mt = worker; mt < p.n_mtiles && ok; mt += nworkers) {
-                    const int c_row = p.x3d ? mt * p.box_r : mt * p.tm;
+                    const int mtx = p.reverse ? p.n_mtiles - 1 - mt : mt;
+                    const int c_row = p.x3d ? mtx * p.box_r : mtx * p.tm;
                     int cx = 0;
                     for (int l = 0; l < loads_per_tile; ++l) {
                         if (!wait_bar(bempty, ph ^ 1u, flags)) { ok = false; break; }
@@ -981,10 +983,13 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             // the next unit of the group is two further on: with one subtile per CTA that is two
             // tiles on, otherwise two subtiles on and at most one step to the next tile
             const int dls = subs == 1 ? 0 : kEpiGroups;
-            const int drow = subs == 1 ? kEpiGroups * nworkers * p.tm : 0, drow_wrap = nworkers * p.tm;
+            // (in a sequence every second layer walks its tiles backwards: what the layer before
+            // wrote last, and is still in L2, is read first)
+            const int dir = p.reverse ? -1 : 1;
+            const int drow = subs == 1 ? dir * kEpiGroups * nworkers * p.tm : 0, drow_wrap = dir * nworkers * p.tm;
             const bool whole_tile = p.tm - q * 32 >= 32;     // a tile gives this warp 32 rows
-            int row0 = mt0 * p.tm + q * 32;             // first row of this warp's slab
-            const int row_end = p.n_mtiles * p.tm + q * 32;
+            int row0 = (p.reverse ? p.n_mtiles - 1 - mt0 : mt0) * p.tm + q * 32;   // first row of this warp's slab
+            const unsigned row_span = (unsigned)(p.n_mtiles * p.tm);
             const uint32_t slab_bytes = 32u * (uint32_t)p.nf;
             int col = (g + ls * p.groups) * p.nt;       // first column of the subtile
             const int dcol = dls * p.groups * p.nt;
@@ -993,7 +998,7 @@ tc_conv_kernel(const __grid_constant__ CUtensorMap xmap, const __grid_constant__
             const uint32_t btoggle = p.nbuf == 4 ? 2u : 0u;
             uint32_t b = (uint32_t)grp, tph = 0;
             uint32_t st = (uint32_t)grp % (uint32_t)p.stages;    // stage of this group's unit (epi_frees)
-            while (row0 < row_end && ok) {
+            while ((unsigned)(row0 - q * 32) < row_span && ok) {
                 // The residual (mode 3): the bytes that sit where this slab goes in Y, in 8-byte
                 // granules across the warp.  The first kResHeld granules of a lane are requested
                 // before the wait for the accumulator, so that their latency hides behind it.

@@ -360,3 +360,29 @@ def test_seeded_random_stacks(oracle):
         got = y.cpu().numpy()
         assert got.shape == cur.shape, (case, got.shape, cur.shape)
         assert np.array_equal(got, cur), (case, [(l["cin"], l["cout"], l["in_stride"], "dw_w" in l) for l in host])
+
+
+def test_tile_order_does_not_change_the_bytes(oracle):
+    """Every second layer walks its row tiles backwards by default: the same bytes as with every
+    layer walking forwards, on a network with subsampled layers and ragged last tiles."""
+    table = synth.mobilenetv2_pointwise_layers(h0=48, w0=80)
+    host, dev = [], []
+    for i, l in enumerate(table):
+        d = synth.make_layer(91, l.cin, l.cout, 0.5, index=i + 1)
+        host.append(dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride, w=d["w"].numpy(), bias=d["bias"].numpy(),
+                         mult=d["mult"].numpy(), shift=d["shift"].numpy()))
+        dev.append(dict(cin=l.cin, cout=l.cout, in_stride=l.in_stride, w_packed=binding.pack_ternary(d["w"].cuda()),
+                        bias=d["bias"].cuda(), mult=d["mult"].cuda(), shift=d["shift"].cuda()))
+    seq = binding.LayerSeq(dev)
+    x0 = synth.act_post_relu6(91, (7, 48, 80, 32))
+    ws = torch.empty((seq.workspace_bytes(7, 48, 80),), dtype=torch.uint8, device="cuda")
+    y1 = binding.pw_layer_seq(seq, x0.cuda(), ws).clone()
+    try:
+        binding.debug_seq_order(False)
+        y0 = binding.pw_layer_seq(seq, x0.cuda(), ws).clone()
+    finally:
+        binding.debug_seq_order(True)
+    torch.cuda.synchronize()
+    assert binding.last_device_status() == binding.PROM_OK
+    assert torch.equal(y0, y1)
+    assert np.array_equal(y1.cpu().numpy(), oracle.layer_seq(host, x0.numpy()))
