@@ -165,11 +165,13 @@ def i8_peak_probe(torch, binding, iters=8192, reps=5, sustained_s=0.0):
 
 def alu_rate_probe(torch, binding, iters=2000):
     """Measured issue rates (lanes per clock per SM) of the requantiser's 32-bit high multiply and,
-    beside it, of mad.lo.s32 and fma.rn.f32: 8 independent chains per thread, 1024 threads per SM."""
+    beside it, of mad.lo.s32, fma.rn.f32, mad.wide.s32, the saturating pack, a shift and fma.rn.f64:
+    8 independent chains per thread, 1024 threads per SM."""
     cycles = torch.zeros((4096,), dtype=torch.int64, device="cuda")
     sink = torch.zeros((1,), dtype=torch.int32, device="cuda")
     out = {}
-    for op, name in ((0, "mul_hi_s32"), (1, "mad_lo_s32"), (2, "fma_f32")):
+    for op, name in ((0, "mul_hi_s32"), (1, "mad_lo_s32"), (2, "fma_f32"), (3, "mad_wide_s32"),
+                     (4, "cvt_pack_sat_u8"), (5, "shr_s32"), (6, "fma_f64")):
         binding.debug_alu_rate(op, 100, sink, cycles)
         grid = binding.debug_alu_rate(op, iters, sink, cycles)
         torch.cuda.synchronize()

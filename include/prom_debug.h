@@ -111,7 +111,8 @@ prom_status prom_debug_wait_timeout(uint64_t limit_ns, int *gave_up_dev, void *c
  *     a bounded wait at the end: 2 * 128 * 256 * 32 * 4 * iters operations per CTA.
  *     1 <= iters <= 2^20.
  *   alu_rate: op 0 = mul.hi.s32 (the requantiser's multiply), 1 = mad.lo.s32,
- *     2 = fma.rn.f32; two CTAs of 512 threads per SM, 8 independent chains per
+ *     2 = fma.rn.f32, 3 = mad.wide.s32 (high word fed back), 4 = cvt.pack.sat.u8.s32,
+ *     5 = shr.s32, 6 = fma.rn.f64; two CTAs of 512 threads per SM, 8 independent chains per
  *     thread, 64 * iters instructions per thread.  sink_dev: one device int.
  * Asynchronous on the stream. */
 prom_status prom_debug_i8_mma_rate(int iters, long long *cycles_dev, int cycles_len, int *grid_out,

@@ -2097,7 +2097,7 @@ prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cyc
                                 int cycles_len, int *grid_out, void *cuda_stream)
 {
     if (!sink_dev || !cycles_dev || !grid_out) return PROM_ERR_NULL;
-    if (op < 0 || op > 2 || iters < 1 || iters > (1 << 24)) return PROM_ERR_SHAPE;
+    if (op < 0 || op > 6 || iters < 1 || iters > (1 << 24)) return PROM_ERR_SHAPE;
     DeviceInfo d = device_info();
     if (!d.ok) return PROM_ERR_CUDA;
     const int grid = 2 * d.sms;
@@ -2106,7 +2106,11 @@ prom_status prom_debug_alu_rate(int op, int iters, int *sink_dev, long long *cyc
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (op == 0) peak::alu_rate_kernel<0><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
     else if (op == 1) peak::alu_rate_kernel<1><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
-    else peak::alu_rate_kernel<2><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
+    else if (op == 2) peak::alu_rate_kernel<2><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
+    else if (op == 3) peak::alu_rate_kernel<3><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
+    else if (op == 4) peak::alu_rate_kernel<4><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
+    else if (op == 5) peak::alu_rate_kernel<5><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
+    else peak::alu_rate_kernel<6><<<grid, peak::kAluThreads, 0, st>>>(iters, 1, sink_dev, cycles_dev);
     ++g_launches;
     return cuda_status(cudaGetLastError());
 }

@@ -79,7 +79,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) i8_mma_rate_kernel(int iters, 
 // cycles[blockIdx.x] = SM clocks of the loop (thread 0 of the block).
 constexpr int kAluThreads = 512;
 constexpr int kAluPerIter = 64;
-template <int OP>   // 0: mul.hi.s32, 1: mad.lo.s32, 2: fma.rn.f32
+// 0: mul.hi.s32, 1: mad.lo.s32, 2: fma.rn.f32, 3: mad.wide.s32 (the high word feeds the next one),
+// 4: cvt.pack.sat.u8.s32, 5: shr.s32, 6: fma.rn.f64
+template <int OP>
 __global__ void __launch_bounds__(kAluThreads, 2) alu_rate_kernel(int iters, int seed, int *sink, long long *cycles)
 {
     int r[8];
@@ -91,6 +93,11 @@ __global__ void __launch_bounds__(kAluThreads, 2) alu_rate_kernel(int iters, int
     }
     const int mult = 0x7FFFFFF1 - (int)(threadIdx.x & 7);
     const float fm = 0.999f, fa = 1e-3f;
+    double d[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) d[j] = 1.0 + (double)(threadIdx.x * 8 + j) * 1e-9;
+    const double dm = 0.999, da = 1e-3;
+    const long long add64 = (long long)seed << 33;
     __syncthreads();
     const long long t0 = clock64();
     for (int it = 0; it < iters; ++it) {
@@ -100,14 +107,22 @@ __global__ void __launch_bounds__(kAluThreads, 2) alu_rate_kernel(int iters, int
             for (int j = 0; j < 8; ++j) {
                 if (OP == 0) asm volatile("mul.hi.s32 %0, %0, %1;" : "+r"(r[j]) : "r"(mult));
                 else if (OP == 1) asm volatile("mad.lo.s32 %0, %0, %1, %1;" : "+r"(r[j]) : "r"(mult));
-                else asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[j]) : "f"(fm), "f"(fa));
+                else if (OP == 2) asm volatile("fma.rn.f32 %0, %0, %1, %2;" : "+f"(f[j]) : "f"(fm), "f"(fa));
+                else if (OP == 3)
+                    asm volatile("{\n\t.reg .b64 t;\n\t.reg .b32 lo;\n\t"
+                                 "mad.wide.s32 t, %0, %1, %2;\n\t"
+                                 "mov.b64 {lo, %0}, t;\n\t}"
+                                 : "+r"(r[j]) : "r"(mult), "l"(add64));
+                else if (OP == 4) asm volatile("cvt.pack.sat.u8.s32.b32 %0, %0, %1, %0;" : "+r"(r[j]) : "r"(mult));
+                else if (OP == 5) asm volatile("shr.s32 %0, %0, %1;" : "+r"(r[j]) : "r"(seed));
+                else asm volatile("fma.rn.f64 %0, %0, %1, %2;" : "+d"(d[j]) : "d"(dm), "d"(da));
             }
         }
     }
     const long long t1 = clock64();
     int acc = 0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc ^= r[j] ^ __float_as_int(f[j]);
+    for (int j = 0; j < 8; ++j) acc ^= r[j] ^ __float_as_int(f[j]) ^ __double2hiint(d[j]);
     if (acc == 0x12345678) *sink = acc;          // keeps the chains alive
     if (threadIdx.x == 0) cycles[blockIdx.x] = t1 - t0;
 }
